@@ -1,0 +1,203 @@
+/*
+ * ba.h -- C ABI of the Block-attention prefilling hot path for NVIDIA B200 (sm_100a).
+ *
+ * The library implements, as CUDA kernels, the three data-parallel steps of
+ * Block-attention inference (arXiv 2409.15355):
+ *
+ *   (a) position re-encoding of cached per-block keys         Section 2.3, Eq. 1-3
+ *   (b) the final block attending every cached block + itself Section 2.5, step 3
+ *   (c) block-diagonal prefill of all blocks in one launch    Section 1; Section 2.4
+ *
+ * plus the integer tables that describe a ragged prompt (Section 2.2, 2.5) and a
+ * flag that switches the same entry points to ordinary full causal attention
+ * (Section 3: the fine-tuned model runs under either mask).
+ *
+ * Conventions
+ * -----------
+ * - Tensors are DEVICE pointers owned by the caller, row-major
+ *   [tokens, heads, head_dim], bfloat16 unless stated, base address 16-byte
+ *   aligned, tokens packed without padding.
+ * - Three packings of a batch of prompts are used.  "prompt packing": every
+ *   block of every sequence in prompt order (n_tokens rows).  "cache packing":
+ *   only the non-final blocks, in the same order.  "final packing": only the
+ *   final block of every sequence, in sequence order.
+ * - Calls are asynchronous on `stream` (a cudaStream_t passed as void*; NULL is
+ *   the default stream).  Argument and launch errors are returned at once.
+ *   Problems only the device can see (inconsistent tables, a bounded wait that
+ *   ran out) are recorded in a status word read by ba_last_device_status().
+ * - Nothing is allocated after ba_create(); a workspace that is too small for a
+ *   call yields BA_ERR_WORKSPACE.  One context serves one stream at a time.
+ * - No C++ exceptions cross this boundary.  There is no CPU fallback: on a
+ *   machine without a usable sm_100 device ba_create() fails.
+ */
+#ifndef BA_H_
+#define BA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct ba_ctx ba_ctx; /* opaque */
+
+typedef enum {
+  BA_OK = 0,
+  BA_ERR_INVALID_ARG = 1, /* null / misaligned pointer, bad enum, inconsistent lengths */
+  BA_ERR_SHAPE = 2,       /* sizes that do not fit together */
+  BA_ERR_UNSUPPORTED = 3, /* head_dim not in {64,128}, n_q_heads % n_kv_heads != 0, ... */
+  BA_ERR_WORKSPACE = 4,   /* workspace given to ba_create too small for this call */
+  BA_ERR_CUDA = 5,        /* a CUDA runtime/driver call failed */
+  BA_ERR_TIMEOUT = 6      /* a bounded device-side wait expired */
+} ba_status;
+
+typedef enum { BA_MODE_BLOCK = 0, BA_MODE_FULL = 1 } ba_mode;
+
+/* Which coordinates form rotary pair m.  Eq. 1 draws 2x2 blocks on the diagonal,
+ * i.e. pairs (2m, 2m+1): BA_ROPE_ADJACENT.  BA_ROPE_HALF pairs (m, m + head_dim/2). */
+typedef enum { BA_ROPE_ADJACENT = 0, BA_ROPE_HALF = 1 } ba_rope_layout;
+
+typedef enum { BA_OUT_BF16 = 0, BA_OUT_F32 = 1 } ba_out_dtype;
+
+typedef struct {
+  int32_t n_q_heads;
+  int32_t n_kv_heads;    /* query head h reads KV head h / (n_q_heads / n_kv_heads) */
+  int32_t head_dim;      /* 64 or 128 */
+  int32_t rope_layout;   /* ba_rope_layout */
+  double rope_theta;     /* base of theta_m = base^(-2m/head_dim) */
+  float softmax_scale;   /* 0 selects 1/sqrt(head_dim) */
+  int32_t reserved;
+} ba_config;
+
+/*
+ * Tables of a ragged batch, produced by ba_segment().  The struct lives on the
+ * host; every pointer is a DEVICE pointer into the caller's table buffer.
+ * B = n_blocks, T = n_tokens, Bc = n_blocks - batch (each sequence has exactly
+ * one final block).
+ */
+typedef struct {
+  int32_t batch, n_blocks, n_tokens, n_cached_blocks;
+  int32_t mode;            /* ba_mode the tables were built for */
+  int32_t q_tile_tokens;   /* tokens per query tile of the attention kernels */
+  /* per sequence, [batch + 1] */
+  int32_t *cu_seq;         /* first row of the sequence, prompt packing */
+  int32_t *cu_cache_seq;   /* first row of the sequence, cache packing */
+  int32_t *cu_final_seq;   /* first row of the sequence, final packing */
+  int32_t *cu_seq_block;   /* index of the sequence's first block */
+  /* per block */
+  int32_t *cu_block;       /* [B+1] first row of the block, prompt packing */
+  int32_t *block_delta;    /* [B] prompt position of the block's first token = re-encoding delta */
+  int32_t *block_seq;      /* [B] sequence the block belongs to */
+  int32_t *block_kv_begin; /* [B] first key row (prompt packing) rows of this block may see */
+  int32_t *block_part_off; /* [B] first row of the block in cache packing (non-final) or final packing (final) */
+  uint8_t *block_is_final; /* [B] */
+  /* the non-final blocks, in order: the arguments of ba_reencode_k */
+  int32_t *cache_block;    /* [Bc] index of the block in the prompt */
+  int32_t *cache_cu;       /* [Bc+1] first row, cache packing */
+  int32_t *cache_delta;    /* [Bc] */
+  /* per token, [T] */
+  int32_t *tok_block;
+  int32_t *tok_pos;        /* position in the prompt (0-based within its sequence) */
+  int32_t *tok_pos_local;  /* position inside its block = position it has in the cache */
+  /* query-tile tables used by the attention kernels (not part of the bit-exact contract) */
+  int32_t *cu_qtile;       /* [B+1] */
+  int32_t *cu_ftile;       /* [batch+1] */
+  int32_t *totals;         /* [8]: cached tokens, final tokens, q tiles, final tiles, ..., [7] = validity word */
+} ba_segments;
+
+/* Create a context on CUDA device `device` and allocate `workspace_bytes` of
+ * scratch there (rotation tables, split-KV partial results).  Fails with
+ * BA_ERR_UNSUPPORTED for shapes outside the supported set and with BA_ERR_CUDA
+ * when the device is missing or is not compute capability 10.x. */
+ba_status ba_create(ba_ctx **ctx, const ba_config *cfg, int device, size_t workspace_bytes);
+ba_status ba_destroy(ba_ctx *ctx);
+const char *ba_status_string(ba_status s);
+
+/* Workspace ba_create() should be given so that calls of at most these sizes fit. */
+ba_status ba_workspace_bytes(const ba_config *cfg, int32_t max_blocks, int32_t max_q_rows, size_t *bytes);
+
+/* Synchronises the context's device and returns (then clears) the first
+ * problem a kernel recorded since the last call: BA_OK, BA_ERR_INVALID_ARG
+ * (tables inconsistent with the lengths given) or BA_ERR_TIMEOUT. */
+ba_status ba_last_device_status(ba_ctx *ctx);
+
+/* Number of this library's kernels launched through `ctx` so far. */
+int64_t ba_launch_count(const ba_ctx *ctx);
+
+/* Bytes of the table buffer ba_segment() needs for these sizes. */
+ba_status ba_segments_bytes(int32_t batch, int32_t n_blocks, int32_t n_tokens, size_t *bytes);
+
+/*
+ * Section 2.2 / 2.5: tables of a ragged batch from its block lengths.
+ *   block_lens  [n_blocks]  length of every block, prompt order; host or device memory
+ *   seq_nblocks [batch]     blocks per sequence (its last block is the final block); host or device
+ *   n_tokens                sum of block_lens (the caller sized its tensors with it)
+ *   mode                    BA_MODE_FULL makes every row see its whole sequence prefix
+ *                           (block_kv_begin = cu_seq); all other tables are unchanged
+ *   table_buf               device buffer of at least ba_segments_bytes() bytes, 16-byte aligned
+ *   out                     host struct, filled with pointers into table_buf
+ * With host arrays the lengths are checked before launching (BA_ERR_INVALID_ARG
+ * for a length < 1 or sums that do not match); with device arrays the same
+ * check runs on the device and is reported by ba_last_device_status().
+ */
+ba_status ba_segment(ba_ctx *ctx, const int32_t *block_lens, const int32_t *seq_nblocks,
+                     int32_t batch, int32_t n_blocks, int32_t n_tokens, ba_mode mode,
+                     void *table_buf, size_t table_bytes, ba_segments *out, void *stream);
+
+/*
+ * Section 2.3, Eq. 1-3: rotate cached keys from their cache positions to their
+ * positions in the new prompt.  For block c (0 <= c < n_blocks) and row t of it,
+ * every KV head and rotary pair m:
+ *     (x, y) <- (x cos(a) - y sin(a), x sin(a) + y cos(a)),  a = delta[c] * theta_m.
+ * A positive delta is Eq. 3 applied after Eq. 2 (the two collapse into one
+ * rotation by the difference, as Section 2.3 notes); a negative delta is Eq. 2
+ * (back to position zero, e.g. to fill the cache after a cold prefill); delta 0
+ * copies bit-exactly.
+ *   k_src    bf16 [n_src_rows, n_kv_heads, head_dim]; block c is read from row src_off[c], or
+ *            from row cu[c] when src_off is NULL.  A source row outside [0, n_src_rows) is
+ *            skipped and reported through ba_last_device_status() as BA_ERR_INVALID_ARG.
+ *   k_dst    bf16 [n_rows, n_kv_heads, head_dim]; block c is written to rows cu[c]..cu[c+1]-1.
+ *            May equal k_src when src_off is NULL (in place).
+ *   cu       device int32 [n_blocks+1], delta device int32 [n_blocks], src_off device int32 or NULL
+ *   n_rows   rows of k_dst (>= cu[n_blocks]); rows beyond cu[n_blocks] are not touched
+ * Uses n_blocks * head_dim * 4 bytes of workspace for the angle table.
+ */
+ba_status ba_reencode_k(ba_ctx *ctx, const void *k_src, const int32_t *src_off, int32_t n_src_rows,
+                        void *k_dst, const int32_t *cu, const int32_t *delta, int32_t n_blocks,
+                        int32_t n_rows, void *stream);
+
+/*
+ * Section 1 / Section 2.4: attention of a packed ragged batch under the
+ * Block-attention mask, all blocks in one launch.  Row i of block b sees key
+ * rows block_kv_begin[b] .. i (prompt packing).  q [T, n_q_heads, head_dim],
+ * k, v [T, n_kv_heads, head_dim] bf16 with RoPE already applied at tok_pos;
+ * o [T, n_q_heads, head_dim] bf16 or fp32; lse fp32 [T, n_q_heads] or NULL
+ * (natural-log softmax denominator).  `mode` must equal seg->mode.
+ */
+ba_status ba_block_prefill(ba_ctx *ctx, const void *q, const void *k, const void *v, void *o,
+                           float *lse, const ba_segments *seg, ba_mode mode,
+                           ba_out_dtype out_dtype, void *stream);
+
+/*
+ * Section 2.5, step 3: the final block of every sequence attends that
+ * sequence's cached blocks and itself (causally).
+ *   q_f, k_f, v_f   final packing, [n_final_rows, heads, head_dim] bf16, RoPE at prompt positions
+ *   k_cache         bf16 keys of the cached blocks at their PROMPT positions (the output
+ *                   of ba_reencode_k), cache packing, n_cache_rows rows
+ *   v_cache         bf16 values of the cached blocks: cache packing when v_src_off is NULL,
+ *                   else a pool of n_v_rows rows in which cached block c starts at v_src_off[c]
+ *   o               final packing, [n_final_rows, n_q_heads, head_dim]; lse [n_final_rows, n_q_heads] or NULL
+ * The mode flag does not change the result (final rows see the same keys under
+ * both masks) but must equal seg->mode.
+ */
+ba_status ba_final_attend(ba_ctx *ctx, const void *q_f, const void *k_f, const void *v_f,
+                          int32_t n_final_rows, const void *k_cache, const void *v_cache,
+                          int32_t n_cache_rows, const int32_t *v_src_off, int32_t n_v_rows,
+                          void *o, float *lse, const ba_segments *seg, ba_mode mode,
+                          ba_out_dtype out_dtype, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BA_H_ */

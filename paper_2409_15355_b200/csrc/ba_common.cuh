@@ -1,0 +1,67 @@
+// Internal declarations shared by the translation units of the library.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include <stddef.h>
+
+#include "ba.h"
+
+#define BA_CUDA_TRY(expr)                          \
+  do {                                             \
+    cudaError_t _e = (expr);                       \
+    if (_e != cudaSuccess) { return BA_ERR_CUDA; } \
+  } while (0)
+
+// Value of ba_segments::totals[7] once ba_segment's kernel has found the lengths consistent.
+#define BA_TABLES_VALID 0x600D
+
+// Context: configuration, workspace and the device status word.
+struct ba_ctx {
+  ba_config cfg;
+  int device;
+  int sm_count;
+  float scale;              // softmax scale actually used
+  void *workspace;          // device
+  size_t workspace_bytes;
+  int32_t *dev_status;      // device word: first non-zero ba_status recorded by a kernel
+  int64_t launches;
+};
+
+static inline size_t ba_align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// Records the first device-side problem; later ones are dropped.
+__device__ __forceinline__ void ba_record_status(int32_t *status, int32_t code) {
+  atomicCAS(status, 0, code);
+}
+
+// Entry points implemented in the individual .cu files.
+ba_status ba_segment_launch(ba_ctx *ctx, const int32_t *d_block_lens, const int32_t *d_seq_nblocks,
+                            int32_t batch, int32_t n_blocks, int32_t n_tokens, int mode,
+                            const ba_segments *seg, cudaStream_t stream);
+
+ba_status ba_reencode_launch(ba_ctx *ctx, const void *k_src, const int32_t *src_off,
+                             int32_t n_src_rows, void *k_dst, const int32_t *cu,
+                             const int32_t *delta, int32_t n_blocks, int32_t n_rows, float2 *table,
+                             cudaStream_t stream);
+
+struct ba_attend_args {
+  // queries / outputs: rows of the q packing (prompt packing for prefill, final packing for final attend)
+  const __nv_bfloat16 *q;
+  void *o;
+  float *lse;
+  int32_t n_q_rows;
+  int out_f32;
+  // primary keys/values: same packing as q (prefill: the whole prompt; final attend: the final blocks)
+  const __nv_bfloat16 *k, *v;
+  int32_t n_kv_rows;
+  // cached keys/values (final attend only)
+  const __nv_bfloat16 *k_cache, *v_cache;
+  int32_t n_cache_rows, n_v_rows;
+  const int32_t *v_src_off;
+  int final_only;  // 1: ba_final_attend, 0: ba_block_prefill
+};
+
+ba_status ba_attend_launch(ba_ctx *ctx, const ba_attend_args &a, const ba_segments *seg,
+                           cudaStream_t stream);
