@@ -1,0 +1,277 @@
+// Host side of the C ABI: argument checks, table-buffer layout, workspace
+// bookkeeping and dispatch to the kernels.  No kernel code lives here.
+#include <new>
+#include <string.h>
+
+#include "ba_common.cuh"
+
+ba_status ba_attend_simt_launch(ba_ctx *ctx, const ba_attend_args &a, const ba_segments *seg,
+                                cudaStream_t stream);
+
+namespace {
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Is `p` ordinary host memory (to be staged), as opposed to device-visible memory?
+bool is_host_pointer(const void *p) {
+  cudaPointerAttributes at;
+  cudaError_t e = cudaPointerGetAttributes(&at, p);
+  if (e != cudaSuccess) { cudaGetLastError(); return true; }
+  return at.type == cudaMemoryTypeUnregistered || at.type == cudaMemoryTypeHost;
+}
+
+ba_status check_config(const ba_config *c) {
+  if (!c) return BA_ERR_INVALID_ARG;
+  if (c->head_dim != 64 && c->head_dim != 128) return BA_ERR_UNSUPPORTED;
+  if (c->n_q_heads < 1 || c->n_kv_heads < 1 || c->n_q_heads % c->n_kv_heads) return BA_ERR_UNSUPPORTED;
+  if (c->rope_layout != BA_ROPE_ADJACENT && c->rope_layout != BA_ROPE_HALF) return BA_ERR_INVALID_ARG;
+  if (!(c->rope_theta > 1.0)) return BA_ERR_INVALID_ARG;
+  if (c->softmax_scale < 0.f) return BA_ERR_INVALID_ARG;
+  return BA_OK;
+}
+
+// Tokens per query tile of the attention kernels.
+int q_tile_tokens(const ba_config &c) {
+  (void)c;
+  return 128;
+}
+
+// Start of the workspace: staging of host-side length arrays.
+size_t stage_bytes_for(int32_t max_blocks) { return ba_align_up((size_t)(2 * (size_t)max_blocks + 64) * 4, 256); }
+
+struct TableLayout {
+  size_t off[20];
+  size_t bytes;
+};
+
+// Carves the caller's table buffer.  Every array starts on a 16-byte boundary.
+TableLayout table_layout(int32_t batch, int32_t B, int32_t T) {
+  TableLayout L;
+  size_t cur = 0;
+  int i = 0;
+  auto take = [&](size_t n_bytes) { L.off[i++] = cur; cur = ba_align_up(cur + n_bytes, 16); };
+  for (int k = 0; k < 4; ++k) take((size_t)(batch + 1) * 4);  // cu_seq, cu_cache_seq, cu_final_seq, cu_seq_block
+  take((size_t)(B + 1) * 4);                                  // cu_block
+  for (int k = 0; k < 4; ++k) take((size_t)B * 4);            // block_delta, block_seq, block_kv_begin, block_part_off
+  take((size_t)B);                                            // block_is_final
+  take((size_t)B * 4);                                        // cache_block
+  take((size_t)(B + 1) * 4);                                  // cache_cu
+  take((size_t)B * 4);                                        // cache_delta
+  for (int k = 0; k < 3; ++k) take((size_t)T * 4);            // tok_block, tok_pos, tok_pos_local
+  take((size_t)(B + 1) * 4);                                  // cu_qtile
+  take((size_t)(batch + 1) * 4);                              // cu_ftile
+  take(8 * 4);                                                // totals
+  L.bytes = cur;
+  return L;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char *ba_status_string(ba_status s) {
+  switch (s) {
+    case BA_OK: return "ok";
+    case BA_ERR_INVALID_ARG: return "invalid argument";
+    case BA_ERR_SHAPE: return "shape mismatch";
+    case BA_ERR_UNSUPPORTED: return "unsupported configuration";
+    case BA_ERR_WORKSPACE: return "workspace too small";
+    case BA_ERR_CUDA: return "CUDA error";
+    case BA_ERR_TIMEOUT: return "device-side wait timed out";
+  }
+  return "unknown status";
+}
+
+ba_status ba_workspace_bytes(const ba_config *cfg, int32_t max_blocks, int32_t max_q_rows, size_t *bytes) {
+  ba_status st = check_config(cfg);
+  if (st != BA_OK) return st;
+  if (!bytes || max_blocks < 1 || max_q_rows < 0) return BA_ERR_INVALID_ARG;
+  size_t table = ba_align_up((size_t)max_blocks * cfg->head_dim * 4, 256);
+  *bytes = stage_bytes_for(max_blocks) + table + 256;
+  return BA_OK;
+}
+
+ba_status ba_create(ba_ctx **out, const ba_config *cfg, int device, size_t workspace_bytes) {
+  if (!out) return BA_ERR_INVALID_ARG;
+  *out = nullptr;
+  ba_status st = check_config(cfg);
+  if (st != BA_OK) return st;
+  int n_dev = 0;
+  if (cudaGetDeviceCount(&n_dev) != cudaSuccess || device < 0 || device >= n_dev) {
+    cudaGetLastError();
+    return BA_ERR_CUDA;
+  }
+  cudaDeviceProp prop;
+  BA_CUDA_TRY(cudaGetDeviceProperties(&prop, device));
+  if (prop.major != 10) return BA_ERR_CUDA;  // kernels are built for sm_100a only
+  BA_CUDA_TRY(cudaSetDevice(device));
+  ba_ctx *ctx = new (std::nothrow) ba_ctx();
+  if (!ctx) return BA_ERR_CUDA;
+  ctx->cfg = *cfg;
+  ctx->device = device;
+  ctx->sm_count = prop.multiProcessorCount;
+  ctx->scale = cfg->softmax_scale > 0.f ? cfg->softmax_scale : 1.0f / sqrtf((float)cfg->head_dim);
+  ctx->workspace_bytes = workspace_bytes;
+  ctx->launches = 0;
+  ctx->workspace = nullptr;
+  ctx->dev_status = nullptr;
+  if (cudaMalloc(&ctx->dev_status, 256) != cudaSuccess ||
+      cudaMemset(ctx->dev_status, 0, 256) != cudaSuccess ||
+      (workspace_bytes && cudaMalloc(&ctx->workspace, workspace_bytes) != cudaSuccess)) {
+    cudaGetLastError();
+    if (ctx->dev_status) cudaFree(ctx->dev_status);
+    delete ctx;
+    return BA_ERR_CUDA;
+  }
+  *out = ctx;
+  return BA_OK;
+}
+
+ba_status ba_destroy(ba_ctx *ctx) {
+  if (!ctx) return BA_ERR_INVALID_ARG;
+  cudaSetDevice(ctx->device);
+  cudaDeviceSynchronize();
+  if (ctx->workspace) cudaFree(ctx->workspace);
+  if (ctx->dev_status) cudaFree(ctx->dev_status);
+  delete ctx;
+  return BA_OK;
+}
+
+ba_status ba_last_device_status(ba_ctx *ctx) {
+  if (!ctx) return BA_ERR_INVALID_ARG;
+  BA_CUDA_TRY(cudaSetDevice(ctx->device));
+  BA_CUDA_TRY(cudaDeviceSynchronize());
+  int32_t h = 0;
+  BA_CUDA_TRY(cudaMemcpy(&h, ctx->dev_status, 4, cudaMemcpyDeviceToHost));
+  if (h != 0) BA_CUDA_TRY(cudaMemset(ctx->dev_status, 0, 4));
+  return (ba_status)h;
+}
+
+int64_t ba_launch_count(const ba_ctx *ctx) { return ctx ? ctx->launches : 0; }
+
+ba_status ba_segments_bytes(int32_t batch, int32_t n_blocks, int32_t n_tokens, size_t *bytes) {
+  if (!bytes || batch < 1 || n_blocks < batch || n_tokens < n_blocks) return BA_ERR_INVALID_ARG;
+  *bytes = table_layout(batch, n_blocks, n_tokens).bytes;
+  return BA_OK;
+}
+
+ba_status ba_segment(ba_ctx *ctx, const int32_t *block_lens, const int32_t *seq_nblocks,
+                     int32_t batch, int32_t n_blocks, int32_t n_tokens, ba_mode mode,
+                     void *table_buf, size_t table_bytes, ba_segments *out, void *stream) {
+  if (!ctx || !block_lens || !seq_nblocks || !table_buf || !out) return BA_ERR_INVALID_ARG;
+  if (mode != BA_MODE_BLOCK && mode != BA_MODE_FULL) return BA_ERR_INVALID_ARG;
+  if (batch < 1 || n_blocks < batch || n_tokens < n_blocks) return BA_ERR_INVALID_ARG;
+  if (!aligned16(table_buf)) return BA_ERR_INVALID_ARG;
+  TableLayout L = table_layout(batch, n_blocks, n_tokens);
+  if (table_bytes < L.bytes) return BA_ERR_SHAPE;
+  BA_CUDA_TRY(cudaSetDevice(ctx->device));
+  cudaStream_t s = (cudaStream_t)stream;
+
+  const int32_t *d_lens = block_lens, *d_nb = seq_nblocks;
+  const bool host_lens = is_host_pointer(block_lens), host_nb = is_host_pointer(seq_nblocks);
+  if (host_lens != host_nb) return BA_ERR_INVALID_ARG;
+  if (host_lens) {
+    long long sum = 0, nb_sum = 0;
+    for (int b = 0; b < n_blocks; ++b) { if (block_lens[b] < 1) return BA_ERR_INVALID_ARG; sum += block_lens[b]; }
+    for (int q = 0; q < batch; ++q) { if (seq_nblocks[q] < 1) return BA_ERR_INVALID_ARG; nb_sum += seq_nblocks[q]; }
+    if (sum != n_tokens || nb_sum != n_blocks) return BA_ERR_INVALID_ARG;
+    size_t need = (size_t)(n_blocks + batch) * 4;
+    if (!ctx->workspace || need > ctx->workspace_bytes) return BA_ERR_WORKSPACE;
+    int32_t *stage = (int32_t *)ctx->workspace;
+    BA_CUDA_TRY(cudaMemcpyAsync(stage, block_lens, (size_t)n_blocks * 4, cudaMemcpyHostToDevice, s));
+    BA_CUDA_TRY(cudaMemcpyAsync(stage + n_blocks, seq_nblocks, (size_t)batch * 4, cudaMemcpyHostToDevice, s));
+    d_lens = stage;
+    d_nb = stage + n_blocks;
+  }
+
+  char *base = (char *)table_buf;
+  int i = 0;
+  memset(out, 0, sizeof(*out));
+  out->batch = batch; out->n_blocks = n_blocks; out->n_tokens = n_tokens;
+  out->n_cached_blocks = n_blocks - batch;
+  out->mode = mode;
+  out->q_tile_tokens = q_tile_tokens(ctx->cfg);
+  auto next = [&]() { return (int32_t *)(base + L.off[i++]); };
+  out->cu_seq = next(); out->cu_cache_seq = next(); out->cu_final_seq = next(); out->cu_seq_block = next();
+  out->cu_block = next();
+  out->block_delta = next(); out->block_seq = next(); out->block_kv_begin = next(); out->block_part_off = next();
+  out->block_is_final = (uint8_t *)next();
+  out->cache_block = next(); out->cache_cu = next(); out->cache_delta = next();
+  out->tok_block = next(); out->tok_pos = next(); out->tok_pos_local = next();
+  out->cu_qtile = next(); out->cu_ftile = next(); out->totals = next();
+  return ba_segment_launch(ctx, d_lens, d_nb, batch, n_blocks, n_tokens, mode, out, s);
+}
+
+ba_status ba_reencode_k(ba_ctx *ctx, const void *k_src, const int32_t *src_off, int32_t n_src_rows,
+                        void *k_dst, const int32_t *cu, const int32_t *delta, int32_t n_blocks,
+                        int32_t n_rows, void *stream) {
+  if (!ctx || !k_src || !k_dst || !cu || !delta) return BA_ERR_INVALID_ARG;
+  if (n_blocks < 0 || n_rows < 0 || n_src_rows < 0) return BA_ERR_INVALID_ARG;
+  if (!aligned16(k_src) || !aligned16(k_dst)) return BA_ERR_INVALID_ARG;
+  if (k_src == k_dst && src_off) return BA_ERR_INVALID_ARG;  // a gather cannot run in place
+  if (n_blocks == 0 || n_rows == 0) return BA_OK;
+  BA_CUDA_TRY(cudaSetDevice(ctx->device));
+  // scratch: the angle table at the end of the workspace (the staging area is at its start)
+  size_t need = ba_align_up((size_t)n_blocks * ctx->cfg.head_dim * 4, 256);  // n_blocks * d/2 * sizeof(float2)
+  if (!ctx->workspace || need > ctx->workspace_bytes) return BA_ERR_WORKSPACE;
+  float2 *table = (float2 *)((char *)ctx->workspace + (ctx->workspace_bytes - need) / 256 * 256);
+  return ba_reencode_launch(ctx, k_src, src_off, n_src_rows, k_dst, cu, delta, n_blocks, n_rows, table,
+                            (cudaStream_t)stream);
+}
+
+static ba_status check_attend_common(ba_ctx *ctx, const void *q, const void *k, const void *v, void *o,
+                                     const ba_segments *seg, ba_mode mode, ba_out_dtype od) {
+  if (!ctx || !q || !k || !v || !o || !seg) return BA_ERR_INVALID_ARG;
+  if (mode != BA_MODE_BLOCK && mode != BA_MODE_FULL) return BA_ERR_INVALID_ARG;
+  if ((int)mode != seg->mode) return BA_ERR_INVALID_ARG;
+  if (od != BA_OUT_BF16 && od != BA_OUT_F32) return BA_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o)) return BA_ERR_INVALID_ARG;
+  if (!seg->totals || !seg->cu_block || !seg->tok_block) return BA_ERR_INVALID_ARG;
+  return BA_OK;
+}
+
+ba_status ba_block_prefill(ba_ctx *ctx, const void *q, const void *k, const void *v, void *o,
+                           float *lse, const ba_segments *seg, ba_mode mode,
+                           ba_out_dtype out_dtype, void *stream) {
+  ba_status st = check_attend_common(ctx, q, k, v, o, seg, mode, out_dtype);
+  if (st != BA_OK) return st;
+  BA_CUDA_TRY(cudaSetDevice(ctx->device));
+  ba_attend_args a;
+  memset(&a, 0, sizeof(a));
+  a.q = (const __nv_bfloat16 *)q; a.k = (const __nv_bfloat16 *)k; a.v = (const __nv_bfloat16 *)v;
+  a.o = o; a.lse = lse; a.n_q_rows = seg->n_tokens; a.n_kv_rows = seg->n_tokens;
+  a.out_f32 = out_dtype == BA_OUT_F32;
+  a.final_only = 0;
+  return ba_attend_launch(ctx, a, seg, (cudaStream_t)stream);
+}
+
+ba_status ba_final_attend(ba_ctx *ctx, const void *q_f, const void *k_f, const void *v_f,
+                          int32_t n_final_rows, const void *k_cache, const void *v_cache,
+                          int32_t n_cache_rows, const int32_t *v_src_off, int32_t n_v_rows,
+                          void *o, float *lse, const ba_segments *seg, ba_mode mode,
+                          ba_out_dtype out_dtype, void *stream) {
+  ba_status st = check_attend_common(ctx, q_f, k_f, v_f, o, seg, mode, out_dtype);
+  if (st != BA_OK) return st;
+  if (n_final_rows < 0 || n_cache_rows < 0) return BA_ERR_INVALID_ARG;
+  if (n_cache_rows > 0 && (!k_cache || !v_cache || !aligned16(k_cache) || !aligned16(v_cache)))
+    return BA_ERR_INVALID_ARG;
+  if (v_src_off && n_v_rows < 1) return BA_ERR_INVALID_ARG;
+  BA_CUDA_TRY(cudaSetDevice(ctx->device));
+  ba_attend_args a;
+  memset(&a, 0, sizeof(a));
+  a.q = (const __nv_bfloat16 *)q_f; a.k = (const __nv_bfloat16 *)k_f; a.v = (const __nv_bfloat16 *)v_f;
+  a.o = o; a.lse = lse; a.n_q_rows = n_final_rows; a.n_kv_rows = n_final_rows;
+  a.k_cache = (const __nv_bfloat16 *)k_cache; a.v_cache = (const __nv_bfloat16 *)v_cache;
+  a.n_cache_rows = n_cache_rows; a.n_v_rows = v_src_off ? n_v_rows : n_cache_rows;
+  a.v_src_off = v_src_off;
+  a.out_f32 = out_dtype == BA_OUT_F32;
+  a.final_only = 1;
+  return ba_attend_launch(ctx, a, seg, (cudaStream_t)stream);
+}
+
+}  // extern "C"
+
+ba_status ba_attend_launch(ba_ctx *ctx, const ba_attend_args &a, const ba_segments *seg,
+                           cudaStream_t stream) {
+  return ba_attend_simt_launch(ctx, a, seg, stream);
+}
