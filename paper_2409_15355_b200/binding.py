@@ -1,0 +1,176 @@
+"""ctypes binding of the C ABI declared in include/ba.h.
+
+Argument marshalling only: every step of the path runs in the CUDA library.
+Tensors are torch CUDA tensors (torch is used for device memory and streams);
+their data pointers are handed to the library unchanged.  There is no CPU
+fallback: loading fails loudly when the library is missing, and ba_create fails
+when no sm_100 device is present.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional
+
+from . import build as _build
+
+BA_OK = 0
+BA_ERR_INVALID_ARG, BA_ERR_SHAPE, BA_ERR_UNSUPPORTED, BA_ERR_WORKSPACE, BA_ERR_CUDA, BA_ERR_TIMEOUT = range(1, 7)
+BA_MODE_BLOCK, BA_MODE_FULL = 0, 1
+BA_ROPE_ADJACENT, BA_ROPE_HALF = 0, 1
+BA_OUT_BF16, BA_OUT_F32 = 0, 1
+
+EXPORTS = [
+    "ba_create", "ba_destroy", "ba_status_string", "ba_workspace_bytes", "ba_last_device_status",
+    "ba_launch_count", "ba_segments_bytes", "ba_segment", "ba_reencode_k", "ba_block_prefill",
+    "ba_final_attend",
+]
+
+
+class ba_config(C.Structure):
+    _fields_ = [("n_q_heads", C.c_int32), ("n_kv_heads", C.c_int32), ("head_dim", C.c_int32),
+                ("rope_layout", C.c_int32), ("rope_theta", C.c_double), ("softmax_scale", C.c_float),
+                ("reserved", C.c_int32)]
+
+
+class ba_segments(C.Structure):
+    _fields_ = [("batch", C.c_int32), ("n_blocks", C.c_int32), ("n_tokens", C.c_int32),
+                ("n_cached_blocks", C.c_int32), ("mode", C.c_int32), ("q_tile_tokens", C.c_int32)] + [
+        (n, C.c_void_p) for n in (
+            "cu_seq", "cu_cache_seq", "cu_final_seq", "cu_seq_block", "cu_block", "block_delta",
+            "block_seq", "block_kv_begin", "block_part_off", "block_is_final", "cache_block",
+            "cache_cu", "cache_delta", "tok_block", "tok_pos", "tok_pos_local", "cu_qtile",
+            "cu_ftile", "totals")]
+
+
+class BaError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} (ba_status {status})")
+
+
+_lib = None
+
+
+def load_library(path: Optional[str] = None) -> C.CDLL:
+    """dlopen libba.so (building it first if its sources changed) and declare prototypes."""
+    global _lib
+    if _lib is not None and path is None:
+        return _lib
+    if path is None:
+        path = _build.build()
+    if not os.path.exists(path):
+        raise FileNotFoundError(f"CUDA library not found: {path}")
+    lib = C.CDLL(path)
+    vp, i32, sz = C.c_void_p, C.c_int32, C.c_size_t
+    lib.ba_create.argtypes = [C.POINTER(vp), C.POINTER(ba_config), C.c_int, sz]
+    lib.ba_destroy.argtypes = [vp]
+    lib.ba_status_string.argtypes = [C.c_int]
+    lib.ba_status_string.restype = C.c_char_p
+    lib.ba_workspace_bytes.argtypes = [C.POINTER(ba_config), i32, i32, C.POINTER(sz)]
+    lib.ba_last_device_status.argtypes = [vp]
+    lib.ba_launch_count.argtypes = [vp]
+    lib.ba_launch_count.restype = C.c_int64
+    lib.ba_segments_bytes.argtypes = [i32, i32, i32, C.POINTER(sz)]
+    lib.ba_segment.argtypes = [vp, vp, vp, i32, i32, i32, C.c_int, vp, sz, C.POINTER(ba_segments), vp]
+    lib.ba_reencode_k.argtypes = [vp, vp, vp, i32, vp, vp, vp, i32, i32, vp]
+    lib.ba_block_prefill.argtypes = [vp, vp, vp, vp, vp, vp, C.POINTER(ba_segments), C.c_int, C.c_int, vp]
+    lib.ba_final_attend.argtypes = [vp, vp, vp, vp, i32, vp, vp, i32, vp, i32, vp, vp,
+                                    C.POINTER(ba_segments), C.c_int, C.c_int, vp]
+    for name in EXPORTS:
+        if name not in ("ba_status_string", "ba_launch_count"):
+            getattr(lib, name).restype = C.c_int
+    _lib = lib
+    return lib
+
+
+def status_string(status: int) -> str:
+    return load_library().ba_status_string(int(status)).decode()
+
+
+def _check(status: int, where: str):
+    if status != BA_OK:
+        raise BaError(status, where)
+
+
+def _ptr(t) -> Optional[int]:
+    """Address of a torch tensor / numpy array / raw address / None."""
+    if t is None or isinstance(t, int):
+        return t
+    if hasattr(t, "data_ptr"):
+        if not t.is_contiguous():
+            raise ValueError("tensor must be contiguous")
+        return t.data_ptr()
+    return t.ctypes.data  # numpy (host arrays of lengths)
+
+
+def _stream_ptr(stream) -> Optional[int]:
+    if stream is None:
+        import torch
+        stream = torch.cuda.current_stream()
+    return stream.cuda_stream or None
+
+
+# ---------------------------------------------------------------------------
+# Same names as the C entry points
+# ---------------------------------------------------------------------------
+def ba_workspace_bytes(cfg: ba_config, max_blocks: int, max_q_rows: int) -> int:
+    out = C.c_size_t(0)
+    _check(load_library().ba_workspace_bytes(C.byref(cfg), max_blocks, max_q_rows, C.byref(out)),
+           "ba_workspace_bytes")
+    return out.value
+
+
+def ba_create(cfg: ba_config, device: int, workspace_bytes: int) -> C.c_void_p:
+    ctx = C.c_void_p()
+    _check(load_library().ba_create(C.byref(ctx), C.byref(cfg), device, workspace_bytes), "ba_create")
+    return ctx
+
+
+def ba_destroy(ctx) -> None:
+    _check(load_library().ba_destroy(ctx), "ba_destroy")
+
+
+def ba_last_device_status(ctx) -> int:
+    return load_library().ba_last_device_status(ctx)
+
+
+def ba_launch_count(ctx) -> int:
+    return int(load_library().ba_launch_count(ctx))
+
+
+def ba_segments_bytes(batch: int, n_blocks: int, n_tokens: int) -> int:
+    out = C.c_size_t(0)
+    _check(load_library().ba_segments_bytes(batch, n_blocks, n_tokens, C.byref(out)), "ba_segments_bytes")
+    return out.value
+
+
+def ba_segment(ctx, block_lens, seq_nblocks, batch, n_blocks, n_tokens, mode, table_buf, stream=None):
+    """block_lens / seq_nblocks: int32 numpy arrays (host) or torch CUDA tensors.
+    table_buf: torch uint8 CUDA tensor of at least ba_segments_bytes() bytes.  Returns ba_segments."""
+    seg = ba_segments()
+    _check(load_library().ba_segment(ctx, _ptr(block_lens), _ptr(seq_nblocks), batch, n_blocks, n_tokens,
+                                     mode, _ptr(table_buf), table_buf.numel() * table_buf.element_size(),
+                                     C.byref(seg), _stream_ptr(stream)), "ba_segment")
+    return seg
+
+
+def ba_reencode_k(ctx, k_src, src_off, n_src_rows, k_dst, cu, delta, n_blocks, n_rows, stream=None):
+    """cu / delta / src_off: device addresses (ints, e.g. seg.cache_cu) or torch int32 CUDA tensors."""
+    _check(load_library().ba_reencode_k(ctx, _ptr(k_src), _ptr(src_off), n_src_rows, _ptr(k_dst),
+                                        _ptr(cu), _ptr(delta), n_blocks, n_rows, _stream_ptr(stream)),
+           "ba_reencode_k")
+
+
+def ba_block_prefill(ctx, q, k, v, o, lse, seg, mode, out_dtype, stream=None):
+    _check(load_library().ba_block_prefill(ctx, _ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(lse),
+                                           C.byref(seg), mode, out_dtype, _stream_ptr(stream)),
+           "ba_block_prefill")
+
+
+def ba_final_attend(ctx, q_f, k_f, v_f, n_final_rows, k_cache, v_cache, n_cache_rows, v_src_off,
+                    n_v_rows, o, lse, seg, mode, out_dtype, stream=None):
+    _check(load_library().ba_final_attend(ctx, _ptr(q_f), _ptr(k_f), _ptr(v_f), n_final_rows,
+                                          _ptr(k_cache), _ptr(v_cache), n_cache_rows, _ptr(v_src_off),
+                                          n_v_rows, _ptr(o), _ptr(lse), C.byref(seg), mode, out_dtype,
+                                          _stream_ptr(stream)), "ba_final_attend")
