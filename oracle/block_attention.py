@@ -124,13 +124,14 @@ def segment_tables(block_lens, seq_nblocks, mode=MODE_BLOCK):
 # ---------------------------------------------------------------------------
 # The explicit mask (Section 1, Section 2.1, Section 2.4)
 # ---------------------------------------------------------------------------
-def mask_rows(block_lens, seq_nblocks, mode, rows):
+def mask_rows(block_lens, seq_nblocks, mode, rows, cols=None):
     """Rows `rows` of the dense 0/1 mask over the packed batch, as bool [n, T].
 
     M[i, j] = 1 iff j is in the same sequence as i, j <= i, and either the
     mode is full attention, or block(j) == block(i), or block(i) is its
     sequence's final block.  Written from the block lists directly (not from
     block_kv_begin) so that the tables and the mask pin one another.
+    `cols` = (c0, c1) restricts the result to key columns c0..c1-1.
     """
     block_lens = [int(x) for x in block_lens]
     T = sum(block_lens)
@@ -140,11 +141,12 @@ def mask_rows(block_lens, seq_nblocks, mode, rows):
     last_block_of_seq = np.cumsum(seq_nblocks) - 1
     is_final_tok = (blk == last_block_of_seq[seq])
     rows = np.asarray(rows, dtype=np.int64)
-    j = np.arange(T)[None, :]
+    c0, c1 = (0, T) if cols is None else cols
+    j = np.arange(c0, c1)[None, :]
     i = rows[:, None]
-    m = (seq[None, :] == seq[rows][:, None]) & (j <= i)
+    m = (seq[None, c0:c1] == seq[rows][:, None]) & (j <= i)
     if mode == MODE_BLOCK:
-        m &= (blk[None, :] == blk[rows][:, None]) | is_final_tok[rows][:, None]
+        m &= (blk[None, c0:c1] == blk[rows][:, None]) | is_final_tok[rows][:, None]
     return m
 
 
@@ -288,16 +290,21 @@ def block_prefill(q, k, v, block_lens, seq_nblocks, mode, rows=None, scale=None)
     rows = np.asarray(rows, dtype=np.int64)
     o = np.empty((len(rows),) + tuple(np.shape(q)[1:]), dtype=np.float64)
     lse = np.empty((len(rows), np.shape(q)[1]), dtype=np.float64)
-    step = 2048
-    qf = np.asarray(q)
-    for lo in range(0, len(rows), step):
-        r = rows[lo:lo + step]
-        m = mask_rows(block_lens, seq_nblocks, mode, r)
-        # keys outside the rows' sequences are masked anyway; trim columns for speed
-        cols = np.flatnonzero(m.any(axis=0))
-        c0, c1 = (int(cols[0]), int(cols[-1]) + 1) if len(cols) else (0, 1)
-        o[lo:lo + step], lse[lo:lo + step] = attention_rows(
-            qf[r], np.asarray(k)[c0:c1], np.asarray(v)[c0:c1], m[:, c0:c1], scale)
+    # rows are handled sequence by sequence: keys of other sequences are masked for
+    # every row, so only the sequence's own key columns are materialised
+    cu_seq = np.concatenate([[0], np.cumsum([sum(int(x) for x in block_lens[a:b]) for a, b in zip(
+        np.concatenate([[0], np.cumsum(seq_nblocks)[:-1]]), np.cumsum(seq_nblocks))])])
+    seq_of_row = np.searchsorted(cu_seq, rows, side="right") - 1
+    step = 1024
+    qf, kf, vf = np.asarray(q), np.asarray(k), np.asarray(v)
+    for s in np.unique(seq_of_row):
+        sel = np.flatnonzero(seq_of_row == s)
+        c0, c1 = int(cu_seq[s]), int(cu_seq[s + 1])
+        for lo in range(0, len(sel), step):
+            idx = sel[lo:lo + step]
+            r = rows[idx]
+            m = mask_rows(block_lens, seq_nblocks, mode, r, cols=(c0, c1))
+            o[idx], lse[idx] = attention_rows(qf[r], kf[c0:c1], vf[c0:c1], m, scale)
     return o, lse
 
 

@@ -383,10 +383,11 @@ def test_pins_catch_planted_mistakes(monkeypatch):
     # final block forgets the earlier blocks
     good_mask = ob.mask_rows
 
-    def bad_mask(block_lens, seq_nblocks, mode, rows):
-        m = good_mask(block_lens, seq_nblocks, ob.MODE_FULL, rows)
+    def bad_mask(block_lens, seq_nblocks, mode, rows, cols=None):
+        m = good_mask(block_lens, seq_nblocks, ob.MODE_FULL, rows, cols)
         blk = np.repeat(np.arange(len(block_lens)), block_lens)
-        return m & (blk[None, :] == blk[np.asarray(rows)][:, None]) if mode == ob.MODE_BLOCK else m
+        c0, c1 = (0, len(blk)) if cols is None else cols
+        return m & (blk[None, c0:c1] == blk[np.asarray(rows)][:, None]) if mode == ob.MODE_BLOCK else m
     monkeypatch.setattr(ob, "mask_rows", bad_mask)
     assert _fails(test_brute_force_tiny, seqs, ob.MODE_BLOCK)
     assert _fails(test_zero_queries_give_prefix_means)
