@@ -1,0 +1,341 @@
+#!/usr/bin/env python
+"""Benchmark of the Block-attention warm path at 32K context.
+
+One step = one pass of the hot path over a 32768-token prompt (32 cached
+passages of 1000 tokens + a 768-token final block, Llama-3-8B attention shape):
+ba_segment once, then for each of 32 layers ba_reencode_k (cached K to prompt
+positions) and ba_final_attend (final block over re-encoded cache + itself),
+every layer with its own seeded K/V/Q.  The metric is microseconds per layer.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+Prints one JSON line.  With N > 1 (torchrun) every rank runs an independent
+replica of the same job (the path has no exchange step); the reported value is
+the time per layer-job over all replicas.  --impl reference times the fp64 CPU
+oracle on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "final-block attend+reencode us/layer at 32K ctx"
+UNIT = "us/layer"
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return dict(hbm_gbs=d["hbm_gbs"], bf16_tflops=d["bf16_tflops"],
+                    bf16_tflops_sustained=d.get("bf16_tflops_sustained"), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+# --------------------------------------------------------------------------- clocks
+class ClockSampler:
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100", "-i", str(self.gpu)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            out = ""
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.strip().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None,
+                "sm_max_mhz": max(mx) if mx else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# --------------------------------------------------------------------------- distributed plumbing
+def dist_env():
+    return int(os.environ.get("RANK", 0)), int(os.environ.get("LOCAL_RANK", 0)), int(os.environ.get("WORLD_SIZE", 1))
+
+
+def max_over_ranks(value: float, device=None) -> float:
+    """Max of a host scalar over all ranks (identity without a process group)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()):
+        return value
+    t = torch.tensor([value], dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def sum_over_ranks(value: float, device=None) -> float:
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()):
+        return value
+    t = torch.tensor([value], dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.SUM)
+    return float(t.item())
+
+
+def aggregate(ms_local: float, layer_jobs_local: float, device=None):
+    """Replica aggregation: the job takes as long as its slowest rank; the work
+    done is the sum over ranks.  Returns (ms, us per layer-job over all ranks)."""
+    ms = max_over_ranks(ms_local, device)
+    jobs = sum_over_ranks(layer_jobs_local, device)
+    return ms, ms * 1e3 / jobs
+
+
+# --------------------------------------------------------------------------- the oracle legs
+def oracle_layer_sample(w, n_rows: int, layer: int = 0):
+    """Time the fp64 oracle on one layer: re-encode of all cached blocks plus
+    final attend for the first `n_rows` rows of the final block; scale the
+    attend part to the whole final block.  Returns microseconds per layer."""
+    from oracle import block_attention as ob
+    from paper_2409_15355_b200 import workloads as W
+    x = W.warm_inputs(w, layer)
+    t = ob.segment_tables(w.block_lens, w.seq_nblocks)
+    Lf = w.final_lens()[0]
+    n_rows = min(n_rows, Lf)
+    kc, vc = W.bf16_bits_to_f64(x["k_cache"]), W.bf16_bits_to_f64(x["v_cache"])
+    qf, kf, vf = (W.bf16_bits_to_f64(x[k]) for k in ("q_f", "k_f", "v_f"))
+    t0 = time.perf_counter()
+    k_re = ob.reencode_blocks(kc, None, t["cache_cu"], t["cache_delta"], w.rope_theta)
+    t1 = time.perf_counter()
+    k_all = np.concatenate([k_re, kf]); v_all = np.concatenate([vc, vf])
+    rows = np.arange(t["n_cached_tokens"], t["n_cached_tokens"] + n_rows)
+    m = ob.mask_rows(w.block_lens, w.seq_nblocks, ob.MODE_BLOCK, rows)
+    ob.attention_rows(qf[:n_rows], k_all, v_all, m)
+    t2 = time.perf_counter()
+    return ((t1 - t0) + (t2 - t1) * (Lf / n_rows)) * 1e6
+
+
+def blas_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 1) for p in threadpool_info() if p.get("user_api") == "blas"]
+        return max(n) if n else 1
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def run_reference(args):
+    rank, _, world = dist_env()
+    if rank != 0:
+        return 0
+    from paper_2409_15355_b200 import workloads as W
+    w = W.config3(1)
+    rows = 48
+    for _ in range(args.warmup):
+        oracle_layer_sample(w, 8)
+    vals = []
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        vals.append(oracle_layer_sample(w, rows))
+    wall = time.perf_counter() - t0
+    v = statistics.mean(vals)
+    sample = f"per step: one layer, re-encode of all 32000 cached rows + final attend of {rows}/768 final rows (all 32 heads), attend time scaled x{768 / rows:.0f}"
+    line = {"impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": wall * 1e3 / max(args.steps, 1),
+            "higher_is_better": False, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+            "data": "synthetic", "config": workload_config(),
+            "cpu_baseline": {"value": v, "unit": UNIT, "cores": blas_threads(), "kind": "oracle", "sample": sample},
+            "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+    return 0
+
+
+def workload_config():
+    return {"workload": "cfg3_32k: 32 cached blocks x 1000 tokens + 768-token final block, "
+                        "32 q heads / 8 kv heads / head_dim 128, 32 layers with independent seeded K/V/Q",
+            "layers": 32, "context": 32768, "final_block": 768, "mode": "block",
+            "l2": "inputs larger than L2 (131 MB of K/V per layer, distinct buffers per layer)"}
+
+
+# --------------------------------------------------------------------------- our arm
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2409_15355_b200 import binding as B
+    from paper_2409_15355_b200 import runtime as R
+    from paper_2409_15355_b200 import workloads as W
+
+    rank, local_rank, world = dist_env()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    L = args.layers
+    w = W.config3(L)
+    Tc, Tf = 32000, 768
+    ctx = R.Context.for_workload(w, device=local_rank)
+    pin = lambda bits: R.bits_to_tensor(bits).pin_memory()
+    host = []
+    for l in range(L):
+        x = W.warm_inputs(w, l)
+        host.append({k: pin(v) for k, v in x.items()})
+    names = ("q_f", "k_f", "v_f", "k_cache", "v_cache")
+    d_in = [{k: h[k].to(dev) for k in names} for h in host]
+    k_re = [torch.empty(Tc, w.n_kv_heads, w.head_dim, dtype=torch.bfloat16, device=dev) for _ in range(L)]
+    o = [torch.empty(Tf, w.n_q_heads, w.head_dim, dtype=torch.bfloat16, device=dev) for _ in range(L)]
+    o_host = [torch.empty(Tf, w.n_q_heads, w.head_dim, dtype=torch.bfloat16).pin_memory() for _ in range(L)]
+    lens = np.asarray(w.block_lens, dtype=np.int32)
+    nb = np.asarray(w.seq_nblocks, dtype=np.int32)
+    nbytes = B.ba_segments_bytes(1, len(lens), w.n_tokens)
+    tbuf = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+    stream = torch.cuda.current_stream()
+
+    att_events = []
+
+    def step(inputs, record=False):
+        seg = B.ba_segment(ctx.ctx, lens, nb, 1, len(lens), w.n_tokens, B.BA_MODE_BLOCK, tbuf)
+        for l in range(L):
+            x = inputs[l]
+            B.ba_reencode_k(ctx.ctx, x["k_cache"], None, Tc, k_re[l], seg.cache_cu, seg.cache_delta,
+                            seg.n_cached_blocks, Tc)
+            if record:
+                e0 = torch.cuda.Event(enable_timing=True); e0.record(stream)
+            B.ba_final_attend(ctx.ctx, x["q_f"], x["k_f"], x["v_f"], Tf, k_re[l], x["v_cache"], Tc, None, 0,
+                              o[l], None, seg, B.BA_MODE_BLOCK, B.BA_OUT_BF16)
+            if record:
+                e1 = torch.cuda.Event(enable_timing=True); e1.record(stream)
+                att_events.append((e0, e1))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step(d_in)
+    barrier()
+    launches0 = ctx.launches()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    barrier()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record(stream)
+    for _ in range(args.steps):
+        step(d_in, record=True)
+    ev1.record(stream)
+    barrier()
+    ms_local = ev0.elapsed_time(ev1) / args.steps
+    clocks = sampler.stop()
+    launches = ctx.launches() - launches0
+    assert ctx.device_status() == B.BA_OK
+    ms, us_per_layer = aggregate(ms_local, float(L), dev)
+
+    att_ms = statistics.mean(a.elapsed_time(b) for a, b in att_events)
+
+    # ---- end to end: host buffers in, host result out, copies inside the timed region
+    e2e_steps = max(1, min(args.steps, 3))
+    h2d = sum(h[k].numel() * 2 for h in host for k in names)
+    d2h = sum(t.numel() * 2 for t in o_host)
+    stage = [{k: torch.empty_like(d_in[l][k]) for k in names} for l in range(L)]
+
+    def e2e_step():
+        for l in range(L):
+            for k in names:
+                stage[l][k].copy_(host[l][k], non_blocking=True)
+        step(stage)
+        for l in range(L):
+            o_host[l].copy_(o[l], non_blocking=True)
+
+    e2e_step()
+    barrier()
+    ev0.record(stream)
+    for _ in range(e2e_steps):
+        e2e_step()
+    ev1.record(stream)
+    barrier()
+    _, e2e_us = aggregate(ev0.elapsed_time(ev1) / e2e_steps, float(L), dev)
+
+    if rank == 0:
+        peaks = load_peaks()
+        pairs = Tf * Tc + Tf * (Tf + 1) // 2
+        flops = 4.0 * w.head_dim * w.n_q_heads * pairs
+        achieved = flops / (att_ms * 1e-3) / 1e12
+        peak = peaks["bf16_tflops_sustained"] or peaks["bf16_tflops"]
+        roofline = {"bound": "tensor", "kernel": "ba_final_attend", "achieved": achieved, "peak": peak,
+                    "unit": "TFLOP/s", "frac": achieved / peak, "traffic": None,
+                    "peak_source": f"{peaks['source']} bf16 sustained (kernel timed inside a 32-layer step); "
+                                   f"burst {peaks['bf16_tflops']}",
+                    "frac_of_burst": achieved / peaks["bf16_tflops"],
+                    "attend_us_per_launch": att_ms * 1e3,
+                    "algorithmic_flops_per_launch": flops}
+        t0 = time.perf_counter()
+        cpu_rows = 96
+        cpu_us = oracle_layer_sample(W.config3(1), cpu_rows)
+        cpu = {"value": cpu_us, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
+               "sample": f"one layer: re-encode of 32000 cached rows + final attend of {cpu_rows}/768 final rows, "
+                         f"attend scaled x{768 // cpu_rows}; {time.perf_counter() - t0:.1f} s of CPU work"}
+        line = {"metric": METRIC, "value": us_per_layer, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": False, "scaling": "weak",
+                "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": workload_config(),
+                "clocks": clocks,
+                "e2e": {"value": e2e_us, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                        "steps": e2e_steps},
+                "gpu_launches": launches, "roofline": roofline, "cpu_baseline": cpu}
+        if L != 32:
+            line["config"]["layers"] = L
+        print(json.dumps(line))
+    ctx.close()
+    if world > 1:
+        dist.destroy_process_group()
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--layers", type=int, default=32, help="layers per step (32 = the metric's workload)")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+    return run_ours(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -205,11 +205,12 @@ ba_status ba_segment(ba_ctx *ctx, const int32_t *block_lens, const int32_t *seq_
 ba_status ba_reencode_k(ba_ctx *ctx, const void *k_src, const int32_t *src_off, int32_t n_src_rows,
                         void *k_dst, const int32_t *cu, const int32_t *delta, int32_t n_blocks,
                         int32_t n_rows, void *stream) {
-  if (!ctx || !k_src || !k_dst || !cu || !delta) return BA_ERR_INVALID_ARG;
+  if (!ctx) return BA_ERR_INVALID_ARG;
   if (n_blocks < 0 || n_rows < 0 || n_src_rows < 0) return BA_ERR_INVALID_ARG;
+  if (n_blocks == 0 || n_rows == 0) return BA_OK;            // nothing cached: nothing to do
+  if (!k_src || !k_dst || !cu || !delta) return BA_ERR_INVALID_ARG;
   if (!aligned16(k_src) || !aligned16(k_dst)) return BA_ERR_INVALID_ARG;
   if (k_src == k_dst && src_off) return BA_ERR_INVALID_ARG;  // a gather cannot run in place
-  if (n_blocks == 0 || n_rows == 0) return BA_OK;
   BA_CUDA_TRY(cudaSetDevice(ctx->device));
   // scratch: the angle table at the end of the workspace (the staging area is at its start)
   size_t need = ba_align_up((size_t)n_blocks * ctx->cfg.head_dim * 4, 256);  // n_blocks * d/2 * sizeof(float2)

@@ -1,0 +1,359 @@
+"""Parity of the CUDA path (through the C ABI) with the fp64 oracle on the same
+seeded inputs.
+
+Tolerances.  Integer tables: bit-exact.  Attention outputs written as fp32
+(bf16 inputs, fp32 accumulation): max-abs <= 1e-2 and mean-abs <= 1e-3 against
+the fp64 oracle, plus a relative Frobenius error <= 5e-3 and log-sum-exp within
+2e-3 (the absolute bounds alone are loose once thousands of keys are averaged).
+Outputs stored as bf16 are compared with the oracle rounded to bf16 under the
+same absolute bounds.  Re-encoded keys are bf16 by contract: each must lie
+within half a bf16 ulp (plus fp32 noise) of the fp64 value, i.e. be a correct
+rounding of it, and within one ulp of the oracle's own rounding.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import block_attention as ob
+from paper_2409_15355_b200 import binding as B
+from paper_2409_15355_b200 import runtime as R
+from paper_2409_15355_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+TABLE_KEYS = ["cu_seq", "cu_cache_seq", "cu_final_seq", "cu_block", "block_delta", "block_seq",
+              "block_kv_begin", "block_part_off", "block_is_final", "cache_block", "cache_cu",
+              "cache_delta", "tok_block", "tok_pos", "tok_pos_local"]
+
+
+def check_attention(o_gpu, o_ref, lse_gpu=None, lse_ref=None, rel=5e-3):
+    o_gpu = np.asarray(o_gpu, dtype=np.float64)
+    d = np.abs(o_gpu - o_ref)
+    assert np.isfinite(o_gpu).all()
+    assert d.max() <= 1e-2, f"max-abs {d.max()}"
+    assert d.mean() <= 1e-3, f"mean-abs {d.mean()}"
+    fro = np.linalg.norm(o_gpu - o_ref) / np.linalg.norm(o_ref)
+    assert fro <= rel, f"relative Frobenius {fro}"
+    if lse_gpu is not None:
+        dl = np.abs(np.asarray(lse_gpu, dtype=np.float64) - lse_ref).max()
+        assert dl <= 2e-3, f"lse {dl}"
+
+
+def round_bf16(x64):
+    return W.bf16_bits_to_f64(W.f32_to_bf16_bits(np.asarray(x64, dtype=np.float32)))
+
+
+def check_reencoded(k_gpu_bits, k_ref64):
+    g = W.bf16_bits_to_f64(k_gpu_bits)
+    # a correct rounding of the fp64 value: within half a bf16 ulp (at most 2^-8 relative) + fp32 noise
+    assert (np.abs(g - k_ref64) <= np.abs(k_ref64) * (2.0 ** -8) * 1.01 + 1e-6 * np.abs(k_ref64) + 1e-30).all()
+    r = round_bf16(k_ref64)
+    d = np.abs(g - r)
+    assert d.mean() <= 1e-3
+    assert (d <= np.abs(r) * 2.0 ** -7 + 1e-30).all()         # at most one ulp from the oracle's rounding
+    assert (g == r).mean() >= 0.995
+
+
+def ctx_for(w, **kw):
+    return R.Context.for_workload(w, **kw)
+
+
+def dev(bits):
+    return R.bits_to_device(bits)
+
+
+# --------------------------------------------------------------------------- tables
+def table_cases():
+    return [W.config1(), W.config2(), W.config3(1), W.config4(), W.config5(),
+            W.random_ragged(11, 5, 7, 300, 4, 2, 64), W.random_ragged(12, 40, 3, 50, 4, 2, 64),
+            W.Workload("one_token", 4, 2, 64, 1e4, [1], [1], seed=1),
+            W.Workload("many_seqs", 4, 2, 64, 1e4, [1] * 3000, [1] * 3000, seed=2),
+            W.Workload("many_blocks", 4, 2, 64, 1e4, [3, 1, 2] * 1000, [3000], seed=3)]
+
+
+@pytest.mark.parametrize("w", table_cases(), ids=lambda w: w.name)
+@pytest.mark.parametrize("mode", [B.BA_MODE_BLOCK, B.BA_MODE_FULL])
+def test_tables_bit_exact(w, mode):
+    c = ctx_for(w)
+    seg, buf = c.segment(w.block_lens, w.seq_nblocks, mode)
+    got = R.read_tables(seg, buf)
+    assert c.device_status() == B.BA_OK
+    ref = ob.segment_tables(w.block_lens, w.seq_nblocks, mode)
+    for k in TABLE_KEYS:
+        assert got[k].tolist() == ref[k].tolist(), k
+    assert got["totals"][0] == ref["n_cached_tokens"] and got["totals"][1] == ref["n_final_tokens"]
+    c.close()
+
+
+def test_tables_from_device_lengths_and_bad_lengths():
+    w = W.config2()
+    c = ctx_for(w)
+    lens = torch.tensor(w.block_lens, dtype=torch.int32, device="cuda")
+    nb = torch.tensor(w.seq_nblocks, dtype=torch.int32, device="cuda")
+    seg, buf = c.segment(lens, nb, B.BA_MODE_BLOCK, n_tokens=w.n_tokens)
+    got = R.read_tables(seg, buf)
+    ref = ob.segment_tables(w.block_lens, w.seq_nblocks)
+    for k in TABLE_KEYS:
+        assert got[k].tolist() == ref[k].tolist(), k
+    assert c.device_status() == B.BA_OK
+    # device-side lengths that do not add up: reported by the status word, nothing faults
+    seg, buf = c.segment(lens, nb, B.BA_MODE_BLOCK, n_tokens=w.n_tokens + 5)
+    assert c.device_status() == B.BA_ERR_INVALID_ARG
+    assert c.device_status() == B.BA_OK          # cleared by the read
+    bad = lens.clone(); bad[3] = 0
+    seg, buf = c.segment(bad, nb, B.BA_MODE_BLOCK, n_tokens=w.n_tokens)
+    assert c.device_status() == B.BA_ERR_INVALID_ARG
+    # tables marked invalid: attention over them does nothing and does not fault
+    q = torch.zeros(w.n_tokens, w.n_q_heads, w.head_dim, dtype=torch.bfloat16, device="cuda")
+    kv = torch.zeros(w.n_tokens, w.n_kv_heads, w.head_dim, dtype=torch.bfloat16, device="cuda")
+    o = torch.full_like(q, 7.0)
+    B.ba_block_prefill(c.ctx, q, kv, kv, o, None, seg, B.BA_MODE_BLOCK, B.BA_OUT_BF16)
+    torch.cuda.synchronize()
+    assert (o == 7.0).all()
+    # host-side lengths are rejected before any launch
+    with pytest.raises(B.BaError) as e:
+        c.segment([3, 0, 2], [3], B.BA_MODE_BLOCK, n_tokens=5)
+    assert e.value.status == B.BA_ERR_INVALID_ARG
+    with pytest.raises(B.BaError):
+        c.segment([3, 1, 2], [2], B.BA_MODE_BLOCK)
+    c.close()
+
+
+# --------------------------------------------------------------------------- re-encode
+def reencode_case(w, layout=B.BA_ROPE_ADJACENT, layer=0):
+    c = ctx_for(w, rope_layout=layout)
+    seg, buf = c.segment(w.block_lens, w.seq_nblocks, B.BA_MODE_BLOCK)
+    t = ob.segment_tables(w.block_lens, w.seq_nblocks)
+    x = W.warm_inputs(w, layer)
+    Tc = t["n_cached_tokens"]
+    if w.pool_lens is None:
+        src, off, off_np = dev(x["k_cache"]), None, None
+        src_np = x["k_cache"]
+    else:
+        src, off_np = dev(x["k_pool"]), x["src_off"]
+        off = torch.from_numpy(off_np).cuda()
+        src_np = x["k_pool"]
+    dst = torch.empty(Tc, w.n_kv_heads, w.head_dim, dtype=torch.bfloat16, device="cuda")
+    B.ba_reencode_k(c.ctx, src, off, src.shape[0], dst, seg.cache_cu, seg.cache_delta,
+                    seg.n_cached_blocks, Tc)
+    assert c.device_status() == B.BA_OK
+    ref = ob.reencode_blocks(W.bf16_bits_to_f64(src_np), off_np, t["cache_cu"], t["cache_delta"],
+                             w.rope_theta, layout)
+    return c, seg, buf, src, dst, ref, t
+
+
+@pytest.mark.parametrize("w", [W.config1(), W.config2(), W.config5(4, 64, 6, 32), W.config3(1)],
+                         ids=lambda w: w.name)
+def test_reencode_parity(w):
+    c, seg, buf, src, dst, ref, t = reencode_case(w)
+    check_reencoded(R.device_to_bits(dst), ref)
+    # the block with delta 0 is copied bit-exactly
+    n0 = int(t["cache_cu"][1])
+    if w.pool_lens is None:
+        assert torch.equal(dst[:n0], src[:n0])
+    c.close()
+
+
+def test_reencode_half_layout_in_place_and_inverse():
+    w = W.config2()
+    c, seg, buf, src, dst, ref, t = reencode_case(w, layout=B.BA_ROPE_HALF)
+    check_reencoded(R.device_to_bits(dst), ref)
+    Tc = t["n_cached_tokens"]
+    # in place
+    inplace = src.clone()
+    B.ba_reencode_k(c.ctx, inplace, None, Tc, inplace, seg.cache_cu, seg.cache_delta, seg.n_cached_blocks, Tc)
+    assert torch.equal(inplace, dst)
+    # negative deltas (Eq. 2: back to position zero) undo the re-encoding up to bf16 rounding
+    neg = torch.from_numpy(-t["cache_delta"]).cuda()
+    back = torch.empty_like(dst)
+    B.ba_reencode_k(c.ctx, dst, None, Tc, back, seg.cache_cu, neg, seg.n_cached_blocks, Tc)
+    ref_back = ob.reencode_blocks(W.bf16_bits_to_f64(R.device_to_bits(dst)), None, t["cache_cu"],
+                                  -t["cache_delta"], w.rope_theta, ob.ROPE_HALF)
+    check_reencoded(R.device_to_bits(back), ref_back)
+    assert c.device_status() == B.BA_OK
+    c.close()
+
+
+def test_reencode_errors_do_not_fault():
+    w = W.config1()
+    c = ctx_for(w)
+    seg, buf = c.segment(w.block_lens, w.seq_nblocks, B.BA_MODE_BLOCK)
+    k = torch.zeros(256, 2, 64, dtype=torch.bfloat16, device="cuda")
+    out = torch.zeros_like(k)
+    off = torch.tensor([0, 64, 128, 250], dtype=torch.int32, device="cuda")   # last block runs off the source
+    B.ba_reencode_k(c.ctx, k, off, 256, out, seg.cache_cu, seg.cache_delta, 4, 256)
+    assert c.device_status() == B.BA_ERR_INVALID_ARG
+    with pytest.raises(B.BaError) as e:
+        B.ba_reencode_k(c.ctx, k, off, 256, k, seg.cache_cu, seg.cache_delta, 4, 256)   # gather in place
+    assert e.value.status == B.BA_ERR_INVALID_ARG
+    with pytest.raises(B.BaError):
+        B.ba_reencode_k(c.ctx, k.view(-1)[1:], None, 255, out, seg.cache_cu, seg.cache_delta, 4, 255)  # misaligned
+    small = R.Context(4, 2, 64, 1e4, max_blocks=1)
+    big = W.Workload("b", 4, 2, 64, 1e4, [1] * 600, [600], seed=1)
+    with pytest.raises(B.BaError) as e:
+        small.segment(big.block_lens, big.seq_nblocks, B.BA_MODE_BLOCK)
+    assert e.value.status == B.BA_ERR_WORKSPACE
+    small.close()
+    c.close()
+
+
+# --------------------------------------------------------------------------- prefill
+def run_prefill(w, mode, out_dtype=B.BA_OUT_F32, rows=None, layer=0):
+    c = ctx_for(w)
+    seg, buf = c.segment(w.block_lens, w.seq_nblocks, mode)
+    qb, kb, vb = W.prefill_inputs(w, layer)
+    q, k, v = dev(qb), dev(kb), dev(vb)
+    T = w.n_tokens
+    o = torch.empty(T, w.n_q_heads, w.head_dim, device="cuda",
+                    dtype=torch.float32 if out_dtype == B.BA_OUT_F32 else torch.bfloat16)
+    lse = torch.empty(T, w.n_q_heads, dtype=torch.float32, device="cuda")
+    B.ba_block_prefill(c.ctx, q, k, v, o, lse, seg, mode, out_dtype)
+    assert c.device_status() == B.BA_OK
+    if rows is None:
+        rows = np.arange(T)
+    o_ref, lse_ref = ob.block_prefill(W.bf16_bits_to_f64(qb), W.bf16_bits_to_f64(kb), W.bf16_bits_to_f64(vb),
+                                      w.block_lens, w.seq_nblocks, mode, rows=rows)
+    c.close()
+    rt = torch.from_numpy(np.asarray(rows)).cuda()
+    return o[rt].float().cpu().numpy(), lse[rt].cpu().numpy(), o_ref, lse_ref
+
+
+PREFILL_CASES = [W.config1(), W.config2(), W.random_ragged(21, 3, 6, 300, 4, 2, 64),
+                 W.random_ragged(22, 2, 5, 400, 8, 2, 128), W.random_ragged(23, 4, 4, 140, 4, 4, 128),
+                 W.Workload("one_token", 4, 2, 64, 1e4, [1], [1], seed=5),
+                 W.Workload("single_block", 8, 8, 128, 1e4, [333], [1], seed=6)]
+
+
+@pytest.mark.parametrize("w", PREFILL_CASES, ids=lambda w: w.name)
+@pytest.mark.parametrize("mode", [B.BA_MODE_BLOCK, B.BA_MODE_FULL])
+def test_prefill_parity(w, mode):
+    o, lse, o_ref, lse_ref = run_prefill(w, mode)
+    check_attention(o, o_ref, lse, lse_ref)
+
+
+def test_prefill_bf16_output():
+    o, lse, o_ref, lse_ref = run_prefill(W.config2(), B.BA_MODE_BLOCK, B.BA_OUT_BF16)
+    check_attention(o, round_bf16(o_ref), lse, lse_ref, rel=8e-3)
+
+
+def sampled_rows(w, per_block=8, extra=128, seed=0):
+    t = ob.segment_tables(w.block_lens, w.seq_nblocks)
+    rows = []
+    for b in range(w.n_blocks):
+        lo, hi = int(t["cu_block"][b]), int(t["cu_block"][b + 1])
+        rows += list(range(lo, min(hi, lo + per_block))) + list(range(max(lo, hi - per_block), hi))
+    rng = np.random.default_rng(seed)
+    rows += [int(x) for x in rng.integers(0, w.n_tokens, size=extra)]
+    return np.unique(np.asarray(rows))
+
+
+def test_prefill_cold_batch_full_size_sampled_rows():
+    # batch 8 x 16384 ragged cold prefill in one launch; the oracle is evaluated on the first and
+    # last rows of every block plus seeded random rows (exact for those rows)
+    w = W.config4()
+    rows = sampled_rows(w, per_block=4, extra=64)
+    o, lse, o_ref, lse_ref = run_prefill(w, B.BA_MODE_BLOCK, rows=rows)
+    check_attention(o, o_ref, lse, lse_ref)
+
+
+def test_prefill_full_causal_32k_sampled_rows():
+    w = W.config3(1)
+    rng = np.random.default_rng(3)
+    rows = np.unique(np.concatenate([np.arange(0, 4), np.arange(32764, 32768), rng.integers(0, 32768, 120)]))
+    o, lse, o_ref, lse_ref = run_prefill(w, B.BA_MODE_FULL, rows=rows)
+    check_attention(o, o_ref, lse, lse_ref)
+
+
+# --------------------------------------------------------------------------- warm path
+def run_warm(w, mode, out_dtype=B.BA_OUT_F32, layer=0, v_from_pool=True):
+    """ba_segment -> ba_reencode_k -> ba_final_attend, against oracle re-encode + final attend.
+    The oracle attends its own unrounded fp64 re-encoded keys."""
+    c = ctx_for(w)
+    seg, buf = c.segment(w.block_lens, w.seq_nblocks, mode)
+    t = ob.segment_tables(w.block_lens, w.seq_nblocks, mode)
+    x = W.warm_inputs(w, layer)
+    Tc, Tf = t["n_cached_tokens"], t["n_final_tokens"]
+    q_f, k_f, v_f = dev(x["q_f"]), dev(x["k_f"]), dev(x["v_f"])
+    k_re = torch.empty(Tc, w.n_kv_heads, w.head_dim, dtype=torch.bfloat16, device="cuda")
+    if w.pool_lens is None:
+        k_src, v_cache, off, off_np = dev(x["k_cache"]), dev(x["v_cache"]), None, None
+        k_src_np, v_np = x["k_cache"], W.bf16_bits_to_f64(x["v_cache"])
+        v_off, n_v = None, 0
+    else:
+        k_src, off_np = dev(x["k_pool"]), x["src_off"]
+        off = torch.from_numpy(off_np).cuda()
+        k_src_np = x["k_pool"]
+        v_pool64 = W.bf16_bits_to_f64(x["v_pool"])
+        v_np = np.concatenate([v_pool64[o_:o_ + (t["cache_cu"][i + 1] - t["cache_cu"][i])]
+                               for i, o_ in enumerate(off_np)], axis=0)
+        if v_from_pool:
+            v_cache, v_off, n_v = dev(x["v_pool"]), off, x["v_pool"].shape[0]
+        else:
+            v_cache, v_off, n_v = dev(W.f32_to_bf16_bits(v_np.astype(np.float32))), None, 0
+    B.ba_reencode_k(c.ctx, k_src, off, k_src.shape[0], k_re, seg.cache_cu, seg.cache_delta,
+                    seg.n_cached_blocks, Tc)
+    o = torch.empty(Tf, w.n_q_heads, w.head_dim, device="cuda",
+                    dtype=torch.float32 if out_dtype == B.BA_OUT_F32 else torch.bfloat16)
+    lse = torch.empty(Tf, w.n_q_heads, dtype=torch.float32, device="cuda")
+    B.ba_final_attend(c.ctx, q_f, k_f, v_f, Tf, k_re, v_cache, Tc, v_off, n_v, o, lse, seg, mode, out_dtype)
+    assert c.device_status() == B.BA_OK
+    k_ref = ob.reencode_blocks(W.bf16_bits_to_f64(k_src_np), off_np, t["cache_cu"], t["cache_delta"], w.rope_theta)
+    o_ref, lse_ref = ob.final_attend(W.bf16_bits_to_f64(x["q_f"]), W.bf16_bits_to_f64(x["k_f"]),
+                                     W.bf16_bits_to_f64(x["v_f"]), k_ref, v_np, w.block_lens, w.seq_nblocks, mode)
+    c.close()
+    return o.float().cpu().numpy(), lse.cpu().numpy(), o_ref, lse_ref
+
+
+WARM_CASES = [W.config1(), W.config2(), W.random_ragged(31, 3, 5, 200, 4, 2, 64),
+              W.Workload("no_cache", 4, 2, 64, 1e4, [50, 1, 130], [1, 1, 1], seed=7),
+              W.config5(4, 64, 6, 32)]
+
+
+@pytest.mark.parametrize("w", WARM_CASES, ids=lambda w: w.name)
+@pytest.mark.parametrize("mode", [B.BA_MODE_BLOCK, B.BA_MODE_FULL])
+def test_warm_path_parity(w, mode):
+    o, lse, o_ref, lse_ref = run_warm(w, mode)
+    check_attention(o, o_ref, lse, lse_ref)
+
+
+def test_warm_path_pool_serving_full_size_and_mode_switch():
+    w = W.config5()
+    half = W.Workload("half", w.n_q_heads, w.n_kv_heads, w.head_dim, w.rope_theta,
+                      w.block_lens[:21 * 8], w.seq_nblocks[:8], w.seed, pool_lens=w.pool_lens,
+                      request_pool_idx=w.request_pool_idx[:8])
+    ob_, lb, o_ref, lse_ref = run_warm(half, B.BA_MODE_BLOCK)
+    check_attention(ob_, o_ref, lb, lse_ref)
+    of_, lf, _, _ = run_warm(half, B.BA_MODE_FULL, v_from_pool=False)
+    # final rows see the same keys under both masks: results agree to the last bit or nearly so
+    assert np.abs(of_ - ob_).max() <= 1e-5
+
+
+def test_warm_path_32k_full_size():
+    w = W.config3(1)
+    o, lse, o_ref, lse_ref = run_warm(w, B.BA_MODE_BLOCK, B.BA_OUT_BF16)
+    check_attention(o, round_bf16(o_ref), lse, lse_ref, rel=2e-2)
+    o2, lse2, _, _ = run_warm(w, B.BA_MODE_BLOCK, B.BA_OUT_F32)
+    check_attention(o2, o_ref, lse2, lse_ref)
+
+
+def test_attention_rejects_mode_mismatch_and_null():
+    w = W.config1()
+    c = ctx_for(w)
+    seg, buf = c.segment(w.block_lens, w.seq_nblocks, B.BA_MODE_BLOCK)
+    q = torch.zeros(288, 4, 64, dtype=torch.bfloat16, device="cuda")
+    kv = torch.zeros(288, 2, 64, dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(B.BaError) as e:
+        B.ba_block_prefill(c.ctx, q, kv, kv, q, None, seg, B.BA_MODE_FULL, B.BA_OUT_BF16)
+    assert e.value.status == B.BA_ERR_INVALID_ARG
+    with pytest.raises(B.BaError):
+        B.ba_block_prefill(c.ctx, q, None, kv, q, None, seg, B.BA_MODE_BLOCK, B.BA_OUT_BF16)
+    with pytest.raises(B.BaError):
+        B.ba_final_attend(c.ctx, q, kv, kv, 32, None, None, 256, None, 0, q, None, seg, B.BA_MODE_BLOCK, B.BA_OUT_BF16)
+    c.close()
+
+
+def test_runs_are_bit_stable():
+    w = W.config2()
+    a = run_warm(w, B.BA_MODE_BLOCK)[0]
+    b = run_warm(w, B.BA_MODE_BLOCK)[0]
+    assert (a == b).all()
