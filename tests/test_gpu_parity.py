@@ -7,7 +7,7 @@ the fp64 oracle, plus a relative Frobenius error <= 5e-3 and log-sum-exp within
 2e-3 (the absolute bounds alone are loose once thousands of keys are averaged).
 Outputs stored as bf16 are compared with the oracle rounded to bf16 under the
 same absolute bounds.  Re-encoded keys are bf16 by contract: each must lie
-within half a bf16 ulp (plus fp32 noise) of the fp64 value, i.e. be a correct
+within half a bf16 ulp (plus 1e-6 of fp32 noise: a rotation can cancel to a tiny value) of the fp64 value, i.e. be a correct
 rounding of it, and within one ulp of the oracle's own rounding.
 """
 import numpy as np
@@ -46,11 +46,11 @@ def round_bf16(x64):
 def check_reencoded(k_gpu_bits, k_ref64):
     g = W.bf16_bits_to_f64(k_gpu_bits)
     # a correct rounding of the fp64 value: within half a bf16 ulp (at most 2^-8 relative) + fp32 noise
-    assert (np.abs(g - k_ref64) <= np.abs(k_ref64) * (2.0 ** -8) * 1.01 + 1e-6 * np.abs(k_ref64) + 1e-30).all()
+    assert (np.abs(g - k_ref64) <= np.abs(k_ref64) * (2.0 ** -8) * 1.01 + 1e-6).all()
     r = round_bf16(k_ref64)
     d = np.abs(g - r)
     assert d.mean() <= 1e-3
-    assert (d <= np.abs(r) * 2.0 ** -7 + 1e-30).all()         # at most one ulp from the oracle's rounding
+    assert (d <= np.abs(r) * 2.0 ** -7 + 1e-6).all()         # at most one ulp from the oracle's rounding
     assert (g == r).mean() >= 0.995
 
 
