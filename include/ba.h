@@ -168,6 +168,43 @@ ba_status ba_reencode_k(ba_ctx *ctx, const void *k_src, const int32_t *src_off, 
                         int32_t n_rows, void *stream);
 
 /*
+ * ba_reencode_k_noalloc -- the same re-encoding as ba_reencode_k for callers that
+ * must not allocate device memory.  (The paper has no counterpart to this entry
+ * point; it exists for integration reasons only.)
+ *
+ * Who needs it: a serving engine that hands all free device memory to its own
+ * pool at start-up (a later cudaMalloc then fails or eats into the pool's
+ * head-room), and code on a latency-critical path that cannot afford the
+ * device-wide synchronisation cudaMalloc/cudaFree imply.  Such callers cannot
+ * use ba_create(), which allocates the workspace the angle table lives in.
+ *
+ * This call needs no context.  The angle table is kept in a fixed array built
+ * into the library image: BA_NOALLOC_MAX_BLOCKS * 64 (cos, sin) pairs = 2 MiB
+ * that every GPU which loads the library holds until the process exits.  The
+ * call itself performs no cudaMalloc/cudaFree and uses no allocating library
+ * routine.
+ *
+ *   cfg, device    as for ba_create (head_dim, n_kv_heads, rope_theta, rope_layout are used)
+ *   status_word    device int32 owned by the caller, or NULL.  A source row out of range is
+ *                  skipped and BA_ERR_INVALID_ARG is stored there if the word is still 0
+ *                  (clear it yourself); with NULL such rows are skipped silently.
+ *   other arguments exactly as for ba_reencode_k
+ *
+ * n_blocks > BA_NOALLOC_MAX_BLOCKS is rejected with BA_ERR_WORKSPACE before anything runs.
+ * The first call on a device looks up the device address of the built-in array;
+ * make that first call outside any stream capture.  All calls on a device share
+ * the one array, which keeps the previous call's contents (every entry a call
+ * reads is rewritten by that call first, so nothing needs clearing): two calls
+ * whose kernels may overlap on the GPU -- different streams, no ordering between
+ * them -- race on it and must be ordered by the caller.
+ */
+#define BA_NOALLOC_MAX_BLOCKS 4096
+ba_status ba_reencode_k_noalloc(const ba_config *cfg, int device, const void *k_src,
+                                const int32_t *src_off, int32_t n_src_rows, void *k_dst,
+                                const int32_t *cu, const int32_t *delta, int32_t n_blocks,
+                                int32_t n_rows, int32_t *status_word, void *stream);
+
+/*
  * Section 1 / Section 2.4: attention of a packed ragged batch under the
  * Block-attention mask, all blocks in one launch.  Row i of block b sees key
  * rows block_kv_begin[b] .. i (prompt packing).  q [T, n_q_heads, head_dim],

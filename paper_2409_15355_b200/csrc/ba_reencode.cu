@@ -183,3 +183,67 @@ ba_status ba_reencode_launch(ba_ctx *ctx, const void *k_src, const int32_t *src_
   ctx->launches += 2;
   return BA_OK;
 }
+
+// ---------------------------------------------------------------------------
+// Allocation-free variant.  The angle table lives in a fixed array that is part
+// of the library image; each device that loads the library gets its own copy.
+// ---------------------------------------------------------------------------
+#include <mutex>
+
+namespace {
+
+constexpr int kNoallocMaxDevices = 64;
+// 4096 blocks x 64 rotary pairs x (cos, sin) = 2 MiB per device
+static __device__ __align__(256) float2 ba_noalloc_table[BA_NOALLOC_MAX_BLOCKS * 64];
+// Receives "bad source row" reports when the caller passes no status word.
+static __device__ int32_t ba_noalloc_status_sink;
+
+// In host code the two names above are host-side handles, not device addresses.
+// The addresses a kernel can use are looked up once per device and kept here.
+float2 *g_noalloc_table[kNoallocMaxDevices];
+int32_t *g_noalloc_sink[kNoallocMaxDevices];
+std::mutex g_noalloc_mutex;
+
+}  // namespace
+
+extern "C" ba_status ba_reencode_k_noalloc(const ba_config *cfg, int device, const void *k_src,
+                                           const int32_t *src_off, int32_t n_src_rows, void *k_dst,
+                                           const int32_t *cu, const int32_t *delta, int32_t n_blocks,
+                                           int32_t n_rows, int32_t *status_word, void *stream) {
+  if (!cfg) return BA_ERR_INVALID_ARG;
+  if (cfg->head_dim != 64 && cfg->head_dim != 128) return BA_ERR_UNSUPPORTED;
+  if (cfg->n_kv_heads < 1) return BA_ERR_UNSUPPORTED;
+  if (cfg->rope_layout != BA_ROPE_ADJACENT && cfg->rope_layout != BA_ROPE_HALF) return BA_ERR_INVALID_ARG;
+  if (!(cfg->rope_theta > 1.0)) return BA_ERR_INVALID_ARG;
+  if (device < 0 || device >= kNoallocMaxDevices) return BA_ERR_INVALID_ARG;
+  if (n_blocks < 0 || n_rows < 0 || n_src_rows < 0) return BA_ERR_INVALID_ARG;
+  if (n_blocks > BA_NOALLOC_MAX_BLOCKS) return BA_ERR_WORKSPACE;   // built-in table too small
+  if (n_blocks == 0 || n_rows == 0) return BA_OK;
+  if (!k_src || !k_dst || !cu || !delta) return BA_ERR_INVALID_ARG;
+  if (((uintptr_t)k_src | (uintptr_t)k_dst) & 15u) return BA_ERR_INVALID_ARG;
+  if (k_src == k_dst && src_off) return BA_ERR_INVALID_ARG;
+  BA_CUDA_TRY(cudaSetDevice(device));
+  {
+    std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+    if (!g_noalloc_table[device]) {   // first call on this device, which is current
+      float2 *t = nullptr;
+      int32_t *sink = nullptr;
+      BA_CUDA_TRY(cudaGetSymbolAddress((void **)&t, ba_noalloc_table));
+      BA_CUDA_TRY(cudaGetSymbolAddress((void **)&sink, ba_noalloc_status_sink));
+      g_noalloc_sink[device] = sink;
+      g_noalloc_table[device] = t;
+    }
+  }
+  // A context on the stack carries the configuration to the shared launch code; nothing is allocated.
+  ba_ctx tmp;
+  tmp.cfg = *cfg;
+  tmp.device = device;
+  tmp.sm_count = 0;
+  tmp.scale = 0.f;
+  tmp.workspace = nullptr;
+  tmp.workspace_bytes = 0;
+  tmp.dev_status = status_word ? status_word : g_noalloc_sink[device];
+  tmp.launches = 0;
+  return ba_reencode_launch(&tmp, k_src, src_off, n_src_rows, k_dst, cu, delta, n_blocks, n_rows,
+                            g_noalloc_table[device], (cudaStream_t)stream);
+}
