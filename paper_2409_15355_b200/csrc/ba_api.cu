@@ -7,6 +7,10 @@
 
 ba_status ba_attend_simt_launch(ba_ctx *ctx, const ba_attend_args &a, const ba_segments *seg,
                                 cudaStream_t stream);
+ba_status ba_attend_sm100_launch(ba_ctx *ctx, const ba_attend_args &a, const ba_segments *seg,
+                                 cudaStream_t stream);
+bool ba_attend_sm100_supported(const ba_ctx *ctx, const ba_attend_args &a);
+int ba_heads_per_tile(const ba_config &c);
 
 namespace {
 
@@ -30,11 +34,9 @@ ba_status check_config(const ba_config *c) {
   return BA_OK;
 }
 
-// Tokens per query tile of the attention kernels.
-int q_tile_tokens(const ba_config &c) {
-  (void)c;
-  return 128;
-}
+// Tokens per work item of the tensor-core attention kernel: two query tiles of
+// 128 rows, each row one (token, head) of the heads packed into a tile.
+int q_tile_tokens(const ba_config &c) { return 2 * 128 / ba_heads_per_tile(c); }
 
 // Start of the workspace: staging of host-side length arrays.
 size_t stage_bytes_for(int32_t max_blocks) { return ba_align_up((size_t)(2 * (size_t)max_blocks + 64) * 4, 256); }
@@ -274,5 +276,8 @@ ba_status ba_final_attend(ba_ctx *ctx, const void *q_f, const void *k_f, const v
 
 ba_status ba_attend_launch(ba_ctx *ctx, const ba_attend_args &a, const ba_segments *seg,
                            cudaStream_t stream) {
+  if (a.n_q_rows == 0) return BA_OK;
+  // the tensor-core kernel takes every case except values gathered from a pool by index
+  if (ba_attend_sm100_supported(ctx, a)) return ba_attend_sm100_launch(ctx, a, seg, stream);
   return ba_attend_simt_launch(ctx, a, seg, stream);
 }

@@ -1,0 +1,450 @@
+// Tensor-core attention under the Block-attention mask for sm_100a.
+//
+// One kernel serves ba_block_prefill (Section 1 / 2.4: a row of a non-final block
+// sees its own block, causally; a row of a final block sees its whole sequence
+// prefix) and ba_final_attend (Section 2.5 step 3: the final block over the
+// re-encoded cached blocks plus itself).  The mask never exists as a matrix: a
+// work item is a pair of query tiles of one block, its keys are one optional
+// "cached" range (all visible) followed by one "own" range (causal).
+//
+// Structure of a CTA (384 threads, one CTA per SM):
+//   warps 0-3   softmax of query tile 0      (one thread per tile row = TMEM lane)
+//   warps 4-7   softmax of query tile 1
+//   warp  8     TMA producer: Q tiles once, then K_j, V_j, K_j+1, ... into a ring of stages
+//   warp  9     MMA issuer (one elected thread): S = Q K^T and O += P V with tcgen05.mma,
+//               accumulators in tensor memory (S0, S1, O0, O1 = 4 x 128 columns)
+// A query tile is 128 rows = (128 / HPT) tokens x HPT query heads of one KV group,
+// so a K/V tile staged once serves every head of the group and both query tiles.
+// Softmax is online in fp32 (base-2 exponent with the scale folded in); P is
+// written back to tensor memory as bf16 over the S columns and used as the A
+// operand of the PV product.  O is rescaled in tensor memory only when the
+// running maximum grows by more than 2^8, which keeps every term bounded and the
+// result exact in real arithmetic.
+#include <math.h>
+
+#include "ba_common.cuh"
+#include "ba_sm100.cuh"
+
+using namespace sm100;
+
+namespace {
+
+constexpr int kThreads = 384;
+constexpr int kBlockN = 128;      // keys per tile
+constexpr int kStages = 3;        // ring of K/V tiles
+constexpr float kRescaleThreshold = 8.0f;
+
+struct AttnParams {
+  void *o;
+  float *lse;
+  int32_t *status;
+  int out_f32;
+  int Hq, Hkv, G;
+  int hpt, hpt_log2, tok;         // heads per tile, tokens per tile (hpt * tok = 128)
+  float scale, scale_log2;
+  int final_only;
+  int n_q_rows;
+  ba_segments seg;
+};
+
+template <int D>
+struct Layout {
+  static constexpr int kChunks = D / 64;                  // 64-column (128-byte) swizzle regions per row
+  static constexpr int kTileBytes = 128 * D * 2;          // one 128-row tile of Q, K or V
+  static constexpr int kRegionBytes = 128 * 128;          // 128 rows x 128 bytes
+  static constexpr int kQ0 = 0;
+  static constexpr int kQ1 = kTileBytes;
+  static constexpr int kRing = 2 * kTileBytes;
+  static constexpr int kCtrl = kRing + kStages * kTileBytes;
+  static constexpr int kBytes = kCtrl + 1024;
+};
+
+struct Ctrl {
+  uint64_t q_full[2];
+  uint64_t kv_full[kStages];
+  uint64_t kv_empty[kStages];
+  uint64_t s_full[2];
+  uint64_t p_full[2];
+  uint64_t o_done[2];
+  uint32_t tmem_base;
+  int abort_flag;
+};
+
+// One work item: two query tiles of one block (or final block) and the key ranges they see.
+struct Item {
+  int q_row0;        // first query row (q packing)
+  int q_rows;        // valid query rows in the pair (1 .. 2*tok)
+  int n_qt;          // 1 or 2 query tiles in use
+  int cache_row0, cache_len;   // cached keys (cache packing), all visible
+  int own_row0;      // first own key row (q packing); row i sees own rows own_row0 .. i
+  int n_cache_tiles, n_tiles;
+};
+
+__device__ __forceinline__ int upper_bound_tbl(const int32_t *a, int n, int x) {
+  int lo = 0, hi = n;
+  while (lo < hi) {
+    int mid = (lo + hi) >> 1;
+    if (__ldg(a + mid) <= x) lo = mid + 1; else hi = mid;
+  }
+  return lo;
+}
+
+__device__ __forceinline__ bool resolve_item(const AttnParams &p, int pair, Item &it) {
+  const ba_segments &sg = p.seg;
+  const int pair_tok = 2 * p.tok;
+  if (p.final_only) {
+    if (pair >= __ldg(sg.totals + 3)) return false;
+    int s = upper_bound_tbl(sg.cu_ftile, sg.batch + 1, pair) - 1;
+    int f0 = __ldg(sg.cu_final_seq + s), f1 = __ldg(sg.cu_final_seq + s + 1);
+    it.q_row0 = f0 + (pair - __ldg(sg.cu_ftile + s)) * pair_tok;
+    it.q_rows = min(pair_tok, f1 - it.q_row0);
+    it.cache_row0 = __ldg(sg.cu_cache_seq + s);
+    it.cache_len = __ldg(sg.cu_cache_seq + s + 1) - it.cache_row0;
+    it.own_row0 = f0;
+  } else {
+    if (pair >= __ldg(sg.totals + 2)) return false;
+    int b = upper_bound_tbl(sg.cu_qtile, sg.n_blocks + 1, pair) - 1;
+    int b0 = __ldg(sg.cu_block + b), b1 = __ldg(sg.cu_block + b + 1);
+    it.q_row0 = b0 + (pair - __ldg(sg.cu_qtile + b)) * pair_tok;
+    it.q_rows = min(pair_tok, b1 - it.q_row0);
+    it.cache_row0 = 0;
+    it.cache_len = 0;
+    it.own_row0 = __ldg(sg.block_kv_begin + b);
+  }
+  if (it.q_rows < 1) return false;
+  it.n_qt = it.q_rows > p.tok ? 2 : 1;
+  it.n_cache_tiles = (it.cache_len + kBlockN - 1) / kBlockN;
+  it.n_tiles = it.n_cache_tiles + (it.q_row0 + it.q_rows - it.own_row0 + kBlockN - 1) / kBlockN;
+  return true;
+}
+
+template <int D>
+__global__ void __launch_bounds__(kThreads, 1)
+ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
+                       const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ CUtensorMap tmap_kc,
+                       const __grid_constant__ CUtensorMap tmap_vc, const AttnParams p) {
+  using L = Layout<D>;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  Ctrl *ctrl = reinterpret_cast<Ctrl *>(smem + L::kCtrl);
+
+  if (__ldg(p.seg.totals + 7) != BA_TABLES_VALID) return;
+  Item it;
+  if (!resolve_item(p, blockIdx.x, it)) return;           // uniform over the CTA
+  const int head0 = blockIdx.y * p.hpt;
+  const int kv_head = head0 / p.G;
+  const int tid = threadIdx.x, warp = tid >> 5;
+
+  if (tid == 0) {
+    mbar_init(&ctrl->q_full[0], 1); mbar_init(&ctrl->q_full[1], 1);
+    for (int s = 0; s < kStages; ++s) { mbar_init(&ctrl->kv_full[s], 1); mbar_init(&ctrl->kv_empty[s], 1); }
+    for (int t = 0; t < 2; ++t) {
+      mbar_init(&ctrl->s_full[t], 1); mbar_init(&ctrl->p_full[t], 128); mbar_init(&ctrl->o_done[t], 1);
+    }
+    ctrl->abort_flag = 0;
+    fence_barrier_init();
+  }
+  if (warp == 9) { tmem_alloc(&ctrl->tmem_base, 512); tmem_relinquish(); }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = ctrl->tmem_base;
+  volatile int *abort_flag = &ctrl->abort_flag;
+  const int n_tiles = it.n_tiles;
+
+  if (warp == 8) {
+    // ------------------------------------------------------------ TMA producer
+    if (elect_one()) {
+      prefetch_tmap(&tmap_q); prefetch_tmap(&tmap_k); prefetch_tmap(&tmap_v);
+      for (int t = 0; t < it.n_qt; ++t) {
+        mbar_arrive_expect_tx(&ctrl->q_full[t], L::kTileBytes);
+        for (int c = 0; c < L::kChunks; ++c)
+          tma_load_3d(smem + (t ? L::kQ1 : L::kQ0) + c * L::kRegionBytes, &tmap_q, &ctrl->q_full[t], c * 64, head0,
+                      it.q_row0 + t * p.tok);
+      }
+      int issued = 0;
+      bool ok = true;
+      for (int j = 0; j < n_tiles && ok; ++j) {
+        const bool cached = j < it.n_cache_tiles;
+        const int row = cached ? it.cache_row0 + j * kBlockN : it.own_row0 + (j - it.n_cache_tiles) * kBlockN;
+        for (int kv = 0; kv < 2; ++kv) {
+          const int idx = 2 * j + kv, stage = idx % kStages;
+          ok = mbar_wait(&ctrl->kv_empty[stage], ((idx / kStages) & 1) ^ 1, abort_flag);
+          if (!ok) break;
+          const CUtensorMap *m = cached ? (kv ? &tmap_vc : &tmap_kc) : (kv ? &tmap_v : &tmap_k);
+          mbar_arrive_expect_tx(&ctrl->kv_full[stage], L::kTileBytes);
+          for (int c = 0; c < L::kChunks; ++c)
+            tma_load_3d(smem + L::kRing + stage * L::kTileBytes + c * L::kRegionBytes, m, &ctrl->kv_full[stage],
+                        c * 64, kv_head, row);
+          ++issued;
+        }
+      }
+      if (!ok) {
+        // leave no copy in flight: wait (bounded) for the tiles already requested
+        for (int idx = max(0, issued - kStages); idx < issued; ++idx)
+          for (uint32_t spin = 0; spin < (1u << 20); ++spin)
+            if (mbar_try_wait(&ctrl->kv_full[idx % kStages], (idx / kStages) & 1)) break;
+      }
+    }
+  } else if (warp == 9) {
+    // ------------------------------------------------------------ MMA issuer
+    if (elect_one()) {
+      const uint32_t tS[2] = {tmem, tmem + 128};
+      const uint32_t tO[2] = {tmem + 256, tmem + 384};
+      constexpr uint32_t idesc_qk = make_idesc_bf16(128, kBlockN, 0);
+      constexpr uint32_t idesc_pv = make_idesc_bf16(128, D, 1);
+      const uint32_t q_addr[2] = {smem_u32(smem + L::kQ0), smem_u32(smem + L::kQ1)};
+      const uint32_t ring = smem_u32(smem + L::kRing);
+      bool ok = true;
+      auto wait_kv = [&](int idx) { return mbar_wait(&ctrl->kv_full[idx % kStages], (idx / kStages) & 1, abort_flag); };
+      auto issue_qk = [&](int t, int idx) {
+        const uint32_t kb = ring + (idx % kStages) * L::kTileBytes;
+#pragma unroll
+        for (int k = 0; k < D / 16; ++k) {
+          const uint32_t off = (k >> 2) * L::kRegionBytes + (k & 3) * 32;
+          mma_ss(tS[t], make_smem_desc(q_addr[t] + off, 16, 1024), make_smem_desc(kb + off, 16, 1024), idesc_qk, k > 0);
+        }
+        mma_commit(&ctrl->s_full[t]);
+      };
+      auto issue_pv = [&](int t, int idx, bool first) {
+        const uint32_t vb = ring + (idx % kStages) * L::kTileBytes;
+#pragma unroll
+        for (int k = 0; k < kBlockN / 16; ++k)
+          mma_ts(tO[t], tS[t] + k * 8, make_smem_desc(vb + k * 2048, L::kRegionBytes, 1024), idesc_pv,
+                 (!first || k > 0) ? 1u : 0u);
+      };
+      for (int t = 0; t < it.n_qt && ok; ++t) ok = mbar_wait(&ctrl->q_full[t], 0, abort_flag);
+      if (ok) ok = wait_kv(0);
+      if (ok) {
+        tc_fence_after();
+        for (int t = 0; t < it.n_qt; ++t) issue_qk(t, 0);
+        mma_commit(&ctrl->kv_empty[0]);
+      }
+      for (int j = 0; j < n_tiles && ok; ++j) {
+        const bool last = j + 1 == n_tiles;
+        ok = wait_kv(2 * j + 1);
+        for (int t = 0; t < it.n_qt && ok; ++t) {
+          ok = mbar_wait(&ctrl->p_full[t], j & 1, abort_flag);
+          if (!ok) break;
+          tc_fence_after();
+          issue_pv(t, 2 * j + 1, j == 0);
+          if (last) mma_commit(&ctrl->o_done[t]);
+          if (t + 1 == it.n_qt) mma_commit(&ctrl->kv_empty[(2 * j + 1) % kStages]);
+          if (!last) {
+            if (t == 0) { ok = wait_kv(2 * j + 2); if (!ok) break; tc_fence_after(); }
+            issue_qk(t, 2 * j + 2);
+            if (t + 1 == it.n_qt) mma_commit(&ctrl->kv_empty[(2 * j + 2) % kStages]);
+          }
+        }
+      }
+    }
+  } else if (warp < 8) {
+    // ------------------------------------------------------------ softmax, one thread per tile row
+    const int t = warp >> 2;
+    if (t < it.n_qt) {
+      const int r = tid & 127;
+      const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
+      const uint32_t tS = tmem + t * 128 + lane_off;
+      const uint32_t tO = tmem + 256 + t * 128 + lane_off;
+      const int q_last = it.q_row0 + it.q_rows - 1;
+      const int row_tok = it.q_row0 + t * p.tok + (r >> p.hpt_log2);
+      const bool row_valid = row_tok <= q_last;
+      const int tok_c = min(row_tok, q_last);               // rows past the block behave like its last row
+      const int head = head0 + (r & (p.hpt - 1));
+      const float sl = p.scale_log2;
+      float m_used = -INFINITY, l = 0.f;
+      bool ok = true;
+
+      for (int j = 0; j < n_tiles; ++j) {
+        ok = mbar_wait(&ctrl->s_full[t], j & 1, abort_flag);
+        if (!ok) break;
+        tc_fence_after();
+        uint32_t s[128];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) tmem_ld_32x32b_x32(tS + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[c * 32]));
+        tmem_wait_ld();
+        // visible columns of this tile for this row: 0 .. lim
+        int lim;
+        if (j < it.n_cache_tiles) lim = it.cache_len - j * kBlockN - 1;
+        else lim = tok_c - (it.own_row0 + (j - it.n_cache_tiles) * kBlockN);
+        if (lim < kBlockN - 1) {
+#pragma unroll
+          for (int c = 0; c < 128; ++c)
+            if (c > lim) s[c] = 0xff800000u;                 // -inf
+        }
+        float mx = __uint_as_float(s[0]);
+#pragma unroll
+        for (int c = 1; c < 128; ++c) mx = fmaxf(mx, __uint_as_float(s[c]));
+        const float m_new = fmaxf(m_used, mx);
+        if (j == 0) {
+          m_used = m_new;
+        } else {
+          const bool grow = (m_new - m_used) * sl > kRescaleThreshold;
+          if (__any_sync(0xffffffffu, grow)) {
+            const float alpha = ex2((m_used - m_new) * sl);   // 1 when this row's maximum did not move
+            m_used = m_new;
+            l *= alpha;
+#pragma unroll
+            for (int c = 0; c < D / 32; ++c) {
+              uint32_t o[32];
+              tmem_ld_32x32b_x32(tO + c * 32, o);
+              tmem_wait_ld();
+#pragma unroll
+              for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+              tmem_st_32x32b_x32(tO + c * 32, o);
+            }
+          }
+        }
+        const float neg_m = -m_used * sl;
+        float sum0 = 0.f, sum1 = 0.f;
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          uint32_t pk[32];
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            float p0 = ex2(fmaf(__uint_as_float(s[h * 64 + 2 * i]), sl, neg_m));
+            float p1 = ex2(fmaf(__uint_as_float(s[h * 64 + 2 * i + 1]), sl, neg_m));
+            sum0 += p0; sum1 += p1;
+            __nv_bfloat162 v = __floats2bfloat162_rn(p0, p1);
+            pk[i] = *reinterpret_cast<uint32_t *>(&v);
+          }
+          tmem_st_32x32b_x32(tS + h * 32, pk);
+        }
+        l += sum0 + sum1;
+        tmem_wait_st();
+        tc_fence_before();
+        mbar_arrive(&ctrl->p_full[t]);
+      }
+
+      if (ok) ok = mbar_wait(&ctrl->o_done[t], 0, abort_flag);
+      if (ok) {
+        tc_fence_after();
+        const float inv = 1.f / l;
+        const size_t orow = ((size_t)row_tok * p.Hq + head) * D;
+#pragma unroll
+        for (int c = 0; c < D / 32; ++c) {
+          uint32_t o[32];
+          tmem_ld_32x32b_x32(tO + c * 32, o);
+          tmem_wait_ld();
+          if (row_valid) {
+            if (p.out_f32) {
+              float4 *dst = reinterpret_cast<float4 *>(reinterpret_cast<float *>(p.o) + orow + c * 32);
+#pragma unroll
+              for (int i = 0; i < 8; ++i)
+                dst[i] = make_float4(__uint_as_float(o[4 * i]) * inv, __uint_as_float(o[4 * i + 1]) * inv,
+                                     __uint_as_float(o[4 * i + 2]) * inv, __uint_as_float(o[4 * i + 3]) * inv);
+            } else {
+              uint4 *dst = reinterpret_cast<uint4 *>(reinterpret_cast<__nv_bfloat16 *>(p.o) + orow + c * 32);
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {
+                uint32_t w[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                  __nv_bfloat162 v = __floats2bfloat162_rn(__uint_as_float(o[8 * i + 2 * e]) * inv,
+                                                           __uint_as_float(o[8 * i + 2 * e + 1]) * inv);
+                  w[e] = *reinterpret_cast<uint32_t *>(&v);
+                }
+                dst[i] = make_uint4(w[0], w[1], w[2], w[3]);
+              }
+            }
+          }
+        }
+        if (row_valid && p.lse) p.lse[(size_t)row_tok * p.Hq + head] = (m_used * sl + log2f(l)) * 0.6931471805599453f;
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (tid == 0 && ctrl->abort_flag) ba_record_status(p.status, BA_ERR_TIMEOUT);
+  if (warp == 9) tmem_dealloc(tmem, 512);
+}
+
+// ------------------------------------------------------------------ host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void *p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess) return nullptr;
+    fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+// [rows, heads, d] bf16 viewed as a 3-D tensor (d, head, row); box = 64 columns x box_heads x box_rows, 128-byte swizzle.
+bool make_map(CUtensorMap *m, const void *ptr, int D, int heads, long long rows, int box_heads, int box_rows) {
+  EncodeTiledFn enc = encode_fn();
+  if (!enc || rows < 1) return false;
+  cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)heads, (cuuint64_t)rows};
+  cuuint64_t strides[2] = {(cuuint64_t)D * 2, (cuuint64_t)heads * D * 2};
+  cuuint32_t box[3] = {64, (cuuint32_t)box_heads, (cuuint32_t)box_rows};
+  cuuint32_t es[3] = {1, 1, 1};
+  return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(ptr), dims, strides, box, es,
+             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+// Heads of one KV group packed into a query tile: the largest of 4, 2, 1 that divides the group size.
+int ba_heads_per_tile(const ba_config &c) {
+  int G = c.n_q_heads / c.n_kv_heads;
+  return (G % 4 == 0) ? 4 : (G % 2 == 0) ? 2 : 1;
+}
+
+bool ba_attend_sm100_supported(const ba_ctx *ctx, const ba_attend_args &a) {
+  (void)ctx;
+  return a.v_src_off == nullptr && a.n_q_rows > 0;
+}
+
+ba_status ba_attend_sm100_launch(ba_ctx *ctx, const ba_attend_args &a, const ba_segments *seg,
+                                 cudaStream_t stream) {
+  const int D = ctx->cfg.head_dim, Hq = ctx->cfg.n_q_heads, Hkv = ctx->cfg.n_kv_heads;
+  AttnParams p;
+  p.o = a.o; p.lse = a.lse; p.status = ctx->dev_status; p.out_f32 = a.out_f32;
+  p.Hq = Hq; p.Hkv = Hkv; p.G = Hq / Hkv;
+  p.hpt = ba_heads_per_tile(ctx->cfg);
+  p.hpt_log2 = p.hpt == 4 ? 2 : p.hpt == 2 ? 1 : 0;
+  p.tok = 128 / p.hpt;
+  p.scale = ctx->scale;
+  p.scale_log2 = ctx->scale * 1.4426950408889634f;
+  p.final_only = a.final_only;
+  p.n_q_rows = a.n_q_rows;
+  p.seg = *seg;
+  if (seg->q_tile_tokens != 2 * p.tok) return BA_ERR_INVALID_ARG;
+
+  CUtensorMap tq, tk, tv, tkc, tvc;
+  if (!make_map(&tq, a.q, D, Hq, a.n_q_rows, p.hpt, p.tok)) return BA_ERR_CUDA;
+  if (!make_map(&tk, a.k, D, Hkv, a.n_kv_rows, 1, kBlockN)) return BA_ERR_CUDA;
+  if (!make_map(&tv, a.v, D, Hkv, a.n_kv_rows, 1, kBlockN)) return BA_ERR_CUDA;
+  if (a.final_only && a.n_cache_rows > 0) {
+    if (!make_map(&tkc, a.k_cache, D, Hkv, a.n_cache_rows, 1, kBlockN)) return BA_ERR_CUDA;
+    if (!make_map(&tvc, a.v_cache, D, Hkv, a.n_cache_rows, 1, kBlockN)) return BA_ERR_CUDA;
+  } else {
+    tkc = tk; tvc = tv;
+  }
+  const int pair_tok = 2 * p.tok;
+  const int n_units = a.final_only ? seg->batch : seg->n_blocks;
+  const unsigned pairs_upper = (unsigned)(a.n_q_rows / pair_tok + n_units);
+  dim3 grid(pairs_upper, Hq / p.hpt);
+  // ask for more than half of the SM's shared memory so that two CTAs never share an SM
+  // (each CTA allocates all 512 tensor-memory columns)
+  if (D == 128) {
+    const int smem = Layout<128>::kBytes + 1024;
+    BA_CUDA_TRY(cudaFuncSetAttribute(ba_attend_sm100_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    ba_attend_sm100_kernel<128><<<grid, kThreads, smem, stream>>>(tq, tk, tv, tkc, tvc, p);
+  } else {
+    const int smem = max(Layout<64>::kBytes + 1024, 120 * 1024);
+    BA_CUDA_TRY(cudaFuncSetAttribute(ba_attend_sm100_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    ba_attend_sm100_kernel<64><<<grid, kThreads, smem, stream>>>(tq, tk, tv, tkc, tvc, p);
+  }
+  BA_CUDA_TRY(cudaGetLastError());
+  ctx->launches += 1;
+  return BA_OK;
+}
