@@ -6,7 +6,8 @@ Tolerances.  Integer tables: bit-exact.  Attention outputs written as fp32
 the fp64 oracle, plus a relative Frobenius error <= 5e-3 and log-sum-exp within
 2e-3 (the absolute bounds alone are loose once thousands of keys are averaged).
 Outputs stored as bf16 are compared with the oracle rounded to bf16 under the
-same absolute bounds.  Re-encoded keys are bf16 by contract: each must lie
+same bounds, except that a difference of one bf16 ulp is accepted where the ulp
+itself exceeds 1e-2 (|x| >= 2).  Re-encoded keys are bf16 by contract: each must lie
 within half a bf16 ulp (plus 1e-6 of fp32 noise: a rotation can cancel to a tiny value) of the fp64 value, i.e. be a correct
 rounding of it, and within one ulp of the oracle's own rounding.
 """
@@ -26,11 +27,16 @@ TABLE_KEYS = ["cu_seq", "cu_cache_seq", "cu_final_seq", "cu_block", "block_delta
               "cache_delta", "tok_block", "tok_pos", "tok_pos_local"]
 
 
-def check_attention(o_gpu, o_ref, lse_gpu=None, lse_ref=None, rel=5e-3):
+def check_attention(o_gpu, o_ref, lse_gpu=None, lse_ref=None, rel=5e-3, bf16_store=False):
     o_gpu = np.asarray(o_gpu, dtype=np.float64)
     d = np.abs(o_gpu - o_ref)
     assert np.isfinite(o_gpu).all()
-    assert d.max() <= 1e-2, f"max-abs {d.max()}"
+    if bf16_store:
+        # a bf16 store may land on the neighbouring bf16 value: one ulp, which exceeds 1e-2 once |x| >= 2
+        ulp = 2.0 ** (np.floor(np.log2(np.maximum(np.abs(o_ref), 1e-30))) - 7)
+        assert (d <= np.maximum(1e-2, ulp)).all(), f"max-abs {d.max()}"
+    else:
+        assert d.max() <= 1e-2, f"max-abs {d.max()}"
     assert d.mean() <= 1e-3, f"mean-abs {d.mean()}"
     fro = np.linalg.norm(o_gpu - o_ref) / np.linalg.norm(o_ref)
     assert fro <= rel, f"relative Frobenius {fro}"
@@ -233,7 +239,7 @@ def test_prefill_parity(w, mode):
 
 def test_prefill_bf16_output():
     o, lse, o_ref, lse_ref = run_prefill(W.config2(), B.BA_MODE_BLOCK, B.BA_OUT_BF16)
-    check_attention(o, round_bf16(o_ref), lse, lse_ref, rel=8e-3)
+    check_attention(o, round_bf16(o_ref), lse, lse_ref, rel=8e-3, bf16_store=True)
 
 
 def sampled_rows(w, per_block=8, extra=128, seed=0):
@@ -323,15 +329,18 @@ def test_warm_path_pool_serving_full_size_and_mode_switch():
                       request_pool_idx=w.request_pool_idx[:8])
     ob_, lb, o_ref, lse_ref = run_warm(half, B.BA_MODE_BLOCK)
     check_attention(ob_, o_ref, lb, lse_ref)
+    # final rows see the same keys under both masks: with the values in the same place the two
+    # modes run the same tiles and agree to the last bit
+    op_, lp, _, _ = run_warm(half, B.BA_MODE_BLOCK, v_from_pool=False)
     of_, lf, _, _ = run_warm(half, B.BA_MODE_FULL, v_from_pool=False)
-    # final rows see the same keys under both masks: results agree to the last bit or nearly so
-    assert np.abs(of_ - ob_).max() <= 1e-5
+    check_attention(op_, o_ref, lp, lse_ref)
+    assert np.abs(of_ - op_).max() <= 1e-6 and np.abs(lf - lp).max() <= 1e-6
 
 
 def test_warm_path_32k_full_size():
     w = W.config3(1)
     o, lse, o_ref, lse_ref = run_warm(w, B.BA_MODE_BLOCK, B.BA_OUT_BF16)
-    check_attention(o, round_bf16(o_ref), lse, lse_ref, rel=2e-2)
+    check_attention(o, round_bf16(o_ref), lse, lse_ref, rel=2e-2, bf16_store=True)
     o2, lse2, _, _ = run_warm(w, B.BA_MODE_BLOCK, B.BA_OUT_F32)
     check_attention(o2, o_ref, lse2, lse_ref)
 
