@@ -89,7 +89,13 @@ ba_status ba_workspace_bytes(const ba_config *cfg, int32_t max_blocks, int32_t m
   if (st != BA_OK) return st;
   if (!bytes || max_blocks < 1 || max_q_rows < 0) return BA_ERR_INVALID_ARG;
   size_t table = ba_align_up((size_t)max_blocks * cfg->head_dim * 4, 256);
-  *bytes = stage_bytes_for(max_blocks) + table + 256;
+  // split-KV partial results are only used for short query sides (few work items)
+  size_t split_rows = (size_t)(max_q_rows < 4096 ? max_q_rows : 4096);
+  size_t splits = split_rows * cfg->n_q_heads * (cfg->head_dim + 1) * sizeof(float) * 6;
+  size_t stage = stage_bytes_for(max_blocks);
+  if (stage < 64 * 1024) stage = 64 * 1024;
+  size_t scratch = table > splits ? table : splits;
+  *bytes = stage + ba_align_up(scratch, 256) + 256;
   return BA_OK;
 }
 
@@ -216,7 +222,7 @@ ba_status ba_reencode_k(ba_ctx *ctx, const void *k_src, const int32_t *src_off, 
   BA_CUDA_TRY(cudaSetDevice(ctx->device));
   // scratch: the angle table at the end of the workspace (the staging area is at its start)
   size_t need = ba_align_up((size_t)n_blocks * ctx->cfg.head_dim * 4, 256);  // n_blocks * d/2 * sizeof(float2)
-  if (!ctx->workspace || need > ctx->workspace_bytes) return BA_ERR_WORKSPACE;
+  if (!ctx->workspace || ba_scratch_offset(ctx) + need > ctx->workspace_bytes) return BA_ERR_WORKSPACE;
   float2 *table = (float2 *)((char *)ctx->workspace + (ctx->workspace_bytes - need) / 256 * 256);
   return ba_reencode_launch(ctx, k_src, src_off, n_src_rows, k_dst, cu, delta, n_blocks, n_rows, table,
                             (cudaStream_t)stream);

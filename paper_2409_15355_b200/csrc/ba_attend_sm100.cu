@@ -44,6 +44,9 @@ struct AttnParams {
   float scale, scale_log2;
   int final_only;
   int n_q_rows;
+  int n_splits;                   // > 1: key tiles are divided among gridDim.z CTAs, partial results combined later
+  float *o_part;                  // [n_splits, n_q_rows, Hq, D] fp32, each normalised by its own denominator
+  float *lse_part;                // [n_splits, n_q_rows, Hq] natural-log denominators (-inf: split saw no key)
   ba_segments seg;
 };
 
@@ -150,13 +153,15 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
   tc_fence_after();
   const uint32_t tmem = ctrl->tmem_base;
   volatile int *abort_flag = &ctrl->abort_flag;
-  const int n_tiles = it.n_tiles;
+  // this CTA's share of the item's key tiles: [tile0, tile0 + n_tiles)
+  const int tile0 = (int)(((long long)it.n_tiles * blockIdx.z) / p.n_splits);
+  const int n_tiles = (int)(((long long)it.n_tiles * (blockIdx.z + 1)) / p.n_splits) - tile0;
 
   if (warp == 8) {
     // ------------------------------------------------------------ TMA producer
     if (elect_one()) {
       prefetch_tmap(&tmap_q); prefetch_tmap(&tmap_k); prefetch_tmap(&tmap_v);
-      for (int t = 0; t < it.n_qt; ++t) {
+      for (int t = 0; t < it.n_qt && n_tiles > 0; ++t) {
         mbar_arrive_expect_tx(&ctrl->q_full[t], L::kTileBytes);
         for (int c = 0; c < L::kChunks; ++c)
           tma_load_3d(smem + (t ? L::kQ1 : L::kQ0) + c * L::kRegionBytes, &tmap_q, &ctrl->q_full[t], c * 64, head0,
@@ -165,8 +170,9 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
       int issued = 0;
       bool ok = true;
       for (int j = 0; j < n_tiles && ok; ++j) {
-        const bool cached = j < it.n_cache_tiles;
-        const int row = cached ? it.cache_row0 + j * kBlockN : it.own_row0 + (j - it.n_cache_tiles) * kBlockN;
+        const int jt = tile0 + j;
+        const bool cached = jt < it.n_cache_tiles;
+        const int row = cached ? it.cache_row0 + jt * kBlockN : it.own_row0 + (jt - it.n_cache_tiles) * kBlockN;
         for (int kv = 0; kv < 2; ++kv) {
           const int idx = 2 * j + kv, stage = idx % kStages;
           ok = mbar_wait(&ctrl->kv_empty[stage], ((idx / kStages) & 1) ^ 1, abort_flag);
@@ -213,6 +219,7 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
           mma_ts(tO[t], tS[t] + k * 8, make_smem_desc(vb + k * 2048, L::kRegionBytes, 1024), idesc_pv,
                  (!first || k > 0) ? 1u : 0u);
       };
+      if (n_tiles == 0) ok = false;                         // nothing to do for this split
       for (int t = 0; t < it.n_qt && ok; ++t) ok = mbar_wait(&ctrl->q_full[t], 0, abort_flag);
       if (ok) ok = wait_kv(0);
       if (ok) {
@@ -265,8 +272,9 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
         tmem_wait_ld();
         // visible columns of this tile for this row: 0 .. lim
         int lim;
-        if (j < it.n_cache_tiles) lim = it.cache_len - j * kBlockN - 1;
-        else lim = tok_c - (it.own_row0 + (j - it.n_cache_tiles) * kBlockN);
+        const int jt = tile0 + j;
+        if (jt < it.n_cache_tiles) lim = it.cache_len - jt * kBlockN - 1;
+        else lim = tok_c - (it.own_row0 + (jt - it.n_cache_tiles) * kBlockN);
         if (lim < kBlockN - 1) {
 #pragma unroll
           for (int c = 0; c < 128; ++c)
@@ -281,7 +289,8 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
         } else {
           const bool grow = (m_new - m_used) * sl > kRescaleThreshold;
           if (__any_sync(0xffffffffu, grow)) {
-            const float alpha = ex2((m_used - m_new) * sl);   // 1 when this row's maximum did not move
+            // 1 when this row's maximum did not move (also when the row has seen no key yet)
+            const float alpha = (m_new == -INFINITY) ? 1.f : ex2((m_used - m_new) * sl);
             m_used = m_new;
             l *= alpha;
 #pragma unroll
@@ -295,7 +304,7 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
             }
           }
         }
-        const float neg_m = -m_used * sl;
+        const float neg_m = (m_used == -INFINITY) ? 0.f : -m_used * sl;   // no visible key so far: every p is 0
         float sum0 = 0.f, sum1 = 0.f;
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
@@ -316,19 +325,27 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
         mbar_arrive(&ctrl->p_full[t]);
       }
 
-      if (ok) ok = mbar_wait(&ctrl->o_done[t], 0, abort_flag);
+      if (ok && n_tiles > 0) ok = mbar_wait(&ctrl->o_done[t], 0, abort_flag);
       if (ok) {
         tc_fence_after();
-        const float inv = 1.f / l;
+        const float inv = l > 0.f ? 1.f / l : 0.f;
+        const float lse_val = l > 0.f ? (m_used * sl + log2f(l)) * 0.6931471805599453f : -INFINITY;
         const size_t orow = ((size_t)row_tok * p.Hq + head) * D;
+        const bool partial = p.n_splits > 1;
+        float *part = partial ? p.o_part + (size_t)blockIdx.z * p.n_q_rows * p.Hq * D + orow : nullptr;
 #pragma unroll
         for (int c = 0; c < D / 32; ++c) {
           uint32_t o[32];
-          tmem_ld_32x32b_x32(tO + c * 32, o);
-          tmem_wait_ld();
+          if (n_tiles > 0) {
+            tmem_ld_32x32b_x32(tO + c * 32, o);
+            tmem_wait_ld();
+          } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) o[i] = 0u;
+          }
           if (row_valid) {
-            if (p.out_f32) {
-              float4 *dst = reinterpret_cast<float4 *>(reinterpret_cast<float *>(p.o) + orow + c * 32);
+            if (partial || p.out_f32) {
+              float4 *dst = reinterpret_cast<float4 *>((partial ? part : reinterpret_cast<float *>(p.o) + orow) + c * 32);
 #pragma unroll
               for (int i = 0; i < 8; ++i)
                 dst[i] = make_float4(__uint_as_float(o[4 * i]) * inv, __uint_as_float(o[4 * i + 1]) * inv,
@@ -349,7 +366,10 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
             }
           }
         }
-        if (row_valid && p.lse) p.lse[(size_t)row_tok * p.Hq + head] = (m_used * sl + log2f(l)) * 0.6931471805599453f;
+        if (row_valid) {
+          if (partial) p.lse_part[((size_t)blockIdx.z * p.n_q_rows + row_tok) * p.Hq + head] = lse_val;
+          else if (p.lse) p.lse[(size_t)row_tok * p.Hq + head] = lse_val;
+        }
       }
     }
   }
@@ -358,6 +378,39 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
   __syncthreads();
   if (tid == 0 && ctrl->abort_flag) ba_record_status(p.status, BA_ERR_TIMEOUT);
   if (warp == 9) tmem_dealloc(tmem, 512);
+}
+
+// Merge of split-KV partial results: o = sum_s w_s o_s / sum_s w_s with w_s = exp(lse_s - max lse).
+// One thread per 4 output columns; the order of the sum is fixed, so results are run-to-run stable.
+template <int D>
+__global__ void __launch_bounds__(256)
+ba_combine_splits_kernel(const float *__restrict__ o_part, const float *__restrict__ lse_part, void *o, float *lse,
+                         int n_rows_heads, int n_splits, int out_f32) {
+  const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+  constexpr int kVec = D / 4;
+  const int rh = idx / kVec, v = idx - rh * kVec;
+  if (rh >= n_rows_heads) return;
+  float mx = -INFINITY;
+  for (int s = 0; s < n_splits; ++s) mx = fmaxf(mx, __ldg(lse_part + (size_t)s * n_rows_heads + rh));
+  float den = 0.f;
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+  for (int s = 0; s < n_splits; ++s) {
+    const float ls = __ldg(lse_part + (size_t)s * n_rows_heads + rh);
+    const float w = (ls == -INFINITY) ? 0.f : __expf(ls - mx);
+    const float4 x = __ldg(reinterpret_cast<const float4 *>(o_part + ((size_t)s * n_rows_heads + rh) * D) + v);
+    den += w;
+    acc.x = fmaf(w, x.x, acc.x); acc.y = fmaf(w, x.y, acc.y); acc.z = fmaf(w, x.z, acc.z); acc.w = fmaf(w, x.w, acc.w);
+  }
+  const float inv = 1.f / den;
+  acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
+  if (out_f32) {
+    reinterpret_cast<float4 *>(reinterpret_cast<float *>(o) + (size_t)rh * D)[v] = acc;
+  } else {
+    __nv_bfloat162 a = __floats2bfloat162_rn(acc.x, acc.y), b = __floats2bfloat162_rn(acc.z, acc.w);
+    uint2 w2 = make_uint2(*reinterpret_cast<uint32_t *>(&a), *reinterpret_cast<uint32_t *>(&b));
+    reinterpret_cast<uint2 *>(reinterpret_cast<__nv_bfloat16 *>(o) + (size_t)rh * D)[v] = w2;
+  }
+  if (lse && v == 0) lse[rh] = mx + logf(den);
 }
 
 // ------------------------------------------------------------------ host side
@@ -419,6 +472,33 @@ ba_status ba_attend_sm100_launch(ba_ctx *ctx, const ba_attend_args &a, const ba_
   p.seg = *seg;
   if (seg->q_tile_tokens != 2 * p.tok) return BA_ERR_INVALID_ARG;
 
+  // Split the keys of each work item over several CTAs when the items alone cannot fill the
+  // GPU (a short final block over a long cache).  The split count minimises
+  // waves x (tiles per CTA + a fixed per-CTA cost) and is capped by the workspace.
+  const int pair_tok = 2 * p.tok;
+  const int n_units = a.final_only ? seg->batch : seg->n_blocks;
+  const unsigned pairs_upper = (unsigned)(a.n_q_rows / pair_tok + n_units);
+  const long long items = (long long)((a.n_q_rows + pair_tok - 1) / pair_tok) * (Hq / p.hpt);
+  int n_splits = 1;
+  if (a.final_only && items < 2LL * ctx->sm_count) {
+    const long long avg_tiles = ((long long)a.n_cache_rows / seg->batch + pair_tok) / kBlockN + 1;
+    const size_t per_split = (size_t)a.n_q_rows * Hq * (D + 1) * sizeof(float);
+    const size_t avail = ctx->workspace_bytes > ba_scratch_offset(ctx) ? ctx->workspace_bytes - ba_scratch_offset(ctx) : 0;
+    const int cap = (int)min((size_t)16, per_split ? avail / per_split : 0);
+    long long best = -1;
+    for (int ns = 1; ns <= cap && ns <= avg_tiles; ++ns) {
+      const long long waves = (items * ns + ctx->sm_count - 1) / ctx->sm_count;
+      const long long cost = waves * ((avg_tiles + ns - 1) / ns + 6);
+      if (best < 0 || cost < best) { best = cost; n_splits = ns; }
+    }
+  }
+  p.n_splits = n_splits;
+  p.o_part = nullptr; p.lse_part = nullptr;
+  if (n_splits > 1) {
+    p.o_part = reinterpret_cast<float *>(reinterpret_cast<char *>(ctx->workspace) + ba_scratch_offset(ctx));
+    p.lse_part = p.o_part + (size_t)n_splits * a.n_q_rows * Hq * D;
+  }
+
   CUtensorMap tq, tk, tv, tkc, tvc;
   if (!make_map(&tq, a.q, D, Hq, a.n_q_rows, p.hpt, p.tok)) return BA_ERR_CUDA;
   if (!make_map(&tk, a.k, D, Hkv, a.n_kv_rows, 1, kBlockN)) return BA_ERR_CUDA;
@@ -429,10 +509,7 @@ ba_status ba_attend_sm100_launch(ba_ctx *ctx, const ba_attend_args &a, const ba_
   } else {
     tkc = tk; tvc = tv;
   }
-  const int pair_tok = 2 * p.tok;
-  const int n_units = a.final_only ? seg->batch : seg->n_blocks;
-  const unsigned pairs_upper = (unsigned)(a.n_q_rows / pair_tok + n_units);
-  dim3 grid(pairs_upper, Hq / p.hpt);
+  dim3 grid(pairs_upper, Hq / p.hpt, n_splits);
   // ask for more than half of the SM's shared memory so that two CTAs never share an SM
   // (each CTA allocates all 512 tensor-memory columns)
   if (D == 128) {
@@ -446,5 +523,16 @@ ba_status ba_attend_sm100_launch(ba_ctx *ctx, const ba_attend_args &a, const ba_
   }
   BA_CUDA_TRY(cudaGetLastError());
   ctx->launches += 1;
+  if (n_splits > 1) {
+    const int n_rh = a.n_q_rows * Hq;
+    const long long threads = (long long)n_rh * (D / 4);
+    const unsigned cgrid = (unsigned)((threads + 255) / 256);
+    if (D == 128)
+      ba_combine_splits_kernel<128><<<cgrid, 256, 0, stream>>>(p.o_part, p.lse_part, a.o, a.lse, n_rh, n_splits, a.out_f32);
+    else
+      ba_combine_splits_kernel<64><<<cgrid, 256, 0, stream>>>(p.o_part, p.lse_part, a.o, a.lse, n_rh, n_splits, a.out_f32);
+    BA_CUDA_TRY(cudaGetLastError());
+    ctx->launches += 1;
+  }
   return BA_OK;
 }

@@ -194,12 +194,17 @@ def test_reencode_errors_do_not_fault():
     assert e.value.status == B.BA_ERR_INVALID_ARG
     with pytest.raises(B.BaError):
         B.ba_reencode_k(c.ctx, k.view(-1)[1:], None, 255, out, seg.cache_cu, seg.cache_delta, 4, 255)  # misaligned
-    small = R.Context(4, 2, 64, 1e4, max_blocks=1)
-    big = W.Workload("b", 4, 2, 64, 1e4, [1] * 600, [600], seed=1)
+    # a context created with a workspace too small for the call reports it instead of overrunning
+    small = B.ba_create(c.cfg, 0, 1024)
+    lens = np.ones(600, dtype=np.int32)
+    tb = torch.empty(B.ba_segments_bytes(1, 600, 600), dtype=torch.uint8, device="cuda")
     with pytest.raises(B.BaError) as e:
-        small.segment(big.block_lens, big.seq_nblocks, B.BA_MODE_BLOCK)
+        B.ba_segment(small, lens, np.asarray([600], dtype=np.int32), 1, 600, 600, B.BA_MODE_BLOCK, tb)
     assert e.value.status == B.BA_ERR_WORKSPACE
-    small.close()
+    with pytest.raises(B.BaError) as e:
+        B.ba_reencode_k(small, k, None, 256, out, seg.cache_cu, seg.cache_delta, 4, 256)   # 4 * 64 * 4 = 1024 > room
+    assert e.value.status == B.BA_ERR_WORKSPACE
+    B.ba_destroy(small)
     c.close()
 
 
