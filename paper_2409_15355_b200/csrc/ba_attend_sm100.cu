@@ -157,8 +157,10 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
   const int tile0 = (int)(((long long)it.n_tiles * blockIdx.z) / p.n_splits);
   const int n_tiles = (int)(((long long)it.n_tiles * (blockIdx.z + 1)) / p.n_splits) - tile0;
 
+  // The softmax warps keep a whole 128-column row in registers; the service warps (8-11) need few.
   if (warp == 8) {
     // ------------------------------------------------------------ TMA producer
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
     if (elect_one()) {
       prefetch_tmap(&tmap_q); prefetch_tmap(&tmap_k); prefetch_tmap(&tmap_v);
       for (int t = 0; t < it.n_qt && n_tiles > 0; ++t) {
@@ -194,6 +196,7 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
     }
   } else if (warp == 9) {
     // ------------------------------------------------------------ MMA issuer
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
     if (elect_one()) {
       const uint32_t tS[2] = {tmem, tmem + 128};
       const uint32_t tO[2] = {tmem + 256, tmem + 384};
@@ -245,8 +248,11 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
         }
       }
     }
-  } else if (warp < 8) {
+  } else if (warp >= 10) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
+  } else {
     // ------------------------------------------------------------ softmax, one thread per tile row
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
     const int t = warp >> 2;
     if (t < it.n_qt) {
       const int r = tid & 127;
@@ -280,9 +286,16 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
           for (int c = 0; c < 128; ++c)
             if (c > lim) s[c] = 0xff800000u;                 // -inf
         }
-        float mx = __uint_as_float(s[0]);
+        // eight independent running maxima keep the dependency chains short
+        float mx8[8];
 #pragma unroll
-        for (int c = 1; c < 128; ++c) mx = fmaxf(mx, __uint_as_float(s[c]));
+        for (int i = 0; i < 8; ++i) mx8[i] = __uint_as_float(s[i]);
+#pragma unroll
+        for (int c = 8; c < 128; c += 8)
+#pragma unroll
+          for (int i = 0; i < 8; ++i) mx8[i] = fmaxf(mx8[i], __uint_as_float(s[c + i]));
+        const float mx = fmaxf(fmaxf(fmaxf(mx8[0], mx8[1]), fmaxf(mx8[2], mx8[3])),
+                               fmaxf(fmaxf(mx8[4], mx8[5]), fmaxf(mx8[6], mx8[7])));
         const float m_new = fmaxf(m_used, mx);
         if (j == 0) {
           m_used = m_new;
@@ -305,7 +318,7 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
           }
         }
         const float neg_m = (m_used == -INFINITY) ? 0.f : -m_used * sl;   // no visible key so far: every p is 0
-        float sum0 = 0.f, sum1 = 0.f;
+        float sum[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
           uint32_t pk[32];
@@ -313,13 +326,13 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
           for (int i = 0; i < 32; ++i) {
             float p0 = ex2(fmaf(__uint_as_float(s[h * 64 + 2 * i]), sl, neg_m));
             float p1 = ex2(fmaf(__uint_as_float(s[h * 64 + 2 * i + 1]), sl, neg_m));
-            sum0 += p0; sum1 += p1;
+            sum[(2 * i) & 7] += p0; sum[(2 * i + 1) & 7] += p1;
             __nv_bfloat162 v = __floats2bfloat162_rn(p0, p1);
             pk[i] = *reinterpret_cast<uint32_t *>(&v);
           }
           tmem_st_32x32b_x32(tS + h * 32, pk);
         }
-        l += sum0 + sum1;
+        l += ((sum[0] + sum[1]) + (sum[2] + sum[3])) + ((sum[4] + sum[5]) + (sum[6] + sum[7]));
         tmem_wait_st();
         tc_fence_before();
         mbar_arrive(&ctrl->p_full[t]);
