@@ -27,6 +27,18 @@
 
 using namespace sm100;
 
+// Optional phase timeline of CTA (0,0,0) for tuning: compile with -DBA_TRACE.
+#ifdef BA_TRACE
+__device__ long long g_ba_trace[3][64][8];
+extern "C" int ba_trace_read(long long *dst) { return (int)cudaMemcpyFromSymbol(dst, g_ba_trace, sizeof(g_ba_trace)); }
+#define BA_TR(role, tile, k)                                                                  \
+  do {                                                                                        \
+    if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && (tile) < 64) g_ba_trace[role][tile][k] = clock64(); \
+  } while (0)
+#else
+#define BA_TR(role, tile, k) do { } while (0)
+#endif
+
 namespace {
 
 constexpr int kThreads = 384;
@@ -67,7 +79,7 @@ struct Ctrl {
   uint64_t kv_full[kStages];
   uint64_t kv_empty[kStages];
   uint64_t s_full[2];
-  uint64_t p_full[2];
+  uint64_t p_full[2][2];          // [query tile][half of the P tile]
   uint64_t o_done[2];
   uint32_t tmem_base;
   int abort_flag;
@@ -82,6 +94,33 @@ struct Item {
   int own_row0;      // first own key row (q packing); row i sees own rows own_row0 .. i
   int n_cache_tiles, n_tiles;
 };
+
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+
+// 2^x on the FMA pipe (x <= ~8): round x to the nearest integer n with the 1.5*2^23 trick,
+// evaluate a cubic fit of 2^r on r = x - n in [-0.5, 0.5] (relative error < 8e-5, far below
+// the bf16 rounding applied to the result) and add n to the exponent field.  Can take a
+// fixed share of the columns off the special-function unit (BA_POLY_PERIOD); off by default:
+// the softmax warps are bound by instruction issue, not by that unit, and it measured slower.
+__device__ __forceinline__ float exp2_poly(float x) {
+  x = fmaxf(x, -126.f);
+  const float t = x + 12582912.f;
+  const float r = x - (t - 12582912.f);
+  const float pr = fmaf(fmaf(fmaf(0.055088684f, r, 0.24260405f), r, 0.69327623f), r, 0.99992895f);
+  return __uint_as_float(__float_as_uint(pr) + (__float_as_uint(t) << 23));
+}
+#ifndef BA_POLY_PERIOD
+#define BA_POLY_PERIOD 0
+#endif
+#ifndef BA_SPLIT_P
+#define BA_SPLIT_P 1
+#endif
+constexpr int kPolyPeriod = BA_POLY_PERIOD;    // one column in kPolyPeriod uses exp2_poly (0: none)
+constexpr bool kSplitP = BA_SPLIT_P;             // hand P to the MMA warp in two halves
 
 __device__ __forceinline__ int upper_bound_tbl(const int32_t *a, int n, int x) {
   int lo = 0, hi = n;
@@ -142,7 +181,8 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
     mbar_init(&ctrl->q_full[0], 1); mbar_init(&ctrl->q_full[1], 1);
     for (int s = 0; s < kStages; ++s) { mbar_init(&ctrl->kv_full[s], 1); mbar_init(&ctrl->kv_empty[s], 1); }
     for (int t = 0; t < 2; ++t) {
-      mbar_init(&ctrl->s_full[t], 1); mbar_init(&ctrl->p_full[t], 128); mbar_init(&ctrl->o_done[t], 1);
+      mbar_init(&ctrl->s_full[t], 1); mbar_init(&ctrl->p_full[t][0], 128); mbar_init(&ctrl->p_full[t][1], 128);
+      mbar_init(&ctrl->o_done[t], 1);
     }
     ctrl->abort_flag = 0;
     fence_barrier_init();
@@ -206,21 +246,25 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
       const uint32_t ring = smem_u32(smem + L::kRing);
       bool ok = true;
       auto wait_kv = [&](int idx) { return mbar_wait(&ctrl->kv_full[idx % kStages], (idx / kStages) & 1, abort_flag); };
+      // descriptors differ only in their start-address field: build them once, add offsets (>> 4)
+      const uint64_t q_desc[2] = {make_smem_desc(q_addr[0], 16, 1024), make_smem_desc(q_addr[1], 16, 1024)};
+      const uint64_t k_desc0 = make_smem_desc(ring, 16, 1024);
+      const uint64_t v_desc0 = make_smem_desc(ring, L::kRegionBytes, 1024);
       auto issue_qk = [&](int t, int idx) {
-        const uint32_t kb = ring + (idx % kStages) * L::kTileBytes;
+        const uint64_t kd = k_desc0 + (uint64_t)(((idx % kStages) * L::kTileBytes) >> 4);
 #pragma unroll
         for (int k = 0; k < D / 16; ++k) {
-          const uint32_t off = (k >> 2) * L::kRegionBytes + (k & 3) * 32;
-          mma_ss(tS[t], make_smem_desc(q_addr[t] + off, 16, 1024), make_smem_desc(kb + off, 16, 1024), idesc_qk, k > 0);
+          const uint64_t off = (uint64_t)(((k >> 2) * L::kRegionBytes + (k & 3) * 32) >> 4);
+          mma_ss(tS[t], q_desc[t] + off, kd + off, idesc_qk, k > 0);
         }
         mma_commit(&ctrl->s_full[t]);
       };
-      auto issue_pv = [&](int t, int idx, bool first) {
-        const uint32_t vb = ring + (idx % kStages) * L::kTileBytes;
+      // half = 0: keys 0..63 of the tile, half = 1: keys 64..127
+      auto issue_pv = [&](int t, int idx, bool first, int half) {
+        const uint64_t vd = v_desc0 + (uint64_t)(((idx % kStages) * L::kTileBytes) >> 4);
 #pragma unroll
-        for (int k = 0; k < kBlockN / 16; ++k)
-          mma_ts(tO[t], tS[t] + k * 8, make_smem_desc(vb + k * 2048, L::kRegionBytes, 1024), idesc_pv,
-                 (!first || k > 0) ? 1u : 0u);
+        for (int k = half * 4; k < half * 4 + 4; ++k)
+          mma_ts(tO[t], tS[t] + k * 8, vd + (uint64_t)((k * 2048) >> 4), idesc_pv, (!first || k > 0) ? 1u : 0u);
       };
       if (n_tiles == 0) ok = false;                         // nothing to do for this split
       for (int t = 0; t < it.n_qt && ok; ++t) ok = mbar_wait(&ctrl->q_full[t], 0, abort_flag);
@@ -234,15 +278,23 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
         const bool last = j + 1 == n_tiles;
         ok = wait_kv(2 * j + 1);
         for (int t = 0; t < it.n_qt && ok; ++t) {
-          ok = mbar_wait(&ctrl->p_full[t], j & 1, abort_flag);
+          BA_TR(2, j, t * 4 + 0);
+          ok = mbar_wait(&ctrl->p_full[t][0], j & 1, abort_flag);
           if (!ok) break;
           tc_fence_after();
-          issue_pv(t, 2 * j + 1, j == 0);
+          BA_TR(2, j, t * 4 + 1);
+          issue_pv(t, 2 * j + 1, j == 0, 0);
+          ok = mbar_wait(&ctrl->p_full[t][1], j & 1, abort_flag);
+          if (!ok) break;
+          tc_fence_after();
+          issue_pv(t, 2 * j + 1, j == 0, 1);
+          BA_TR(2, j, t * 4 + 2);
           if (last) mma_commit(&ctrl->o_done[t]);
           if (t + 1 == it.n_qt) mma_commit(&ctrl->kv_empty[(2 * j + 1) % kStages]);
           if (!last) {
             if (t == 0) { ok = wait_kv(2 * j + 2); if (!ok) break; tc_fence_after(); }
             issue_qk(t, 2 * j + 2);
+            BA_TR(2, j, t * 4 + 3);
             if (t + 1 == it.n_qt) mma_commit(&ctrl->kv_empty[(2 * j + 2) % kStages]);
           }
         }
@@ -269,13 +321,16 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
       bool ok = true;
 
       for (int j = 0; j < n_tiles; ++j) {
+        if (r == 0) BA_TR(t, j, 0);
         ok = mbar_wait(&ctrl->s_full[t], j & 1, abort_flag);
         if (!ok) break;
         tc_fence_after();
+        if (r == 0) BA_TR(t, j, 1);
         uint32_t s[128];
 #pragma unroll
         for (int c = 0; c < 4; ++c) tmem_ld_32x32b_x32(tS + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[c * 32]));
         tmem_wait_ld();
+        if (r == 0) BA_TR(t, j, 2);
         // visible columns of this tile for this row: 0 .. lim
         int lim;
         const int jt = tile0 + j;
@@ -286,17 +341,17 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
           for (int c = 0; c < 128; ++c)
             if (c > lim) s[c] = 0xff800000u;                 // -inf
         }
-        // eight independent running maxima keep the dependency chains short
+        // eight independent running maxima (three-input max) keep the dependency chains short
         float mx8[8];
 #pragma unroll
-        for (int i = 0; i < 8; ++i) mx8[i] = __uint_as_float(s[i]);
+        for (int i = 0; i < 8; ++i) mx8[i] = fmaxf(__uint_as_float(s[i]), __uint_as_float(s[8 + i]));
 #pragma unroll
-        for (int c = 8; c < 128; c += 8)
+        for (int c = 16; c < 128; c += 16)
 #pragma unroll
-          for (int i = 0; i < 8; ++i) mx8[i] = fmaxf(mx8[i], __uint_as_float(s[c + i]));
-        const float mx = fmaxf(fmaxf(fmaxf(mx8[0], mx8[1]), fmaxf(mx8[2], mx8[3])),
-                               fmaxf(fmaxf(mx8[4], mx8[5]), fmaxf(mx8[6], mx8[7])));
+          for (int i = 0; i < 8; ++i) mx8[i] = max3(mx8[i], __uint_as_float(s[c + i]), __uint_as_float(s[c + 8 + i]));
+        const float mx = fmaxf(max3(mx8[0], mx8[1], mx8[2]), max3(max3(mx8[3], mx8[4], mx8[5]), mx8[6], mx8[7]));
         const float m_new = fmaxf(m_used, mx);
+        if (r == 0) BA_TR(t, j, 3);
         if (j == 0) {
           m_used = m_new;
         } else {
@@ -319,23 +374,32 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
         }
         const float neg_m = (m_used == -INFINITY) ? 0.f : -m_used * sl;   // no visible key so far: every p is 0
         float sum[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+        // P is handed to the MMA warp in two halves so that PV can start on the first 64 keys
+        // while the second 64 are still being exponentiated
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
           uint32_t pk[32];
 #pragma unroll
           for (int i = 0; i < 32; ++i) {
-            float p0 = ex2(fmaf(__uint_as_float(s[h * 64 + 2 * i]), sl, neg_m));
-            float p1 = ex2(fmaf(__uint_as_float(s[h * 64 + 2 * i + 1]), sl, neg_m));
-            sum[(2 * i) & 7] += p0; sum[(2 * i + 1) & 7] += p1;
+            const int e0 = h * 64 + 2 * i, e1 = e0 + 1;
+            const float x0 = fmaf(__uint_as_float(s[e0]), sl, neg_m);
+            const float x1 = fmaf(__uint_as_float(s[e1]), sl, neg_m);
+            const float p0 = (kPolyPeriod > 0 && e0 % (kPolyPeriod > 0 ? kPolyPeriod : 1) == kPolyPeriod - 1) ? exp2_poly(x0) : ex2(x0);
+            const float p1 = (kPolyPeriod > 0 && e1 % (kPolyPeriod > 0 ? kPolyPeriod : 1) == kPolyPeriod - 1) ? exp2_poly(x1) : ex2(x1);
+            sum[e0 & 7] += p0; sum[e1 & 7] += p1;
             __nv_bfloat162 v = __floats2bfloat162_rn(p0, p1);
             pk[i] = *reinterpret_cast<uint32_t *>(&v);
           }
           tmem_st_32x32b_x32(tS + h * 32, pk);
+          if (kSplitP || h == 1) {
+            tmem_wait_st();
+            tc_fence_before();
+            if (!kSplitP) mbar_arrive(&ctrl->p_full[t][0]);
+            mbar_arrive(&ctrl->p_full[t][h]);
+          }
+          if (r == 0) BA_TR(t, j, 4 + h);
         }
         l += ((sum[0] + sum[1]) + (sum[2] + sum[3])) + ((sum[4] + sum[5]) + (sum[6] + sum[7]));
-        tmem_wait_st();
-        tc_fence_before();
-        mbar_arrive(&ctrl->p_full[t]);
       }
 
       if (ok && n_tiles > 0) ok = mbar_wait(&ctrl->o_done[t], 0, abort_flag);
