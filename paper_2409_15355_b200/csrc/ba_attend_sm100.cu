@@ -29,7 +29,7 @@ using namespace sm100;
 
 // Optional phase timeline of CTA (0,0,0) for tuning: compile with -DBA_TRACE.
 #ifdef BA_TRACE
-__device__ long long g_ba_trace[3][64][8];
+__device__ long long g_ba_trace[4][64][8];
 extern "C" int ba_trace_read(long long *dst) { return (int)cudaMemcpyFromSymbol(dst, g_ba_trace, sizeof(g_ba_trace)); }
 #define BA_TR(role, tile, k)                                                                  \
   do {                                                                                        \
@@ -43,7 +43,10 @@ namespace {
 
 constexpr int kThreads = 384;
 constexpr int kBlockN = 128;      // keys per tile
-constexpr int kStages = 3;        // ring of K/V tiles
+#ifndef BA_STAGES
+#define BA_STAGES 3
+#endif
+constexpr int kStages = BA_STAGES;   // ring of K/V tiles (K_j, V_j, K_j+1, ...)
 constexpr float kRescaleThreshold = 8.0f;
 
 struct AttnParams {
@@ -121,6 +124,10 @@ __device__ __forceinline__ float exp2_poly(float x) {
 #endif
 constexpr int kPolyPeriod = BA_POLY_PERIOD;    // one column in kPolyPeriod uses exp2_poly (0: none)
 constexpr bool kSplitP = BA_SPLIT_P;             // hand P to the MMA warp in two halves
+#ifndef BA_PACKED
+#define BA_PACKED 1
+#endif
+constexpr bool kPacked = BA_PACKED;              // packed fp32x2 arithmetic in the exponent loop
 
 __device__ __forceinline__ int upper_bound_tbl(const int32_t *a, int n, int x) {
   int lo = 0, hi = n;
@@ -276,7 +283,9 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
       }
       for (int j = 0; j < n_tiles && ok; ++j) {
         const bool last = j + 1 == n_tiles;
+        BA_TR(3, j, 0);
         ok = wait_kv(2 * j + 1);
+        BA_TR(3, j, 1);
         for (int t = 0; t < it.n_qt && ok; ++t) {
           BA_TR(2, j, t * 4 + 0);
           ok = mbar_wait(&ctrl->p_full[t][0], j & 1, abort_flag);
@@ -292,7 +301,7 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
           if (last) mma_commit(&ctrl->o_done[t]);
           if (t + 1 == it.n_qt) mma_commit(&ctrl->kv_empty[(2 * j + 1) % kStages]);
           if (!last) {
-            if (t == 0) { ok = wait_kv(2 * j + 2); if (!ok) break; tc_fence_after(); }
+            if (t == 0) { BA_TR(3, j, 2); ok = wait_kv(2 * j + 2); if (!ok) break; tc_fence_after(); BA_TR(3, j, 3); }
             issue_qk(t, 2 * j + 2);
             BA_TR(2, j, t * 4 + 3);
             if (t + 1 == it.n_qt) mma_commit(&ctrl->kv_empty[(2 * j + 2) % kStages]);
@@ -374,6 +383,8 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
         }
         const float neg_m = (m_used == -INFINITY) ? 0.f : -m_used * sl;   // no visible key so far: every p is 0
         float sum[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+        uint64_t sum2[4] = {0ull, 0ull, 0ull, 0ull};       // packed (0.f, 0.f)
+        const uint64_t sl2 = pack2(sl, sl), negm2 = pack2(neg_m, neg_m);
         // P is handed to the MMA warp in two halves so that PV can start on the first 64 keys
         // while the second 64 are still being exponentiated
 #pragma unroll
@@ -382,11 +393,19 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
 #pragma unroll
           for (int i = 0; i < 32; ++i) {
             const int e0 = h * 64 + 2 * i, e1 = e0 + 1;
-            const float x0 = fmaf(__uint_as_float(s[e0]), sl, neg_m);
-            const float x1 = fmaf(__uint_as_float(s[e1]), sl, neg_m);
-            const float p0 = (kPolyPeriod > 0 && e0 % (kPolyPeriod > 0 ? kPolyPeriod : 1) == kPolyPeriod - 1) ? exp2_poly(x0) : ex2(x0);
-            const float p1 = (kPolyPeriod > 0 && e1 % (kPolyPeriod > 0 ? kPolyPeriod : 1) == kPolyPeriod - 1) ? exp2_poly(x1) : ex2(x1);
-            sum[e0 & 7] += p0; sum[e1 & 7] += p1;
+            float p0, p1;
+            if (kPacked) {
+              float x0, x1;
+              unpack2(fma2(pack2(__uint_as_float(s[e0]), __uint_as_float(s[e1])), sl2, negm2), x0, x1);
+              p0 = ex2(x0); p1 = ex2(x1);
+              sum2[i & 3] = add2(sum2[i & 3], pack2(p0, p1));
+            } else {
+              const float x0 = fmaf(__uint_as_float(s[e0]), sl, neg_m);
+              const float x1 = fmaf(__uint_as_float(s[e1]), sl, neg_m);
+              p0 = (kPolyPeriod > 0 && e0 % (kPolyPeriod > 0 ? kPolyPeriod : 1) == kPolyPeriod - 1) ? exp2_poly(x0) : ex2(x0);
+              p1 = (kPolyPeriod > 0 && e1 % (kPolyPeriod > 0 ? kPolyPeriod : 1) == kPolyPeriod - 1) ? exp2_poly(x1) : ex2(x1);
+              sum[e0 & 7] += p0; sum[e1 & 7] += p1;
+            }
             __nv_bfloat162 v = __floats2bfloat162_rn(p0, p1);
             pk[i] = *reinterpret_cast<uint32_t *>(&v);
           }
@@ -398,6 +417,10 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
             mbar_arrive(&ctrl->p_full[t][h]);
           }
           if (r == 0) BA_TR(t, j, 4 + h);
+        }
+        if (kPacked) {
+#pragma unroll
+          for (int i = 0; i < 4; ++i) unpack2(sum2[i], sum[2 * i], sum[2 * i + 1]);
         }
         l += ((sum[0] + sum[1]) + (sum[2] + sum[3])) + ((sum[4] + sum[5]) + (sum[6] + sum[7]));
       }
