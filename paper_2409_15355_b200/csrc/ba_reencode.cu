@@ -10,7 +10,7 @@
 // Kernel 1 builds that table in fp64 (angles reach tens of thousands of radians,
 // far beyond what fast fp32 sin/cos can reduce) and stores it as fp32.
 // Kernel 2 is a pure bandwidth kernel: every thread moves 16-byte vectors
-// (8 bf16), four rows in flight, rotating in fp32 and rounding once to bf16.
+// (8 bf16), eight rows in flight, rotating in fp32 and rounding once to bf16.
 #include "ba_common.cuh"
 
 namespace {
@@ -86,17 +86,25 @@ ba_reencode_kernel(const uint4 *src, uint4 *dst,  // may alias (in place): no __
   uint4 x[kRows], y[kRows];
   int blk[kRows];
   bool live[kRows];
+  // Rows of a thread are close together, so they usually share a block: the block of a row is
+  // looked up again only when the row leaves [c_begin, c_end).
+  int c = 0, c_begin = 0, c_end = -1;
+  long long shift = 0;                                        // source row = row + shift
 #pragma unroll
   for (int i = 0; i < kRows; ++i) {
-    int r = row0 + i * row_step;
+    const int r = row0 + i * row_step;
     live[i] = r < total_rows;
     blk[i] = 0;
     if (live[i]) {
-      int c = upper_bound_i32(cu, n_blocks + 1, r) - 1;
-      c = min(max(c, 0), n_blocks - 1);
+      if (r < c_begin || r >= c_end) {
+        c = upper_bound_i32(cu, n_blocks + 1, r) - 1;
+        c = min(max(c, 0), n_blocks - 1);
+        c_begin = __ldg(cu + c);
+        c_end = __ldg(cu + c + 1);
+        shift = src_off ? (long long)__ldg(src_off + c) - c_begin : 0;
+      }
       blk[i] = c;
-      int c_start = __ldg(cu + c);
-      long long sr = (src_off ? (long long)__ldg(src_off + c) : (long long)c_start) + (r - c_start);
+      const long long sr = r + shift;
       if (sr < 0 || sr >= n_src_rows) {
         ba_record_status(status, BA_ERR_INVALID_ARG);
         live[i] = false;
@@ -107,19 +115,28 @@ ba_reencode_kernel(const uint4 *src, uint4 *dst,  // may alias (in place): no __
       }
     }
   }
+  // (cos, sin) of this thread's rotary pairs, reloaded only when the block changes
+  int t_blk = -1, t_delta = 0;
+  float4 tcs[4];
 #pragma unroll
   for (int i = 0; i < kRows; ++i) {
     if (!live[i]) continue;
     int r = row0 + i * row_step;
     uint4 *q = dst + (long long)r * row_vecs;
-    if (__ldg(delta + blk[i]) == 0) {           // identity: copy bit-exactly
+    if (blk[i] != t_blk) {
+      t_blk = blk[i];
+      t_delta = __ldg(delta + t_blk);
+      const float4 *t4 = reinterpret_cast<const float4 *>(table + t_blk * half_dim + m0);
+      tcs[0] = __ldg(t4); tcs[1] = __ldg(t4 + 1);
+      if (kLayout == BA_ROPE_HALF) { tcs[2] = __ldg(t4 + 2); tcs[3] = __ldg(t4 + 3); }
+    }
+    if (t_delta == 0) {                          // identity: copy bit-exactly
       q[vec_x] = x[i];
       if (kLayout == BA_ROPE_HALF) q[vec_y] = y[i];
       continue;
     }
-    const float4 *t4 = reinterpret_cast<const float4 *>(table + blk[i] * half_dim + m0);
     if (kLayout == BA_ROPE_ADJACENT) {
-      float4 a = __ldg(t4), b = __ldg(t4 + 1);                  // two (cos,sin) pairs per float4
+      const float4 a = tcs[0], b = tcs[1];                      // two (cos,sin) pairs per float4
       uint32_t w[4] = {x[i].x, x[i].y, x[i].z, x[i].w};
       float2 cs[4] = {make_float2(a.x, a.y), make_float2(a.z, a.w), make_float2(b.x, b.y), make_float2(b.z, b.w)};
       uint32_t o[4];
@@ -136,7 +153,7 @@ ba_reencode_kernel(const uint4 *src, uint4 *dst,  // may alias (in place): no __
       uint32_t ox[4], oy[4];
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
-        float4 cs = __ldg(t4 + j);                            // pairs m0+2j, m0+2j+1
+        const float4 cs = tcs[j];                             // pairs m0+2j, m0+2j+1
         float x0, y0, x1, y1;
         rot2(bf16_lo(wx[j]), bf16_lo(wy[j]), make_float2(cs.x, cs.y), x0, y0);
         rot2(bf16_hi(wx[j]), bf16_hi(wy[j]), make_float2(cs.z, cs.w), x1, y1);
@@ -162,7 +179,7 @@ ba_status ba_reencode_launch(ba_ctx *ctx, const void *k_src, const int32_t *src_
   ba_rope_table_kernel<<<(n + 127) / 128, 128, 0, stream>>>(delta, n_blocks, half, k, table);
   BA_CUDA_TRY(cudaGetLastError());
 
-  constexpr int kRows = 4;
+  constexpr int kRows = 8;
   const int row_vecs = H * D / 8;
   const bool adjacent = ctx->cfg.rope_layout == BA_ROPE_ADJACENT;
   const int units = adjacent ? row_vecs : row_vecs / 2;
