@@ -56,7 +56,7 @@ __device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w 
 // a thread moves both.
 // A thread owns one vector column (ADJACENT) or one column pair (HALF) of kRows rows.
 template <int kLayout, int kRows>
-__global__ void __launch_bounds__(1024)
+__global__ void __launch_bounds__(512)
 ba_reencode_kernel(const uint4 *src, uint4 *dst,  // may alias (in place): no __restrict__
                    const int32_t *__restrict__ src_off, int n_src_rows,
                    const int32_t *__restrict__ cu, const int32_t *__restrict__ delta, int n_blocks,
@@ -185,7 +185,7 @@ ba_status ba_reencode_launch(ba_ctx *ctx, const void *k_src, const int32_t *src_
   const int units = adjacent ? row_vecs : row_vecs / 2;
   // threads per CTA: a multiple of the units per row, close to 256
   int threads = units >= 256 ? units : (256 / units) * units;
-  if (threads > 1024) return BA_ERR_UNSUPPORTED;
+  if (threads > 512) return BA_ERR_UNSUPPORTED;   // more than 4096 bf16 per row
   const int rows_per_cta = (threads / units) * kRows;
   const int grid = (n_rows + rows_per_cta - 1) / rows_per_cta;
   if (adjacent)
