@@ -10,7 +10,7 @@
 // Kernel 1 builds that table in fp64 (angles reach tens of thousands of radians,
 // far beyond what fast fp32 sin/cos can reduce) and stores it as fp32.
 // Kernel 2 is a pure bandwidth kernel: every thread moves 16-byte vectors
-// (8 bf16), eight rows in flight, rotating in fp32 and rounding once to bf16.
+// (8 bf16), several rows in flight, rotating in fp32 and rounding once to bf16.
 #include "ba_common.cuh"
 
 namespace {
@@ -179,7 +179,10 @@ ba_status ba_reencode_launch(ba_ctx *ctx, const void *k_src, const int32_t *src_
   ba_rope_table_kernel<<<(n + 127) / 128, 128, 0, stream>>>(delta, n_blocks, half, k, table);
   BA_CUDA_TRY(cudaGetLastError());
 
-  constexpr int kRows = 8;
+#ifndef BA_REENCODE_ROWS
+#define BA_REENCODE_ROWS 2
+#endif
+  constexpr int kRows = BA_REENCODE_ROWS;   // rows in flight per thread
   const int row_vecs = H * D / 8;
   const bool adjacent = ctx->cfg.rope_layout == BA_ROPE_ADJACENT;
   const int units = adjacent ? row_vecs : row_vecs / 2;
