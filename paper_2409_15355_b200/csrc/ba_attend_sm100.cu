@@ -179,7 +179,10 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
 
   if (__ldg(p.seg.totals + 7) != BA_TABLES_VALID) return;
   Item it;
-  if (!resolve_item(p, blockIdx.x, it)) return;           // uniform over the CTA
+  // Work items are taken in descending index order: within a sequence the cost of an item grows
+  // with its index (causal rows see more keys, the final block comes last), so the heaviest
+  // items start first and the launch does not end on them.
+  if (!resolve_item(p, (int)(gridDim.x - 1 - blockIdx.x), it)) return;   // uniform over the CTA
   const int head0 = blockIdx.y * p.hpt;
   const int kv_head = head0 / p.G;
   const int tid = threadIdx.x, warp = tid >> 5;
