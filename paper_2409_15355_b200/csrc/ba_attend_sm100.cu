@@ -34,7 +34,7 @@ __device__ long long g_ba_trace[4][64][8];
 extern "C" int ba_trace_read(long long *dst) { return (int)cudaMemcpyFromSymbol(dst, g_ba_trace, sizeof(g_ba_trace)); }
 #define BA_TR(role, tile, k)                                                                  \
   do {                                                                                        \
-    if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && (tile) < 64) g_ba_trace[role][tile][k] = clock64(); \
+    if (blockIdx.x == 1 && blockIdx.y == 0 && blockIdx.z == 0 && (tile) < 64) g_ba_trace[role][tile][k] = clock64(); \
   } while (0)
 #else
 #define BA_TR(role, tile, k) do { } while (0)
@@ -385,14 +385,15 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
             const float alpha = (m_new == -INFINITY) ? 1.f : ex2((m_used - m_new) * sl);
             m_used = m_new;
             l *= alpha;
-#pragma unroll
-            for (int c = 0; c < D / 64; ++c) {
-              uint32_t o[32];
-              tmem_ld_32x32b_x32(tO + c * 32, o);
+            // rare path: 16 columns at a time keeps the register footprint of the loop small
+#pragma unroll 1
+            for (int c = 0; c < D / 32; ++c) {
+              uint32_t o[16];
+              tmem_ld_32x32b_x16(tO + c * 16, o);
               tmem_wait_ld();
 #pragma unroll
-              for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
-              tmem_st_32x32b_x32(tO + c * 32, o);
+              for (int i = 0; i < 16; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+              tmem_st_32x32b_x16(tO + c * 16, o);
             }
           }
         }
