@@ -7,12 +7,11 @@
 // work item is a pair of query tiles of one block, its keys are one optional
 // "cached" range (all visible) followed by one "own" range (causal).
 //
-// Structure of a CTA (640 threads, one CTA per SM):
-//   warps 0-7   softmax of query tile 0: two threads per tile row (= TMEM lane), warps 0-3 take
-//               key columns 0-63 of a tile, warps 4-7 columns 64-127
-//   warps 8-15  softmax of query tile 1, same split
-//   warp  16    TMA producer: Q tiles once, then K_j, V_j, K_j+1, ... into a ring of stages
-//   warp  17    MMA issuer (one elected thread): S = Q K^T and O += P V with tcgen05.mma,
+// Structure of a CTA (384 threads, one CTA per SM):
+//   warps 0-3   softmax of query tile 0      (one thread per tile row = TMEM lane)
+//   warps 4-7   softmax of query tile 1
+//   warp  8     TMA producer: Q tiles once, then K_j, V_j, K_j+1, ... into a ring of stages
+//   warp  9     MMA issuer (one elected thread): S = Q K^T and O += P V with tcgen05.mma,
 //               accumulators in tensor memory (S0, S1, O0, O1 = 4 x 128 columns)
 // A query tile is 128 rows = (128 / HPT) tokens x HPT query heads of one KV group,
 // so a K/V tile staged once serves every head of the group and both query tiles.
@@ -42,9 +41,7 @@ extern "C" int ba_trace_read(long long *dst) { return (int)cudaMemcpyFromSymbol(
 
 namespace {
 
-constexpr int kThreads = 640;      // 16 softmax warps + 4 service warps
-constexpr int kServiceWarp0 = 16;  // warp 16: TMA producer, warp 17: MMA issuer, 18-19 idle
-constexpr int kXchgStride = 128;
+constexpr int kThreads = 384;
 constexpr int kBlockN = 128;      // keys per tile
 #ifndef BA_STAGES
 #define BA_STAGES 3
@@ -77,7 +74,7 @@ struct Layout {
   static constexpr int kQ1 = kTileBytes;
   static constexpr int kRing = 2 * kTileBytes;
   static constexpr int kCtrl = kRing + kStages * kTileBytes;
-  static constexpr int kBytes = kCtrl + 8192;
+  static constexpr int kBytes = kCtrl + 1024;
 };
 
 struct Ctrl {
@@ -87,10 +84,8 @@ struct Ctrl {
   uint64_t s_full[2];
   uint64_t p_full[2][2];          // [query tile][half of the P tile]
   uint64_t o_done[2];
-  uint64_t xchg_bar[2];           // [query tile]: the two threads of each row exchange partial results
   uint32_t tmem_base;
   int abort_flag;
-  float xchg[2][2][3 * kXchgStride];   // [query tile][column half][slot: tile parity 0/1, final sum][row]
 };
 
 // One work item: two query tiles of one block (or final block) and the key ranges they see.
@@ -124,7 +119,15 @@ __device__ __forceinline__ float exp2_poly(float x) {
 #ifndef BA_POLY_PERIOD
 #define BA_POLY_PERIOD 0
 #endif
+#ifndef BA_SPLIT_P
+#define BA_SPLIT_P 1
+#endif
 constexpr int kPolyPeriod = BA_POLY_PERIOD;    // one column in kPolyPeriod uses exp2_poly (0: none)
+constexpr bool kSplitP = BA_SPLIT_P;             // hand P to the MMA warp in two halves
+#ifndef BA_PACKED
+#define BA_PACKED 1
+#endif
+constexpr bool kPacked = BA_PACKED;              // packed fp32x2 arithmetic in the exponent loop
 
 __device__ __forceinline__ int upper_bound_tbl(const int32_t *a, int n, int x) {
   int lo = 0, hi = n;
@@ -189,12 +192,12 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
     for (int s = 0; s < kStages; ++s) { mbar_init(&ctrl->kv_full[s], 1); mbar_init(&ctrl->kv_empty[s], 1); }
     for (int t = 0; t < 2; ++t) {
       mbar_init(&ctrl->s_full[t], 1); mbar_init(&ctrl->p_full[t][0], 128); mbar_init(&ctrl->p_full[t][1], 128);
-      mbar_init(&ctrl->o_done[t], 1); mbar_init(&ctrl->xchg_bar[t], 256);
+      mbar_init(&ctrl->o_done[t], 1);
     }
     ctrl->abort_flag = 0;
     fence_barrier_init();
   }
-  if (warp == kServiceWarp0 + 1) { tmem_alloc(&ctrl->tmem_base, 512); tmem_relinquish(); }
+  if (warp == 9) { tmem_alloc(&ctrl->tmem_base, 512); tmem_relinquish(); }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -204,10 +207,10 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
   const int tile0 = (int)(((long long)it.n_tiles * blockIdx.z) / p.n_splits);
   const int n_tiles = (int)(((long long)it.n_tiles * (blockIdx.z + 1)) / p.n_splits) - tile0;
 
-  // The softmax warps keep 64 columns of a row in registers; the service warps need few.
-  if (warp == kServiceWarp0) {
+  // The softmax warps keep a whole 128-column row in registers; the service warps (8-11) need few.
+  if (warp == 8) {
     // ------------------------------------------------------------ TMA producer
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 64;");
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
     if (elect_one()) {
       prefetch_tmap(&tmap_q); prefetch_tmap(&tmap_k); prefetch_tmap(&tmap_v);
       for (int t = 0; t < it.n_qt && n_tiles > 0; ++t) {
@@ -241,9 +244,9 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
             if (mbar_try_wait(&ctrl->kv_full[idx % kStages], (idx / kStages) & 1)) break;
       }
     }
-  } else if (warp == kServiceWarp0 + 1) {
+  } else if (warp == 9) {
     // ------------------------------------------------------------ MMA issuer
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 64;");
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
     if (elect_one()) {
       const uint32_t tS[2] = {tmem, tmem + 128};
       const uint32_t tO[2] = {tmem + 256, tmem + 384};
@@ -309,142 +312,132 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
         }
       }
     }
-  } else if (warp >= kServiceWarp0 + 2) {
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 64;");
+  } else if (warp >= 10) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
   } else {
-    // ------------------------------------------------------------ softmax
-    // Two threads per tile row: warp group 2t handles columns 0-63 of query tile t, warp group
-    // 2t+1 columns 64-127 (a warp may touch TMEM lanes 32*(warp%4).. only, so both threads of a
-    // row sit in warps with the same warp%4).  They exchange their partial row maxima through
-    // shared memory and one 256-arrival mbarrier phase per tile (a bounded wait, like all others).
-    asm volatile("setmaxnreg.inc.sync.aligned.u32 104;");
-    const int wg = warp >> 2;
-    const int t = wg >> 1, half = wg & 1;
+    // ------------------------------------------------------------ softmax, one thread per tile row
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
+    const int t = warp >> 2;
     if (t < it.n_qt) {
       const int r = tid & 127;
       const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
-      const uint32_t tS = tmem + t * 128 + lane_off;                       // S row; P goes to columns half*32..
-      const uint32_t tO = tmem + 256 + t * 128 + half * (D / 2) + lane_off; // this thread's half of the O row
+      const uint32_t tS = tmem + t * 128 + lane_off;
+      const uint32_t tO = tmem + 256 + t * 128 + lane_off;
       const int q_last = it.q_row0 + it.q_rows - 1;
       const int row_tok = it.q_row0 + t * p.tok + (r >> p.hpt_log2);
       const bool row_valid = row_tok <= q_last;
       const int tok_c = min(row_tok, q_last);               // rows past the block behave like its last row
       const int head = head0 + (r & (p.hpt - 1));
       const float sl = p.scale_log2;
-      float *xchg_mine = &ctrl->xchg[t][half][r], *xchg_other = &ctrl->xchg[t][half ^ 1][r];
       float m_used = -INFINITY, l = 0.f;
       bool ok = true;
 
       for (int j = 0; j < n_tiles; ++j) {
-        if (r == 0 && half == 0) BA_TR(t, j, 0);
+        if (r == 0) BA_TR(t, j, 0);
         ok = mbar_wait(&ctrl->s_full[t], j & 1, abort_flag);
         if (!ok) break;
         tc_fence_after();
-        if (r == 0 && half == 0) BA_TR(t, j, 1);
-        uint32_t s[64];
-        tmem_ld_32x32b_x32(tS + half * 64, *reinterpret_cast<uint32_t(*)[32]>(&s[0]));
-        tmem_ld_32x32b_x32(tS + half * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&s[32]));
+        if (r == 0) BA_TR(t, j, 1);
+        uint32_t s[128];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) tmem_ld_32x32b_x32(tS + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[c * 32]));
         tmem_wait_ld();
-        if (r == 0 && half == 0) BA_TR(t, j, 2);
-        // visible columns of this tile for this row: 0 .. lim (tile-local), i.e. 0 .. lim - 64*half here
+        if (r == 0) BA_TR(t, j, 2);
+        // visible columns of this tile for this row: 0 .. lim
         int lim;
         const int jt = tile0 + j;
         if (jt < it.n_cache_tiles) lim = it.cache_len - jt * kBlockN - 1;
         else lim = tok_c - (it.own_row0 + (jt - it.n_cache_tiles) * kBlockN);
-        lim -= half * 64;
-        if (lim < 63) {
+        if (lim < kBlockN - 1) {
 #pragma unroll
-          for (int c = 0; c < 64; ++c)
+          for (int c = 0; c < 128; ++c)
             if (c > lim) s[c] = 0xff800000u;                 // -inf
         }
+        // eight independent running maxima (three-input max) keep the dependency chains short
         float mx8[8];
 #pragma unroll
         for (int i = 0; i < 8; ++i) mx8[i] = fmaxf(__uint_as_float(s[i]), __uint_as_float(s[8 + i]));
 #pragma unroll
-        for (int c = 16; c < 64; c += 16)
+        for (int c = 16; c < 128; c += 16)
 #pragma unroll
           for (int i = 0; i < 8; ++i) mx8[i] = max3(mx8[i], __uint_as_float(s[c + i]), __uint_as_float(s[c + 8 + i]));
-        const float mx_half = fmaxf(max3(mx8[0], mx8[1], mx8[2]), max3(max3(mx8[3], mx8[4], mx8[5]), mx8[6], mx8[7]));
-        // exchange with the thread that holds the other 64 columns of this row; the slot is
-        // double-buffered by tile parity
-        xchg_mine[(j & 1) * kXchgStride] = mx_half;
-        mbar_arrive(&ctrl->xchg_bar[t]);
-        ok = mbar_wait(&ctrl->xchg_bar[t], j & 1, abort_flag);
-        if (!ok) break;
-        const float mx = fmaxf(mx_half, xchg_other[(j & 1) * kXchgStride]);
+        const float mx = fmaxf(max3(mx8[0], mx8[1], mx8[2]), max3(max3(mx8[3], mx8[4], mx8[5]), mx8[6], mx8[7]));
         const float m_new = fmaxf(m_used, mx);
-        if (r == 0 && half == 0) BA_TR(t, j, 3);
+        if (r == 0) BA_TR(t, j, 3);
         if (j == 0) {
           m_used = m_new;
         } else {
-          // both threads of a row see the same maxima and their warps cover the same rows, so the
-          // two warps take the same decision
           const bool grow = (m_new - m_used) * sl > kRescaleThreshold;
           if (__any_sync(0xffffffffu, grow)) {
             // 1 when this row's maximum did not move (also when the row has seen no key yet)
             const float alpha = (m_new == -INFINITY) ? 1.f : ex2((m_used - m_new) * sl);
             m_used = m_new;
             l *= alpha;
-            // rare path: 16 columns at a time keeps the register footprint of the loop small
-#pragma unroll 1
+#pragma unroll
             for (int c = 0; c < D / 32; ++c) {
-              uint32_t o[16];
-              tmem_ld_32x32b_x16(tO + c * 16, o);
+              uint32_t o[32];
+              tmem_ld_32x32b_x32(tO + c * 32, o);
               tmem_wait_ld();
 #pragma unroll
-              for (int i = 0; i < 16; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
-              tmem_st_32x32b_x16(tO + c * 16, o);
+              for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+              tmem_st_32x32b_x32(tO + c * 32, o);
             }
           }
         }
         const float neg_m = (m_used == -INFINITY) ? 0.f : -m_used * sl;   // no visible key so far: every p is 0
+        float sum[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
         uint64_t sum2[4] = {0ull, 0ull, 0ull, 0ull};       // packed (0.f, 0.f)
         const uint64_t sl2 = pack2(sl, sl), negm2 = pack2(neg_m, neg_m);
-        // P (bf16, two keys per column) overwrites the S columns: this thread's 64 keys go to
-        // columns half*32 .. half*32+31, and the MMA warp starts PV on a half as soon as it is there
+        // P is handed to the MMA warp in two halves so that PV can start on the first 64 keys
+        // while the second 64 are still being exponentiated
 #pragma unroll
-        for (int q = 0; q < 2; ++q) {
-          uint32_t pk[16];
+        for (int h = 0; h < 2; ++h) {
+          uint32_t pk[32];
 #pragma unroll
-          for (int i = 0; i < 16; ++i) {
-            const int e = q * 32 + 2 * i;
-            float x0, x1;
-            unpack2(fma2(pack2(__uint_as_float(s[e]), __uint_as_float(s[e + 1])), sl2, negm2), x0, x1);
-            const float p0 = (kPolyPeriod > 0 && e % (kPolyPeriod > 0 ? kPolyPeriod : 1) == kPolyPeriod - 1) ? exp2_poly(x0) : ex2(x0);
-            const float p1 = (kPolyPeriod > 0 && (e + 1) % (kPolyPeriod > 0 ? kPolyPeriod : 1) == kPolyPeriod - 1) ? exp2_poly(x1) : ex2(x1);
-            sum2[i & 3] = add2(sum2[i & 3], pack2(p0, p1));
+          for (int i = 0; i < 32; ++i) {
+            const int e0 = h * 64 + 2 * i, e1 = e0 + 1;
+            float p0, p1;
+            if (kPacked) {
+              float x0, x1;
+              unpack2(fma2(pack2(__uint_as_float(s[e0]), __uint_as_float(s[e1])), sl2, negm2), x0, x1);
+              p0 = ex2(x0); p1 = ex2(x1);
+              sum2[i & 3] = add2(sum2[i & 3], pack2(p0, p1));
+            } else {
+              const float x0 = fmaf(__uint_as_float(s[e0]), sl, neg_m);
+              const float x1 = fmaf(__uint_as_float(s[e1]), sl, neg_m);
+              p0 = (kPolyPeriod > 0 && e0 % (kPolyPeriod > 0 ? kPolyPeriod : 1) == kPolyPeriod - 1) ? exp2_poly(x0) : ex2(x0);
+              p1 = (kPolyPeriod > 0 && e1 % (kPolyPeriod > 0 ? kPolyPeriod : 1) == kPolyPeriod - 1) ? exp2_poly(x1) : ex2(x1);
+              sum[e0 & 7] += p0; sum[e1 & 7] += p1;
+            }
             __nv_bfloat162 v = __floats2bfloat162_rn(p0, p1);
             pk[i] = *reinterpret_cast<uint32_t *>(&v);
           }
-          tmem_st_32x32b_x16(tS + half * 32 + q * 16, pk);
+          tmem_st_32x32b_x32(tS + h * 32, pk);
+          if (kSplitP || h == 1) {
+            tmem_wait_st();
+            tc_fence_before();
+            if (!kSplitP) mbar_arrive(&ctrl->p_full[t][0]);
+            mbar_arrive(&ctrl->p_full[t][h]);
+          }
+          if (r == 0) BA_TR(t, j, 4 + h);
         }
-        tmem_wait_st();
-        tc_fence_before();
-        mbar_arrive(&ctrl->p_full[t][half]);
-        if (r == 0 && half == 0) BA_TR(t, j, 4);
-        float s0, s1, s2, s3, s4, s5, s6, s7;
-        unpack2(sum2[0], s0, s1); unpack2(sum2[1], s2, s3); unpack2(sum2[2], s4, s5); unpack2(sum2[3], s6, s7);
-        l += ((s0 + s1) + (s2 + s3)) + ((s4 + s5) + (s6 + s7));
+        if (kPacked) {
+#pragma unroll
+          for (int i = 0; i < 4; ++i) unpack2(sum2[i], sum[2 * i], sum[2 * i + 1]);
+        }
+        l += ((sum[0] + sum[1]) + (sum[2] + sum[3])) + ((sum[4] + sum[5]) + (sum[6] + sum[7]));
       }
 
-      // the two partial denominators of a row are added in a fixed order (columns 0-63 first)
-      if (ok) {
-        xchg_mine[2 * kXchgStride] = l;
-        mbar_arrive(&ctrl->xchg_bar[t]);
-        ok = mbar_wait(&ctrl->xchg_bar[t], n_tiles & 1, abort_flag);
-        const float l_other = xchg_other[2 * kXchgStride];
-        l = half == 0 ? l + l_other : l_other + l;
-      }
       if (ok && n_tiles > 0) ok = mbar_wait(&ctrl->o_done[t], 0, abort_flag);
       if (ok) {
         tc_fence_after();
         const float inv = l > 0.f ? 1.f / l : 0.f;
         const float lse_val = l > 0.f ? (m_used * sl + log2f(l)) * 0.6931471805599453f : -INFINITY;
-        const size_t orow = ((size_t)row_tok * p.Hq + head) * D + half * (D / 2);
+        const size_t orow = ((size_t)row_tok * p.Hq + head) * D;
         const bool partial = p.n_splits > 1;
         float *part = partial ? p.o_part + (size_t)blockIdx.z * p.n_q_rows * p.Hq * D + orow : nullptr;
 #pragma unroll
-        for (int c = 0; c < D / 64; ++c) {
+        for (int c = 0; c < D / 32; ++c) {
           uint32_t o[32];
           if (n_tiles > 0) {
             tmem_ld_32x32b_x32(tO + c * 32, o);
@@ -476,7 +469,7 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
             }
           }
         }
-        if (row_valid && half == 0) {
+        if (row_valid) {
           if (partial) p.lse_part[((size_t)blockIdx.z * p.n_q_rows + row_tok) * p.Hq + head] = lse_val;
           else if (p.lse) p.lse[(size_t)row_tok * p.Hq + head] = lse_val;
         }
@@ -487,7 +480,7 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
   tc_fence_before();
   __syncthreads();
   if (tid == 0 && ctrl->abort_flag) ba_record_status(p.status, BA_ERR_TIMEOUT);
-  if (warp == kServiceWarp0 + 1) tmem_dealloc(tmem, 512);
+  if (warp == 9) tmem_dealloc(tmem, 512);
 }
 
 // Merge of split-KV partial results: o = sum_s w_s o_s / sum_s w_s with w_s = exp(lse_s - max lse).
