@@ -33,7 +33,7 @@ __device__ long long g_ba_trace[4][64][8];
 extern "C" int ba_trace_read(long long *dst) { return (int)cudaMemcpyFromSymbol(dst, g_ba_trace, sizeof(g_ba_trace)); }
 #define BA_TR(role, tile, k)                                                                  \
   do {                                                                                        \
-    if (blockIdx.x == 1 && blockIdx.y == 0 && blockIdx.z == 0 && (tile) < 64) g_ba_trace[role][tile][k] = clock64(); \
+    if (blockIdx.x == 0 && (tile) < 64) g_ba_trace[role][tile][k] = clock64(); \
   } while (0)
 #else
 #define BA_TR(role, tile, k) do { } while (0)
@@ -59,7 +59,8 @@ struct AttnParams {
   float scale, scale_log2;
   int final_only;
   int n_q_rows;
-  int n_splits;                   // > 1: key tiles are divided among gridDim.z CTAs, partial results combined later
+  int n_chunks;                   // head chunks per token (Hq / hpt)
+  int n_splits;                   // > 1: the key tiles of an item are divided among n_splits work entries, combined later
   float *o_part;                  // [n_splits, n_q_rows, Hq, D] fp32, each normalised by its own denominator
   float *lse_part;                // [n_splits, n_q_rows, Hq] natural-log denominators (-inf: split saw no key)
   ba_segments seg;
@@ -79,11 +80,13 @@ struct Layout {
 
 struct Ctrl {
   uint64_t q_full[2];
+  uint64_t q_empty;               // every QK^T of the current item has completed: Q may be reloaded
   uint64_t kv_full[kStages];
   uint64_t kv_empty[kStages];
   uint64_t s_full[2];
   uint64_t p_full[2][2];          // [query tile][half of the P tile]
   uint64_t o_done[2];
+  uint64_t o_free[2];             // the softmax warps have read O_t out of tensor memory
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -167,6 +170,32 @@ __device__ __forceinline__ bool resolve_item(const AttnParams &p, int pair, Item
   return true;
 }
 
+// One entry of a CTA's work list: an item, the heads it covers and its share of the key tiles.
+struct Work {
+  Item it;
+  int head0, kv_head;
+  int tile0, n_tiles;   // key tiles [tile0, tile0 + n_tiles) of the item (split-KV share)
+  int split;
+};
+
+// Decodes work index w: items are ordered heaviest-first (descending pair index: within a
+// sequence an item's cost grows with its index, the final block comes last), then head chunk,
+// then split.  Returns false past the end of the list.
+__device__ __forceinline__ bool next_work(const AttnParams &p, int w, Work &wk) {
+  const int per_pair = p.n_chunks * p.n_splits;
+  const int rank = w / per_pair, rem = w - rank * per_pair;
+  const int total_pairs = __ldg(p.seg.totals + (p.final_only ? 3 : 2));
+  if (rank >= total_pairs) return false;
+  if (!resolve_item(p, total_pairs - 1 - rank, wk.it)) return false;
+  const int chunk = rem / p.n_splits;
+  wk.split = rem - chunk * p.n_splits;
+  wk.head0 = chunk * p.hpt;
+  wk.kv_head = wk.head0 / p.G;
+  wk.tile0 = (int)(((long long)wk.it.n_tiles * wk.split) / p.n_splits);
+  wk.n_tiles = (int)(((long long)wk.it.n_tiles * (wk.split + 1)) / p.n_splits) - wk.tile0;
+  return true;
+}
+
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
 ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
@@ -178,21 +207,14 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
   Ctrl *ctrl = reinterpret_cast<Ctrl *>(smem + L::kCtrl);
 
   if (__ldg(p.seg.totals + 7) != BA_TABLES_VALID) return;
-  Item it;
-  // Work items are taken in descending index order: within a sequence the cost of an item grows
-  // with its index (causal rows see more keys, the final block comes last), so the heaviest
-  // items start first and the launch does not end on them.
-  if (!resolve_item(p, (int)(gridDim.x - 1 - blockIdx.x), it)) return;   // uniform over the CTA
-  const int head0 = blockIdx.y * p.hpt;
-  const int kv_head = head0 / p.G;
   const int tid = threadIdx.x, warp = tid >> 5;
 
   if (tid == 0) {
-    mbar_init(&ctrl->q_full[0], 1); mbar_init(&ctrl->q_full[1], 1);
+    mbar_init(&ctrl->q_full[0], 1); mbar_init(&ctrl->q_full[1], 1); mbar_init(&ctrl->q_empty, 1);
     for (int s = 0; s < kStages; ++s) { mbar_init(&ctrl->kv_full[s], 1); mbar_init(&ctrl->kv_empty[s], 1); }
     for (int t = 0; t < 2; ++t) {
       mbar_init(&ctrl->s_full[t], 1); mbar_init(&ctrl->p_full[t][0], 128); mbar_init(&ctrl->p_full[t][1], 128);
-      mbar_init(&ctrl->o_done[t], 1);
+      mbar_init(&ctrl->o_done[t], 1); mbar_init(&ctrl->o_free[t], 128);
     }
     ctrl->abort_flag = 0;
     fence_barrier_init();
@@ -203,50 +225,62 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
   tc_fence_after();
   const uint32_t tmem = ctrl->tmem_base;
   volatile int *abort_flag = &ctrl->abort_flag;
-  // this CTA's share of the item's key tiles: [tile0, tile0 + n_tiles)
-  const int tile0 = (int)(((long long)it.n_tiles * blockIdx.z) / p.n_splits);
-  const int n_tiles = (int)(((long long)it.n_tiles * (blockIdx.z + 1)) / p.n_splits) - tile0;
 
+  // The CTA is persistent: it walks the work list w = blockIdx.x, blockIdx.x + gridDim.x, ...
+  // Every role derives the same sequence of work items on its own; mbarrier phases simply keep
+  // counting across items, so the producer and the MMA warp run ahead into the next item while
+  // the softmax warps still write out the previous one.
   // The softmax warps keep a whole 128-column row in registers; the service warps (8-11) need few.
   if (warp == 8) {
     // ------------------------------------------------------------ TMA producer
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 88;");
     if (elect_one()) {
       prefetch_tmap(&tmap_q); prefetch_tmap(&tmap_k); prefetch_tmap(&tmap_v);
-      for (int t = 0; t < it.n_qt && n_tiles > 0; ++t) {
-        mbar_arrive_expect_tx(&ctrl->q_full[t], L::kTileBytes);
-        for (int c = 0; c < L::kChunks; ++c)
-          tma_load_3d(smem + (t ? L::kQ1 : L::kQ0) + c * L::kRegionBytes, &tmap_q, &ctrl->q_full[t], c * 64, head0,
-                      it.q_row0 + t * p.tok);
-      }
-      int issued = 0;
+      prefetch_tmap(&tmap_kc); prefetch_tmap(&tmap_vc);
+      int gidx = 0;                       // K/V tiles requested so far (ring position)
+      int n_items = 0;                    // items with at least one tile so far
       bool ok = true;
-      for (int j = 0; j < n_tiles && ok; ++j) {
-        const int jt = tile0 + j;
-        const bool cached = jt < it.n_cache_tiles;
-        const int row = cached ? it.cache_row0 + jt * kBlockN : it.own_row0 + (jt - it.n_cache_tiles) * kBlockN;
-        for (int kv = 0; kv < 2; ++kv) {
-          const int idx = 2 * j + kv, stage = idx % kStages;
-          ok = mbar_wait(&ctrl->kv_empty[stage], ((idx / kStages) & 1) ^ 1, abort_flag);
-          if (!ok) break;
-          const CUtensorMap *m = cached ? (kv ? &tmap_vc : &tmap_kc) : (kv ? &tmap_v : &tmap_k);
-          mbar_arrive_expect_tx(&ctrl->kv_full[stage], L::kTileBytes);
+      Work wk;
+      for (int w = blockIdx.x; ok && next_work(p, w, wk); w += gridDim.x) {
+        if (wk.n_tiles == 0) continue;
+        const Item &it = wk.it;
+        // the Q buffers are free once every QK^T of the previous item has completed
+        ok = mbar_wait(&ctrl->q_empty, (n_items & 1) ^ 1, abort_flag);
+        if (!ok) break;
+        ++n_items;
+        for (int t = 0; t < it.n_qt; ++t) {
+          mbar_arrive_expect_tx(&ctrl->q_full[t], L::kTileBytes);
           for (int c = 0; c < L::kChunks; ++c)
-            tma_load_3d(smem + L::kRing + stage * L::kTileBytes + c * L::kRegionBytes, m, &ctrl->kv_full[stage],
-                        c * 64, kv_head, row);
-          ++issued;
+            tma_load_3d(smem + (t ? L::kQ1 : L::kQ0) + c * L::kRegionBytes, &tmap_q, &ctrl->q_full[t], c * 64,
+                        wk.head0, it.q_row0 + t * p.tok);
+        }
+        for (int j = 0; j < wk.n_tiles && ok; ++j) {
+          const int jt = wk.tile0 + j;
+          const bool cached = jt < it.n_cache_tiles;
+          const int row = cached ? it.cache_row0 + jt * kBlockN : it.own_row0 + (jt - it.n_cache_tiles) * kBlockN;
+          for (int kv = 0; kv < 2; ++kv) {
+            const int stage = gidx % kStages;
+            ok = mbar_wait(&ctrl->kv_empty[stage], ((gidx / kStages) & 1) ^ 1, abort_flag);
+            if (!ok) break;
+            const CUtensorMap *m = cached ? (kv ? &tmap_vc : &tmap_kc) : (kv ? &tmap_v : &tmap_k);
+            mbar_arrive_expect_tx(&ctrl->kv_full[stage], L::kTileBytes);
+            for (int c = 0; c < L::kChunks; ++c)
+              tma_load_3d(smem + L::kRing + stage * L::kTileBytes + c * L::kRegionBytes, m, &ctrl->kv_full[stage],
+                          c * 64, wk.kv_head, row);
+            ++gidx;
+          }
         }
       }
       if (!ok) {
         // leave no copy in flight: wait (bounded) for the tiles already requested
-        for (int idx = max(0, issued - kStages); idx < issued; ++idx)
+        for (int idx = max(0, gidx - kStages); idx < gidx; ++idx)
           for (uint32_t spin = 0; spin < (1u << 20); ++spin)
             if (mbar_try_wait(&ctrl->kv_full[idx % kStages], (idx / kStages) & 1)) break;
       }
     }
   } else if (warp == 9) {
     // ------------------------------------------------------------ MMA issuer
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 88;");
     if (elect_one()) {
       const uint32_t tS[2] = {tmem, tmem + 128};
       const uint32_t tO[2] = {tmem + 256, tmem + 384};
@@ -276,66 +310,89 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
         for (int k = half * 4; k < half * 4 + 4; ++k)
           mma_ts(tO[t], tS[t] + k * 8, vd + (uint64_t)((k * 2048) >> 4), idesc_pv, (!first || k > 0) ? 1u : 0u);
       };
-      if (n_tiles == 0) ok = false;                         // nothing to do for this split
-      for (int t = 0; t < it.n_qt && ok; ++t) ok = mbar_wait(&ctrl->q_full[t], 0, abort_flag);
-      if (ok) ok = wait_kv(0);
-      if (ok) {
+      int gidx = 0;                        // K/V tiles consumed so far (ring position)
+      int q_uses[2] = {0, 0};              // items in which query tile t was loaded
+      int p_uses[2] = {0, 0};              // P tiles of query tile t consumed
+      Work wk;
+      for (int w = blockIdx.x; ok && next_work(p, w, wk); w += gridDim.x) {
+        const int n_tiles = wk.n_tiles, n_qt = wk.it.n_qt;
+        if (n_tiles == 0) continue;
+        for (int t = 0; t < n_qt && ok; ++t) ok = mbar_wait(&ctrl->q_full[t], q_uses[t] & 1, abort_flag);
+        if (ok) ok = wait_kv(gidx);
+        if (!ok) break;
         tc_fence_after();
-        for (int t = 0; t < it.n_qt; ++t) issue_qk(t, 0);
-        mma_commit(&ctrl->kv_empty[0]);
-      }
-      for (int j = 0; j < n_tiles && ok; ++j) {
-        const bool last = j + 1 == n_tiles;
-        BA_TR(3, j, 0);
-        ok = wait_kv(2 * j + 1);
-        BA_TR(3, j, 1);
-        for (int t = 0; t < it.n_qt && ok; ++t) {
-          BA_TR(2, j, t * 4 + 0);
-          ok = mbar_wait(&ctrl->p_full[t][0], j & 1, abort_flag);
-          if (!ok) break;
-          tc_fence_after();
-          BA_TR(2, j, t * 4 + 1);
-          issue_pv(t, 2 * j + 1, j == 0, 0);
-          ok = mbar_wait(&ctrl->p_full[t][1], j & 1, abort_flag);
-          if (!ok) break;
-          tc_fence_after();
-          issue_pv(t, 2 * j + 1, j == 0, 1);
-          BA_TR(2, j, t * 4 + 2);
-          if (last) mma_commit(&ctrl->o_done[t]);
-          if (t + 1 == it.n_qt) mma_commit(&ctrl->kv_empty[(2 * j + 1) % kStages]);
-          if (!last) {
-            if (t == 0) { BA_TR(3, j, 2); ok = wait_kv(2 * j + 2); if (!ok) break; tc_fence_after(); BA_TR(3, j, 3); }
-            issue_qk(t, 2 * j + 2);
-            BA_TR(2, j, t * 4 + 3);
-            if (t + 1 == it.n_qt) mma_commit(&ctrl->kv_empty[(2 * j + 2) % kStages]);
+        for (int t = 0; t < n_qt; ++t) issue_qk(t, gidx);
+        mma_commit(&ctrl->kv_empty[gidx % kStages]);
+        if (n_tiles == 1) mma_commit(&ctrl->q_empty);
+        for (int j = 0; j < n_tiles && ok; ++j) {
+          const bool last = j + 1 == n_tiles;
+          const int iv = gidx + 2 * j + 1, ik = gidx + 2 * j + 2;   // ring positions of V_j and K_(j+1)
+          BA_TR(3, j, 0);
+          ok = wait_kv(iv);
+          BA_TR(3, j, 1);
+          for (int t = 0; t < n_qt && ok; ++t) {
+            BA_TR(2, j, t * 4 + 0);
+            // the first PV of an item overwrites O_t: the previous item's rows must have been read out
+            if (j == 0) { ok = mbar_wait(&ctrl->o_free[t], (q_uses[t] & 1) ^ 1, abort_flag); if (!ok) break; }
+            ok = mbar_wait(&ctrl->p_full[t][0], p_uses[t] & 1, abort_flag);
+            if (!ok) break;
+            tc_fence_after();
+            BA_TR(2, j, t * 4 + 1);
+            issue_pv(t, iv, j == 0, 0);
+            ok = mbar_wait(&ctrl->p_full[t][1], p_uses[t] & 1, abort_flag);
+            if (!ok) break;
+            tc_fence_after();
+            issue_pv(t, iv, j == 0, 1);
+            ++p_uses[t];
+            BA_TR(2, j, t * 4 + 2);
+            if (last) mma_commit(&ctrl->o_done[t]);
+            if (t + 1 == n_qt) mma_commit(&ctrl->kv_empty[iv % kStages]);
+            if (!last) {
+              if (t == 0) { BA_TR(3, j, 2); ok = wait_kv(ik); if (!ok) break; tc_fence_after(); BA_TR(3, j, 3); }
+              issue_qk(t, ik);
+              BA_TR(2, j, t * 4 + 3);
+              if (t + 1 == n_qt) {
+                mma_commit(&ctrl->kv_empty[ik % kStages]);
+                if (j + 2 == n_tiles) mma_commit(&ctrl->q_empty);   // that was the item's last QK^T
+              }
+            }
           }
         }
+        gidx += 2 * n_tiles;
+        for (int t = 0; t < n_qt; ++t) ++q_uses[t];
       }
     }
   } else if (warp >= 10) {
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 88;");
   } else {
     // ------------------------------------------------------------ softmax, one thread per tile row
-    asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 208;");
     const int t = warp >> 2;
-    if (t < it.n_qt) {
-      const int r = tid & 127;
-      const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
-      const uint32_t tS = tmem + t * 128 + lane_off;
-      const uint32_t tO = tmem + 256 + t * 128 + lane_off;
+    const int r = tid & 127;
+    const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
+    const uint32_t tS = tmem + t * 128 + lane_off;
+    const uint32_t tO = tmem + 256 + t * 128 + lane_off;
+    const float sl = p.scale_log2;
+    int s_uses = 0;                       // S tiles of this query tile consumed so far
+    int o_uses = 0;                       // items in which this query tile was active
+    bool ok = true;
+    Work wk;
+    for (int w = blockIdx.x; ok && next_work(p, w, wk); w += gridDim.x) {
+      const Item &it = wk.it;
+      const int n_tiles = wk.n_tiles, tile0 = wk.tile0, head0 = wk.head0;
+      if (t < it.n_qt) {
       const int q_last = it.q_row0 + it.q_rows - 1;
       const int row_tok = it.q_row0 + t * p.tok + (r >> p.hpt_log2);
       const bool row_valid = row_tok <= q_last;
       const int tok_c = min(row_tok, q_last);               // rows past the block behave like its last row
       const int head = head0 + (r & (p.hpt - 1));
-      const float sl = p.scale_log2;
       float m_used = -INFINITY, l = 0.f;
-      bool ok = true;
 
       for (int j = 0; j < n_tiles; ++j) {
         if (r == 0) BA_TR(t, j, 0);
-        ok = mbar_wait(&ctrl->s_full[t], j & 1, abort_flag);
+        ok = mbar_wait(&ctrl->s_full[t], s_uses & 1, abort_flag);
         if (!ok) break;
+        ++s_uses;
         tc_fence_after();
         if (r == 0) BA_TR(t, j, 1);
         uint32_t s[128];
@@ -428,14 +485,14 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
         l += ((sum[0] + sum[1]) + (sum[2] + sum[3])) + ((sum[4] + sum[5]) + (sum[6] + sum[7]));
       }
 
-      if (ok && n_tiles > 0) ok = mbar_wait(&ctrl->o_done[t], 0, abort_flag);
+      if (ok && n_tiles > 0) { ok = mbar_wait(&ctrl->o_done[t], o_uses & 1, abort_flag); ++o_uses; }
       if (ok) {
         tc_fence_after();
         const float inv = l > 0.f ? 1.f / l : 0.f;
         const float lse_val = l > 0.f ? (m_used * sl + log2f(l)) * 0.6931471805599453f : -INFINITY;
         const size_t orow = ((size_t)row_tok * p.Hq + head) * D;
         const bool partial = p.n_splits > 1;
-        float *part = partial ? p.o_part + (size_t)blockIdx.z * p.n_q_rows * p.Hq * D + orow : nullptr;
+        float *part = partial ? p.o_part + (size_t)wk.split * p.n_q_rows * p.Hq * D + orow : nullptr;
 #pragma unroll
         for (int c = 0; c < D / 32; ++c) {
           uint32_t o[32];
@@ -469,10 +526,16 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
             }
           }
         }
+        if (n_tiles > 0) {
+          // O_t has been read out of tensor memory: the next item's first PV may overwrite it
+          tc_fence_before();
+          mbar_arrive(&ctrl->o_free[t]);
+        }
         if (row_valid) {
-          if (partial) p.lse_part[((size_t)blockIdx.z * p.n_q_rows + row_tok) * p.Hq + head] = lse_val;
+          if (partial) p.lse_part[((size_t)wk.split * p.n_q_rows + row_tok) * p.Hq + head] = lse_val;
           else if (p.lse) p.lse[(size_t)row_tok * p.Hq + head] = lse_val;
         }
+      }
       }
     }
   }
@@ -591,11 +654,12 @@ ba_status ba_attend_sm100_launch(ba_ctx *ctx, const ba_attend_args &a, const ba_
     long long best = -1;
     for (int ns = 1; ns <= cap && ns <= avg_tiles; ++ns) {
       const long long waves = (items * ns + ctx->sm_count - 1) / ctx->sm_count;
-      const long long cost = waves * ((avg_tiles + ns - 1) / ns + 6);
+      const long long cost = waves * ((avg_tiles + ns - 1) / ns + 3);
       if (best < 0 || cost < best) { best = cost; n_splits = ns; }
     }
   }
   p.n_splits = n_splits;
+  p.n_chunks = Hq / p.hpt;
   p.o_part = nullptr; p.lse_part = nullptr;
   if (n_splits > 1) {
     p.o_part = reinterpret_cast<float *>(reinterpret_cast<char *>(ctx->workspace) + ba_scratch_offset(ctx));
@@ -612,7 +676,9 @@ ba_status ba_attend_sm100_launch(ba_ctx *ctx, const ba_attend_args &a, const ba_
   } else {
     tkc = tk; tvc = tv;
   }
-  dim3 grid(pairs_upper, Hq / p.hpt, n_splits);
+  // persistent CTAs: one per SM (each owns all of the SM's tensor memory), fewer if the work list is shorter
+  const long long work_upper = (long long)pairs_upper * (Hq / p.hpt) * n_splits;
+  dim3 grid((unsigned)(work_upper < ctx->sm_count ? work_upper : ctx->sm_count));
   // ask for more than half of the SM's shared memory so that two CTAs never share an SM
   // (each CTA allocates all 512 tensor-memory columns)
   if (D == 128) {
