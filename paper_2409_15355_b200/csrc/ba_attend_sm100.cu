@@ -48,6 +48,15 @@ constexpr int kBlockN = 128;      // keys per tile
 #endif
 constexpr int kStages = BA_STAGES;   // ring of K/V tiles (K_j, V_j, K_j+1, ...)
 constexpr float kRescaleThreshold = 8.0f;
+constexpr int kWorkSlots = 4;      // ring of published work entries (power of two)
+// Register split after launch (168 per thread): service warps give registers to the softmax warps.
+// 128 * BA_SVC_REGS + 256 * BA_SMX_REGS <= 384 * 168.
+#ifndef BA_SVC_REGS
+#define BA_SVC_REGS 88
+#endif
+#ifndef BA_SMX_REGS
+#define BA_SMX_REGS 208
+#endif
 
 struct AttnParams {
   void *o;
@@ -63,6 +72,7 @@ struct AttnParams {
   int n_splits;                   // > 1: the key tiles of an item are divided among n_splits work entries, combined later
   float *o_part;                  // [n_splits, n_q_rows, Hq, D] fp32, each normalised by its own denominator
   float *lse_part;                // [n_splits, n_q_rows, Hq] natural-log denominators (-inf: split saw no key)
+  int32_t *work_counter;          // device word, zero at launch: next entry of the work list
   ba_segments seg;
 };
 
@@ -87,6 +97,9 @@ struct Ctrl {
   uint64_t p_full[2][2];          // [query tile][half of the P tile]
   uint64_t o_done[2];
   uint64_t o_free[2];             // the softmax warps have read O_t out of tensor memory
+  uint64_t work_full[kWorkSlots];  // work entry published by the scheduler (producer thread)
+  uint64_t work_empty[kWorkSlots]; // entry read by the MMA thread and the 8 softmax warps
+  int work_ring[kWorkSlots];
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -216,6 +229,7 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
       mbar_init(&ctrl->s_full[t], 1); mbar_init(&ctrl->p_full[t][0], 128); mbar_init(&ctrl->p_full[t][1], 128);
       mbar_init(&ctrl->o_done[t], 1); mbar_init(&ctrl->o_free[t], 128);
     }
+    for (int k = 0; k < kWorkSlots; ++k) { mbar_init(&ctrl->work_full[k], 1); mbar_init(&ctrl->work_empty[k], 9); }
     ctrl->abort_flag = 0;
     fence_barrier_init();
   }
@@ -226,14 +240,14 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
   const uint32_t tmem = ctrl->tmem_base;
   volatile int *abort_flag = &ctrl->abort_flag;
 
-  // The CTA is persistent: it walks the work list w = blockIdx.x, blockIdx.x + gridDim.x, ...
-  // Every role derives the same sequence of work items on its own; mbarrier phases simply keep
-  // counting across items, so the producer and the MMA warp run ahead into the next item while
+  // The CTA is persistent: its producer thread draws entries of the global work list from an
+  // atomic counter (heaviest items first, whichever SM is free takes the next) and publishes them
+  // to the other roles through a small ring; mbarrier phases simply keep counting across items, so the producer and the MMA warp run ahead into the next item while
   // the softmax warps still write out the previous one.
   // The softmax warps keep a whole 128-column row in registers; the service warps (8-11) need few.
   if (warp == 8) {
     // ------------------------------------------------------------ TMA producer
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 88;");
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(BA_SVC_REGS));
     if (elect_one()) {
       prefetch_tmap(&tmap_q); prefetch_tmap(&tmap_k); prefetch_tmap(&tmap_v);
       prefetch_tmap(&tmap_kc); prefetch_tmap(&tmap_vc);
@@ -241,7 +255,18 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
       int n_items = 0;                    // items with at least one tile so far
       bool ok = true;
       Work wk;
-      for (int w = blockIdx.x; ok && next_work(p, w, wk); w += gridDim.x) {
+      int n_work = 0;                    // work entries published so far
+      for (;;) {
+        // scheduler: take the next entry of the global work list and publish it to the other roles
+        const int slot = n_work & (kWorkSlots - 1);
+        ok = mbar_wait(&ctrl->work_empty[slot], ((n_work / kWorkSlots) & 1) ^ 1, abort_flag);
+        if (!ok) break;
+        const int w = atomicAdd(p.work_counter, 1);
+        const bool more = next_work(p, w, wk);
+        ctrl->work_ring[slot] = more ? w : -1;
+        mbar_arrive(&ctrl->work_full[slot]);
+        ++n_work;
+        if (!more) break;
         if (wk.n_tiles == 0) continue;
         const Item &it = wk.it;
         // the Q buffers are free once every QK^T of the previous item has completed
@@ -280,7 +305,7 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
     }
   } else if (warp == 9) {
     // ------------------------------------------------------------ MMA issuer
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 88;");
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(BA_SVC_REGS));
     if (elect_one()) {
       const uint32_t tS[2] = {tmem, tmem + 128};
       const uint32_t tO[2] = {tmem + 256, tmem + 384};
@@ -314,7 +339,15 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
       int q_uses[2] = {0, 0};              // items in which query tile t was loaded
       int p_uses[2] = {0, 0};              // P tiles of query tile t consumed
       Work wk;
-      for (int w = blockIdx.x; ok && next_work(p, w, wk); w += gridDim.x) {
+      int n_work = 0;
+      for (;;) {
+        const int slot = n_work & (kWorkSlots - 1);
+        ok = mbar_wait(&ctrl->work_full[slot], (n_work / kWorkSlots) & 1, abort_flag);
+        if (!ok) break;
+        const int w = ctrl->work_ring[slot];
+        ++n_work;
+        if (w < 0 || !next_work(p, w, wk)) break;
+        mbar_arrive(&ctrl->work_empty[slot]);          // the entry has been decoded into registers
         const int n_tiles = wk.n_tiles, n_qt = wk.it.n_qt;
         if (n_tiles == 0) continue;
         for (int t = 0; t < n_qt && ok; ++t) ok = mbar_wait(&ctrl->q_full[t], q_uses[t] & 1, abort_flag);
@@ -363,10 +396,10 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
       }
     }
   } else if (warp >= 10) {
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 88;");
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(BA_SVC_REGS));
   } else {
     // ------------------------------------------------------------ softmax, one thread per tile row
-    asm volatile("setmaxnreg.inc.sync.aligned.u32 208;");
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(BA_SMX_REGS));
     const int t = warp >> 2;
     const int r = tid & 127;
     const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
@@ -377,7 +410,16 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
     int o_uses = 0;                       // items in which this query tile was active
     bool ok = true;
     Work wk;
-    for (int w = blockIdx.x; ok && next_work(p, w, wk); w += gridDim.x) {
+    int n_work = 0;
+    for (;;) {
+      const int slot = n_work & (kWorkSlots - 1);
+      ok = mbar_wait(&ctrl->work_full[slot], (n_work / kWorkSlots) & 1, abort_flag);
+      if (!ok) break;
+      const int w = ctrl->work_ring[slot];
+      ++n_work;
+      if (w < 0 || !next_work(p, w, wk)) break;
+      __syncwarp();
+      if ((tid & 31) == 0) mbar_arrive(&ctrl->work_empty[slot]);   // one arrival per softmax warp
       const Item &it = wk.it;
       const int n_tiles = wk.n_tiles, tile0 = wk.tile0, head0 = wk.head0;
       if (t < it.n_qt) {
@@ -660,6 +702,10 @@ ba_status ba_attend_sm100_launch(ba_ctx *ctx, const ba_attend_args &a, const ba_
   }
   p.n_splits = n_splits;
   p.n_chunks = Hq / p.hpt;
+  // the work counter lives in the last 256 bytes below the scratch area and is cleared per launch
+  if (!ctx->workspace || ctx->workspace_bytes < ba_scratch_offset(ctx)) return BA_ERR_WORKSPACE;
+  p.work_counter = reinterpret_cast<int32_t *>(reinterpret_cast<char *>(ctx->workspace) + ba_scratch_offset(ctx) - 256);
+  BA_CUDA_TRY(cudaMemsetAsync(p.work_counter, 0, sizeof(int32_t), stream));
   p.o_part = nullptr; p.lse_part = nullptr;
   if (n_splits > 1) {
     p.o_part = reinterpret_cast<float *>(reinterpret_cast<char *>(ctx->workspace) + ba_scratch_offset(ctx));
