@@ -52,10 +52,10 @@ constexpr int kWorkSlots = 4;      // ring of published work entries (power of t
 // Register split after launch (168 per thread): service warps give registers to the softmax warps.
 // 128 * BA_SVC_REGS + 256 * BA_SMX_REGS <= 384 * 168.
 #ifndef BA_SVC_REGS
-#define BA_SVC_REGS 88
+#define BA_SVC_REGS 72
 #endif
 #ifndef BA_SMX_REGS
-#define BA_SMX_REGS 208
+#define BA_SMX_REGS 216
 #endif
 
 struct AttnParams {
