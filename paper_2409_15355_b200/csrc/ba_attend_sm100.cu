@@ -72,6 +72,7 @@ struct AttnParams {
   int n_splits;                   // > 1: the key tiles of an item are divided among n_splits work entries, combined later
   float *o_part;                  // [n_splits, n_q_rows, Hq, D] fp32, each normalised by its own denominator
   float *lse_part;                // [n_splits, n_q_rows, Hq] natural-log denominators (-inf: split saw no key)
+  int persistent;                 // 1: CTAs draw work from work_counter; 0: CTA b handles entry b only
   int32_t *work_counter;          // device word, zero at launch: next entry of the work list
   ba_segments seg;
 };
@@ -261,7 +262,8 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
         const int slot = n_work & (kWorkSlots - 1);
         ok = mbar_wait(&ctrl->work_empty[slot], ((n_work / kWorkSlots) & 1) ^ 1, abort_flag);
         if (!ok) break;
-        const int w = atomicAdd(p.work_counter, 1);
+        // persistent launch: next entry of the global list; one-item launch: this CTA's own entry, then stop
+        const int w = p.persistent ? atomicAdd(p.work_counter, 1) : (n_work == 0 ? (int)blockIdx.x : 0x7fffffff);
         const bool more = next_work(p, w, wk);
         ctrl->work_ring[slot] = more ? w : -1;
         mbar_arrive(&ctrl->work_full[slot]);
@@ -702,10 +704,19 @@ ba_status ba_attend_sm100_launch(ba_ctx *ctx, const ba_attend_args &a, const ba_
   }
   p.n_splits = n_splits;
   p.n_chunks = Hq / p.hpt;
-  // the work counter lives in the last 256 bytes below the scratch area and is cleared per launch
-  if (!ctx->workspace || ctx->workspace_bytes < ba_scratch_offset(ctx)) return BA_ERR_WORKSPACE;
-  p.work_counter = reinterpret_cast<int32_t *>(reinterpret_cast<char *>(ctx->workspace) + ba_scratch_offset(ctx) - 256);
-  BA_CUDA_TRY(cudaMemsetAsync(p.work_counter, 0, sizeof(int32_t), stream));
+  // Many more entries than SMs (cold prefill): persistent CTAs, one per SM, draw entries from a
+  // counter, which hides each item's start-up and write-out behind its neighbours.  A list of at
+  // most two entries per SM (final block over a long cache) gains nothing from that and is
+  // launched one CTA per entry.
+  const long long work_upper = (long long)pairs_upper * (Hq / p.hpt) * n_splits;
+  p.persistent = work_upper > 2LL * ctx->sm_count;
+  p.work_counter = nullptr;
+  if (p.persistent) {
+    // the counter lives in the last 256 bytes below the scratch area and is cleared per launch
+    if (!ctx->workspace || ctx->workspace_bytes < ba_scratch_offset(ctx)) return BA_ERR_WORKSPACE;
+    p.work_counter = reinterpret_cast<int32_t *>(reinterpret_cast<char *>(ctx->workspace) + ba_scratch_offset(ctx) - 256);
+    BA_CUDA_TRY(cudaMemsetAsync(p.work_counter, 0, sizeof(int32_t), stream));
+  }
   p.o_part = nullptr; p.lse_part = nullptr;
   if (n_splits > 1) {
     p.o_part = reinterpret_cast<float *>(reinterpret_cast<char *>(ctx->workspace) + ba_scratch_offset(ctx));
@@ -722,9 +733,7 @@ ba_status ba_attend_sm100_launch(ba_ctx *ctx, const ba_attend_args &a, const ba_
   } else {
     tkc = tk; tvc = tv;
   }
-  // persistent CTAs: one per SM (each owns all of the SM's tensor memory), fewer if the work list is shorter
-  const long long work_upper = (long long)pairs_upper * (Hq / p.hpt) * n_splits;
-  dim3 grid((unsigned)(work_upper < ctx->sm_count ? work_upper : ctx->sm_count));
+  dim3 grid((unsigned)(p.persistent ? ctx->sm_count : work_upper));
   // ask for more than half of the SM's shared memory so that two CTAs never share an SM
   // (each CTA allocates all 512 tensor-memory columns)
   if (D == 128) {
