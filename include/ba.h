@@ -103,6 +103,7 @@ typedef struct {
   /* query-tile tables used by the attention kernels (not part of the bit-exact contract) */
   int32_t *cu_qtile;       /* [B+1] */
   int32_t *cu_ftile;       /* [batch+1] */
+  int32_t *cache_tile_cu;  /* [Bc+1] prefix sum of 128-key tiles per cached block (a tile never spans two blocks) */
   int32_t *totals;         /* [8]: cached tokens, final tokens, q tiles, final tiles, ..., [7] = validity word */
 } ba_segments;
 

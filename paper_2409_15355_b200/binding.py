@@ -41,7 +41,7 @@ class ba_segments(C.Structure):
             "cu_seq", "cu_cache_seq", "cu_final_seq", "cu_seq_block", "cu_block", "block_delta",
             "block_seq", "block_kv_begin", "block_part_off", "block_is_final", "cache_block",
             "cache_cu", "cache_delta", "tok_block", "tok_pos", "tok_pos_local", "cu_qtile",
-            "cu_ftile", "totals")]
+            "cu_ftile", "cache_tile_cu", "totals")]
 
 
 class BaError(RuntimeError):

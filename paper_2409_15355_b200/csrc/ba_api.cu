@@ -42,7 +42,7 @@ int q_tile_tokens(const ba_config &c) { return 2 * 128 / ba_heads_per_tile(c); }
 size_t stage_bytes_for(int32_t max_blocks) { return ba_align_up((size_t)(2 * (size_t)max_blocks + 64) * 4, 256); }
 
 struct TableLayout {
-  size_t off[20];
+  size_t off[24];
   size_t bytes;
 };
 
@@ -62,6 +62,7 @@ TableLayout table_layout(int32_t batch, int32_t B, int32_t T) {
   for (int k = 0; k < 3; ++k) take((size_t)T * 4);            // tok_block, tok_pos, tok_pos_local
   take((size_t)(B + 1) * 4);                                  // cu_qtile
   take((size_t)(batch + 1) * 4);                              // cu_ftile
+  take((size_t)(B + 1) * 4);                                  // cache_tile_cu
   take(8 * 4);                                                // totals
   L.bytes = cur;
   return L;
@@ -206,7 +207,7 @@ ba_status ba_segment(ba_ctx *ctx, const int32_t *block_lens, const int32_t *seq_
   out->block_is_final = (uint8_t *)next();
   out->cache_block = next(); out->cache_cu = next(); out->cache_delta = next();
   out->tok_block = next(); out->tok_pos = next(); out->tok_pos_local = next();
-  out->cu_qtile = next(); out->cu_ftile = next(); out->totals = next();
+  out->cu_qtile = next(); out->cu_ftile = next(); out->cache_tile_cu = next(); out->totals = next();
   return ba_segment_launch(ctx, d_lens, d_nb, batch, n_blocks, n_tokens, mode, out, s);
 }
 

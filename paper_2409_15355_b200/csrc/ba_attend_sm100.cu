@@ -72,6 +72,7 @@ struct AttnParams {
   int n_splits;                   // > 1: the key tiles of an item are divided among n_splits work entries, combined later
   float *o_part;                  // [n_splits, n_q_rows, Hq, D] fp32, each normalised by its own denominator
   float *lse_part;                // [n_splits, n_q_rows, Hq] natural-log denominators (-inf: split saw no key)
+  const int32_t *v_src_off;       // non-null: values of cached block c start at pool row v_src_off[c]
   int persistent;                 // 1: CTAs draw work from work_counter; 0: CTA b handles entry b only
   int32_t *work_counter;          // device word, zero at launch: next entry of the work list
   ba_segments seg;
@@ -101,6 +102,7 @@ struct Ctrl {
   uint64_t work_full[kWorkSlots];  // work entry published by the scheduler (producer thread)
   uint64_t work_empty[kWorkSlots]; // entry read by the MMA thread and the 8 softmax warps
   int work_ring[kWorkSlots];
+  int tile_valid[8];              // pool mode: valid key columns of the cached tiles in flight
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -113,6 +115,8 @@ struct Item {
   int cache_row0, cache_len;   // cached keys (cache packing), all visible
   int own_row0;      // first own key row (q packing); row i sees own rows own_row0 .. i
   int n_cache_tiles, n_tiles;
+  int cb0;           // index (cache order) of the sequence's first cached block
+  int ctile0;        // cache_tile_cu[cb0]: pool mode walks cached keys block by block
 };
 
 __device__ __forceinline__ float max3(float a, float b, float c) {
@@ -167,6 +171,10 @@ __device__ __forceinline__ bool resolve_item(const AttnParams &p, int pair, Item
     it.cache_row0 = __ldg(sg.cu_cache_seq + s);
     it.cache_len = __ldg(sg.cu_cache_seq + s + 1) - it.cache_row0;
     it.own_row0 = f0;
+    it.cb0 = __ldg(sg.cu_seq_block + s) - s;           // every earlier sequence has one final block
+    it.ctile0 = __ldg(sg.cache_tile_cu + it.cb0);
+    it.n_cache_tiles = p.v_src_off ? __ldg(sg.cache_tile_cu + (__ldg(sg.cu_seq_block + s + 1) - s - 1)) - it.ctile0
+                                   : (it.cache_len + kBlockN - 1) / kBlockN;
   } else {
     if (pair >= __ldg(sg.totals + 2)) return false;
     int b = upper_bound_tbl(sg.cu_qtile, sg.n_blocks + 1, pair) - 1;
@@ -176,10 +184,10 @@ __device__ __forceinline__ bool resolve_item(const AttnParams &p, int pair, Item
     it.cache_row0 = 0;
     it.cache_len = 0;
     it.own_row0 = __ldg(sg.block_kv_begin + b);
+    it.cb0 = 0; it.ctile0 = 0; it.n_cache_tiles = 0;
   }
   if (it.q_rows < 1) return false;
   it.n_qt = it.q_rows > p.tok ? 2 : 1;
-  it.n_cache_tiles = (it.cache_len + kBlockN - 1) / kBlockN;
   it.n_tiles = it.n_cache_tiles + (it.q_row0 + it.q_rows - it.own_row0 + kBlockN - 1) / kBlockN;
   return true;
 }
@@ -281,10 +289,35 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
             tma_load_3d(smem + (t ? L::kQ1 : L::kQ0) + c * L::kRegionBytes, &tmap_q, &ctrl->q_full[t], c * 64,
                         wk.head0, it.q_row0 + t * p.tok);
         }
+        // pool mode: cached keys are walked block by block (block pc, row offset poff inside it)
+        int pc = 0, poff = 0;
+        if (p.v_src_off && wk.tile0 < it.n_cache_tiles) {
+          const int target = it.ctile0 + wk.tile0;
+          // last block whose first tile is <= target; the sequence's blocks follow cb0 in cache order
+          int lo = it.cb0, hi = p.seg.n_cached_blocks;
+          while (lo < hi) {
+            const int mid = (lo + hi + 1) >> 1;
+            if (__ldg(p.seg.cache_tile_cu + mid) <= target) lo = mid; else hi = mid - 1;
+          }
+          pc = lo;
+          poff = (target - __ldg(p.seg.cache_tile_cu + pc)) * kBlockN;
+        }
         for (int j = 0; j < wk.n_tiles && ok; ++j) {
           const int jt = wk.tile0 + j;
           const bool cached = jt < it.n_cache_tiles;
-          const int row = cached ? it.cache_row0 + jt * kBlockN : it.own_row0 + (jt - it.n_cache_tiles) * kBlockN;
+          int k_row, v_row;
+          if (!cached) {
+            k_row = v_row = it.own_row0 + (jt - it.n_cache_tiles) * kBlockN;
+          } else if (!p.v_src_off) {
+            k_row = v_row = it.cache_row0 + jt * kBlockN;
+          } else {
+            const int c_begin = __ldg(p.seg.cache_cu + pc), c_len = __ldg(p.seg.cache_cu + pc + 1) - c_begin;
+            k_row = c_begin + poff;
+            v_row = __ldg(p.v_src_off + pc) + poff;
+            ctrl->tile_valid[(gidx >> 1) & 7] = min(kBlockN, c_len - poff);   // read by the softmax warps
+            poff += kBlockN;
+            if (poff >= c_len) { ++pc; poff = 0; }
+          }
           for (int kv = 0; kv < 2; ++kv) {
             const int stage = gidx % kStages;
             ok = mbar_wait(&ctrl->kv_empty[stage], ((gidx / kStages) & 1) ^ 1, abort_flag);
@@ -293,7 +326,7 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
             mbar_arrive_expect_tx(&ctrl->kv_full[stage], L::kTileBytes);
             for (int c = 0; c < L::kChunks; ++c)
               tma_load_3d(smem + L::kRing + stage * L::kTileBytes + c * L::kRegionBytes, m, &ctrl->kv_full[stage],
-                          c * 64, wk.kv_head, row);
+                          c * 64, wk.kv_head, kv ? v_row : k_row);
             ++gidx;
           }
         }
@@ -410,6 +443,7 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
     const float sl = p.scale_log2;
     int s_uses = 0;                       // S tiles of this query tile consumed so far
     int o_uses = 0;                       // items in which this query tile was active
+    int tiles_before = 0;                 // key tiles of all earlier items (the producer counts the same way)
     bool ok = true;
     Work wk;
     int n_work = 0;
@@ -447,7 +481,8 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
         // visible columns of this tile for this row: 0 .. lim
         int lim;
         const int jt = tile0 + j;
-        if (jt < it.n_cache_tiles) lim = it.cache_len - jt * kBlockN - 1;
+        if (jt < it.n_cache_tiles) lim = p.v_src_off ? ctrl->tile_valid[(tiles_before + j) & 7] - 1
+                                                     : it.cache_len - jt * kBlockN - 1;
         else lim = tok_c - (it.own_row0 + (jt - it.n_cache_tiles) * kBlockN);
         if (lim < kBlockN - 1) {
 #pragma unroll
@@ -581,6 +616,7 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
         }
       }
       }
+      tiles_before += n_tiles;
     }
   }
 
@@ -663,7 +699,7 @@ int ba_heads_per_tile(const ba_config &c) {
 
 bool ba_attend_sm100_supported(const ba_ctx *ctx, const ba_attend_args &a) {
   (void)ctx;
-  return a.v_src_off == nullptr && a.n_q_rows > 0;
+  return a.n_q_rows > 0;
 }
 
 ba_status ba_attend_sm100_launch(ba_ctx *ctx, const ba_attend_args &a, const ba_segments *seg,
@@ -678,6 +714,7 @@ ba_status ba_attend_sm100_launch(ba_ctx *ctx, const ba_attend_args &a, const ba_
   p.scale = ctx->scale;
   p.scale_log2 = ctx->scale * 1.4426950408889634f;
   p.final_only = a.final_only;
+  p.v_src_off = a.final_only ? a.v_src_off : nullptr;
   p.n_q_rows = a.n_q_rows;
   p.seg = *seg;
   if (seg->q_tile_tokens != 2 * p.tok) return BA_ERR_INVALID_ARG;
@@ -729,7 +766,7 @@ ba_status ba_attend_sm100_launch(ba_ctx *ctx, const ba_attend_args &a, const ba_
   if (!make_map(&tv, a.v, D, Hkv, a.n_kv_rows, 1, kBlockN)) return BA_ERR_CUDA;
   if (a.final_only && a.n_cache_rows > 0) {
     if (!make_map(&tkc, a.k_cache, D, Hkv, a.n_cache_rows, 1, kBlockN)) return BA_ERR_CUDA;
-    if (!make_map(&tvc, a.v_cache, D, Hkv, a.n_cache_rows, 1, kBlockN)) return BA_ERR_CUDA;
+    if (!make_map(&tvc, a.v_cache, D, Hkv, a.v_src_off ? a.n_v_rows : a.n_cache_rows, 1, kBlockN)) return BA_ERR_CUDA;
   } else {
     tkc = tk; tvc = tv;
   }

@@ -81,7 +81,7 @@ ba_segment_blocks_kernel(const int32_t *__restrict__ lens, const int32_t *__rest
   }
 
   // --- per-block prefix sums: rows (prompt, cache, final packing) and query tiles
-  int c_all = 0, c_cache = 0, c_final = 0, c_tile = 0;
+  int c_all = 0, c_cache = 0, c_final = 0, c_tile = 0, c_ktile = 0;
   for (int base = 0; base < B; base += kScanThreads) {
     int b = base + tid;
     int len = 0, fin = 0, s = 0;
@@ -91,11 +91,12 @@ ba_segment_blocks_kernel(const int32_t *__restrict__ lens, const int32_t *__rest
       s = upper_bound(seg.cu_seq_block, batch + 1, b) - 1;
       fin = (b == seg.cu_seq_block[s + 1] - 1);
     }
-    int t_all, t_cache, t_final, t_tile;
+    int t_all, t_cache, t_final, t_tile, t_ktile;
     int e_all = cta_exclusive_scan(len, scan_smem, t_all);
     int e_cache = cta_exclusive_scan(fin ? 0 : len, scan_smem, t_cache);
     int e_final = cta_exclusive_scan(fin ? len : 0, scan_smem, t_final);
     int e_tile = cta_exclusive_scan((len + tile_tok - 1) / tile_tok, scan_smem, t_tile);
+    int e_ktile = cta_exclusive_scan(fin ? 0 : (len + 127) / 128, scan_smem, t_ktile);
     if (b < B) {
       seg.cu_block[b] = c_all + e_all;
       seg.block_seq[b] = s;
@@ -107,13 +108,15 @@ ba_segment_blocks_kernel(const int32_t *__restrict__ lens, const int32_t *__rest
         int c = b - s;
         seg.cache_block[c] = b;
         seg.cache_cu[c] = c_cache + e_cache;
+        seg.cache_tile_cu[c] = c_ktile + e_ktile;
       }
     }
-    c_all += t_all; c_cache += t_cache; c_final += t_final; c_tile += t_tile;
+    c_all += t_all; c_cache += t_cache; c_final += t_final; c_tile += t_tile; c_ktile += t_ktile;
   }
   if (tid == 0) {
     seg.cu_block[B] = c_all;
     seg.cache_cu[B - batch] = c_cache;
+    seg.cache_tile_cu[B - batch] = c_ktile;
     seg.cu_qtile[B] = c_tile;
     seg.totals[0] = c_cache;
     seg.totals[1] = c_final;

@@ -77,7 +77,7 @@ _TABLE_SIZES = {
     "block_seq": ("n_blocks", 0), "block_kv_begin": ("n_blocks", 0), "block_part_off": ("n_blocks", 0),
     "cache_block": ("n_cached_blocks", 0), "cache_cu": ("n_cached_blocks", 1),
     "cache_delta": ("n_cached_blocks", 0), "tok_block": ("n_tokens", 0), "tok_pos": ("n_tokens", 0),
-    "tok_pos_local": ("n_tokens", 0), "cu_qtile": ("n_blocks", 1), "cu_ftile": ("batch", 1),
+    "tok_pos_local": ("n_tokens", 0), "cu_qtile": ("n_blocks", 1), "cu_ftile": ("batch", 1), "cache_tile_cu": ("n_cached_blocks", 1),
 }
 
 
