@@ -5,11 +5,8 @@
 
 #include "ba_common.cuh"
 
-ba_status ba_attend_simt_launch(ba_ctx *ctx, const ba_attend_args &a, const ba_segments *seg,
-                                cudaStream_t stream);
 ba_status ba_attend_sm100_launch(ba_ctx *ctx, const ba_attend_args &a, const ba_segments *seg,
                                  cudaStream_t stream);
-bool ba_attend_sm100_supported(const ba_ctx *ctx, const ba_attend_args &a);
 int ba_heads_per_tile(const ba_config &c);
 
 namespace {
@@ -284,7 +281,5 @@ ba_status ba_final_attend(ba_ctx *ctx, const void *q_f, const void *k_f, const v
 ba_status ba_attend_launch(ba_ctx *ctx, const ba_attend_args &a, const ba_segments *seg,
                            cudaStream_t stream) {
   if (a.n_q_rows == 0) return BA_OK;
-  // the tensor-core kernel takes every case except values gathered from a pool by index
-  if (ba_attend_sm100_supported(ctx, a)) return ba_attend_sm100_launch(ctx, a, seg, stream);
-  return ba_attend_simt_launch(ctx, a, seg, stream);
+  return ba_attend_sm100_launch(ctx, a, seg, stream);
 }

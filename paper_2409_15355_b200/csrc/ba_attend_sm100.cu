@@ -697,11 +697,6 @@ int ba_heads_per_tile(const ba_config &c) {
   return (G % 4 == 0) ? 4 : (G % 2 == 0) ? 2 : 1;
 }
 
-bool ba_attend_sm100_supported(const ba_ctx *ctx, const ba_attend_args &a) {
-  (void)ctx;
-  return a.n_q_rows > 0;
-}
-
 ba_status ba_attend_sm100_launch(ba_ctx *ctx, const ba_attend_args &a, const ba_segments *seg,
                                  cudaStream_t stream) {
   const int D = ctx->cfg.head_dim, Hq = ctx->cfg.n_q_heads, Hkv = ctx->cfg.n_kv_heads;
