@@ -122,27 +122,40 @@ def aggregate(ms_local: float, layer_jobs_local: float, device=None):
 
 
 # --------------------------------------------------------------------------- the oracle legs
-def oracle_layer_sample(w, n_rows: int, layer: int = 0):
-    """Time the fp64 oracle on one layer: re-encode of all cached blocks plus
-    final attend for the first `n_rows` rows of the final block; scale the
-    attend part to the whole final block.  Returns microseconds per layer."""
-    from oracle import block_attention as ob
-    from paper_2409_15355_b200 import workloads as W
-    x = W.warm_inputs(w, layer)
-    t = ob.segment_tables(w.block_lens, w.seq_nblocks)
-    Lf = w.final_lens()[0]
-    n_rows = min(n_rows, Lf)
-    kc, vc = W.bf16_bits_to_f64(x["k_cache"]), W.bf16_bits_to_f64(x["v_cache"])
-    qf, kf, vf = (W.bf16_bits_to_f64(x[k]) for k in ("q_f", "k_f", "v_f"))
-    t0 = time.perf_counter()
-    k_re = ob.reencode_blocks(kc, None, t["cache_cu"], t["cache_delta"], w.rope_theta)
-    t1 = time.perf_counter()
-    k_all = np.concatenate([k_re, kf]); v_all = np.concatenate([vc, vf])
-    rows = np.arange(t["n_cached_tokens"], t["n_cached_tokens"] + n_rows)
-    m = ob.mask_rows(w.block_lens, w.seq_nblocks, ob.MODE_BLOCK, rows)
-    ob.attention_rows(qf[:n_rows], k_all, v_all, m)
-    t2 = time.perf_counter()
-    return ((t1 - t0) + (t2 - t1) * (Lf / n_rows)) * 1e6
+class OracleSampler:
+    """The fp64 oracle on one layer of the workload, timed on a bounded sample: re-encode of the
+    first `n_blocks` cached blocks and final attend of the first `n_rows` rows of the final block,
+    each scaled linearly to the whole layer (rows and blocks are independent, so a subset is
+    exact for what it covers).  Inputs are generated and widened to fp64 once, outside the timing."""
+
+    def __init__(self, w, layer: int = 0):
+        from oracle import block_attention as ob
+        from paper_2409_15355_b200 import workloads as W
+        self.ob, self.w = ob, w
+        x = W.warm_inputs(w, layer)
+        self.t = ob.segment_tables(w.block_lens, w.seq_nblocks)
+        self.Lf = w.final_lens()[0]
+        f64 = W.bf16_bits_to_f64
+        self.kc, self.vc = f64(x["k_cache"]), f64(x["v_cache"])
+        self.qf, self.kf, self.vf = f64(x["q_f"]), f64(x["k_f"]), f64(x["v_f"])
+        self.k_re = ob.reencode_blocks(self.kc, None, self.t["cache_cu"], self.t["cache_delta"], w.rope_theta)
+
+    def sample(self, n_rows: int, n_blocks: int):
+        """Returns (microseconds per layer, seconds actually spent)."""
+        ob, t, w = self.ob, self.t, self.w
+        nb_all = len(t["cache_delta"])
+        n_blocks = max(1, min(n_blocks, nb_all))
+        n_rows = max(1, min(n_rows, self.Lf))
+        t0 = time.perf_counter()
+        ob.reencode_blocks(self.kc, None, t["cache_cu"][:n_blocks + 1], t["cache_delta"][:n_blocks], w.rope_theta)
+        t1 = time.perf_counter()
+        k_all = np.concatenate([self.k_re, self.kf]); v_all = np.concatenate([self.vc, self.vf])
+        rows = np.arange(t["n_cached_tokens"], t["n_cached_tokens"] + n_rows)
+        m = ob.mask_rows(w.block_lens, w.seq_nblocks, ob.MODE_BLOCK, rows)
+        ob.attention_rows(self.qf[:n_rows], k_all, v_all, m)
+        t2 = time.perf_counter()
+        us = ((t1 - t0) * (nb_all / n_blocks) + (t2 - t1) * (self.Lf / n_rows)) * 1e6
+        return us, t2 - t0
 
 
 def blas_threads():
@@ -155,21 +168,27 @@ def blas_threads():
 
 
 def run_reference(args):
+    """The oracle as it stands, on host cores.  Every step is a bounded sample of one layer,
+    sized from the first warm-up so that the whole run stays within about two minutes."""
     rank, _, world = dist_env()
     if rank != 0:
         return 0
     from paper_2409_15355_b200 import workloads as W
-    w = W.config3(1)
-    rows = 48
+    smp = OracleSampler(W.config3(1))
+    _, sec = smp.sample(4, 1)                          # calibration: 4 rows, 1 block
+    budget = 110.0 / max(1, args.steps + args.warmup)  # seconds per step
+    scale = max(1.0, min(24.0, 0.8 * budget / max(sec, 1e-3)))
+    rows, blocks = int(4 * scale), int(max(1, min(32, scale)))
     for _ in range(args.warmup):
-        oracle_layer_sample(w, 8)
+        smp.sample(rows, blocks)
     vals = []
     t0 = time.perf_counter()
     for _ in range(args.steps):
-        vals.append(oracle_layer_sample(w, rows))
+        vals.append(smp.sample(rows, blocks)[0])
     wall = time.perf_counter() - t0
-    v = statistics.mean(vals)
-    sample = f"per step: one layer, re-encode of all 32000 cached rows + final attend of {rows}/768 final rows (all 32 heads), attend time scaled x{768 / rows:.0f}"
+    v = statistics.mean(vals) if vals else float("nan")
+    sample = (f"per step: one layer; re-encode of {blocks}/32 cached blocks scaled x{32 / blocks:.1f} + final attend "
+              f"of {rows}/768 final rows (all 32 heads) scaled x{768 / rows:.1f}")
     line = {"impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": wall * 1e3 / max(args.steps, 1),
             "higher_is_better": False, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
@@ -289,6 +308,37 @@ def run_ours(args):
     barrier()
     _, e2e_us = aggregate(ev0.elapsed_time(ev1) / e2e_steps, float(L), dev)
 
+    # ---- secondary number: cold block-diagonal prefill (batch 8 x 16384 ragged blocks), one launch
+    prefill = None
+    if rank == 0 and not args.no_prefill:
+        from oracle import block_attention as ob     # closed-form pair count only (no oracle compute)
+        w4 = W.config4()
+        ctx4 = R.Context.for_workload(w4, device=local_rank)
+        seg4, buf4 = ctx4.segment(w4.block_lens, w4.seq_nblocks, B.BA_MODE_BLOCK)
+        g = torch.Generator(device=dev); g.manual_seed(4004)
+        T4 = w4.n_tokens
+        q4 = torch.randn(T4, w4.n_q_heads, w4.head_dim, device=dev, generator=g).bfloat16()
+        k4 = torch.randn(T4, w4.n_kv_heads, w4.head_dim, device=dev, generator=g).bfloat16()
+        v4 = torch.randn(T4, w4.n_kv_heads, w4.head_dim, device=dev, generator=g).bfloat16()
+        o4 = torch.empty_like(q4)
+        for _ in range(3):
+            B.ba_block_prefill(ctx4.ctx, q4, k4, v4, o4, None, seg4, B.BA_MODE_BLOCK, B.BA_OUT_BF16)
+        torch.cuda.synchronize()
+        reps = 10
+        ev0.record(stream)
+        for _ in range(reps):
+            B.ba_block_prefill(ctx4.ctx, q4, k4, v4, o4, None, seg4, B.BA_MODE_BLOCK, B.BA_OUT_BF16)
+        ev1.record(stream)
+        torch.cuda.synchronize()
+        ms4 = ev0.elapsed_time(ev1) / reps
+        pairs4 = ob.allowed_pairs(w4.block_lens, w4.seq_nblocks, ob.MODE_BLOCK)
+        fl4 = 4.0 * w4.head_dim * w4.n_q_heads * pairs4
+        prefill = {"workload": "cfg4: batch 8 x 16384 tokens, ragged blocks U[64,2048], one ba_block_prefill launch",
+                   "ms": ms4, "algorithmic_flops": fl4, "tflops": fl4 / ms4 / 1e9, "allowed_pairs_per_head": pairs4}
+        assert ctx4.device_status() == B.BA_OK
+        ctx4.close()
+        del q4, k4, v4, o4
+
     if rank == 0:
         peaks = load_peaks()
         pairs = Tf * Tc + Tf * (Tf + 1) // 2
@@ -304,7 +354,7 @@ def run_ours(args):
                     "algorithmic_flops_per_launch": flops}
         t0 = time.perf_counter()
         cpu_rows = 96
-        cpu_us = oracle_layer_sample(W.config3(1), cpu_rows)
+        cpu_us, _ = OracleSampler(W.config3(1)).sample(cpu_rows, 32)
         cpu = {"value": cpu_us, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
                "sample": f"one layer: re-encode of 32000 cached rows + final attend of {cpu_rows}/768 final rows, "
                          f"attend scaled x{768 // cpu_rows}; {time.perf_counter() - t0:.1f} s of CPU work"}
@@ -315,6 +365,9 @@ def run_ours(args):
                 "e2e": {"value": e2e_us, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                         "steps": e2e_steps},
                 "gpu_launches": launches, "roofline": roofline, "cpu_baseline": cpu}
+        if prefill is not None:
+            prefill["frac_of_bf16_burst"] = prefill["tflops"] / peaks["bf16_tflops"]
+            line["block_prefill"] = prefill
         if L != 32:
             line["config"]["layers"] = L
         print(json.dumps(line))
@@ -331,6 +384,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--layers", type=int, default=32, help="layers per step (32 = the metric's workload)")
+    ap.add_argument("--no-prefill", action="store_true", help="skip the secondary cold-prefill measurement")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
