@@ -407,6 +407,9 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
             tc_fence_after();
             BA_TR(2, j, t * 4 + 1);
             issue_pv(t, iv, j == 0, 0);
+            // K_(j+1) is needed right after the second half of PV: make sure of it while P is still
+            // being finished, off the critical path
+            if (t == 0 && !last) { BA_TR(3, j, 2); ok = wait_kv(ik); if (!ok) break; BA_TR(3, j, 3); }
             ok = mbar_wait(&ctrl->p_full[t][1], p_uses[t] & 1, abort_flag);
             if (!ok) break;
             tc_fence_after();
@@ -416,7 +419,6 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
             if (last) mma_commit(&ctrl->o_done[t]);
             if (t + 1 == n_qt) mma_commit(&ctrl->kv_empty[iv % kStages]);
             if (!last) {
-              if (t == 0) { BA_TR(3, j, 2); ok = wait_kv(ik); if (!ok) break; tc_fence_after(); BA_TR(3, j, 3); }
               issue_qk(t, ik);
               BA_TR(2, j, t * 4 + 3);
               if (t + 1 == n_qt) {
