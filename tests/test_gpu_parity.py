@@ -232,7 +232,9 @@ def run_prefill(w, mode, out_dtype=B.BA_OUT_F32, rows=None, layer=0):
 PREFILL_CASES = [W.config1(), W.config2(), W.random_ragged(21, 3, 6, 300, 4, 2, 64),
                  W.random_ragged(22, 2, 5, 400, 8, 2, 128), W.random_ragged(23, 4, 4, 140, 4, 4, 128),
                  W.Workload("one_token", 4, 2, 64, 1e4, [1], [1], seed=5),
-                 W.Workload("single_block", 8, 8, 128, 1e4, [333], [1], seed=6)]
+                 W.Workload("single_block", 8, 8, 128, 1e4, [333], [1], seed=6),
+                 # enough work items for the persistent launch (several items per CTA, ragged)
+                 W.random_ragged(24, 14, 8, 300, 8, 2, 128), W.random_ragged(25, 30, 6, 200, 4, 1, 64)]
 
 
 @pytest.mark.parametrize("w", PREFILL_CASES, ids=lambda w: w.name)
@@ -317,7 +319,9 @@ def run_warm(w, mode, out_dtype=B.BA_OUT_F32, layer=0, v_from_pool=True):
 
 WARM_CASES = [W.config1(), W.config2(), W.random_ragged(31, 3, 5, 200, 4, 2, 64),
               W.Workload("no_cache", 4, 2, 64, 1e4, [50, 1, 130], [1, 1, 1], seed=7),
-              W.config5(4, 64, 6, 32)]
+              W.config5(4, 64, 6, 32),
+              # many requests: split keys and the persistent launch together
+              W.random_ragged(32, 40, 4, 150, 8, 2, 128), W.config5(48, 64, 5, 40)]
 
 
 @pytest.mark.parametrize("w", WARM_CASES, ids=lambda w: w.name)
