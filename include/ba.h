@@ -123,6 +123,12 @@ ba_status ba_workspace_bytes(const ba_config *cfg, int32_t max_blocks, int32_t m
  * (tables inconsistent with the lengths given) or BA_ERR_TIMEOUT. */
 ba_status ba_last_device_status(ba_ctx *ctx);
 
+/* Diagnostic (no counterpart in the paper): launches one CTA that waits, with the library's
+ * bounded wait, on a barrier nothing completes.  After about a second the wait gives up and
+ * ba_last_device_status() returns BA_ERR_TIMEOUT; the device stays usable.  Lets a deployment
+ * check the expiry path of the attention kernels without provoking a fault. */
+ba_status ba_selftest_wait_expiry(ba_ctx *ctx, void *stream);
+
 /* Number of this library's kernels launched through `ctx` so far. */
 int64_t ba_launch_count(const ba_ctx *ctx);
 

@@ -23,7 +23,7 @@ BA_OUT_BF16, BA_OUT_F32 = 0, 1
 EXPORTS = [
     "ba_create", "ba_destroy", "ba_status_string", "ba_workspace_bytes", "ba_last_device_status",
     "ba_launch_count", "ba_segments_bytes", "ba_segment", "ba_reencode_k", "ba_block_prefill",
-    "ba_final_attend", "ba_reencode_k_noalloc",
+    "ba_final_attend", "ba_reencode_k_noalloc", "ba_selftest_wait_expiry",
 ]
 BA_NOALLOC_MAX_BLOCKS = 4096
 
@@ -76,6 +76,7 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.ba_segment.argtypes = [vp, vp, vp, i32, i32, i32, C.c_int, vp, sz, C.POINTER(ba_segments), vp]
     lib.ba_reencode_k.argtypes = [vp, vp, vp, i32, vp, vp, vp, i32, i32, vp]
     lib.ba_reencode_k_noalloc.argtypes = [C.POINTER(ba_config), C.c_int, vp, vp, i32, vp, vp, vp, i32, i32, vp, vp]
+    lib.ba_selftest_wait_expiry.argtypes = [vp, vp]
     lib.ba_block_prefill.argtypes = [vp, vp, vp, vp, vp, vp, C.POINTER(ba_segments), C.c_int, C.c_int, vp]
     lib.ba_final_attend.argtypes = [vp, vp, vp, vp, i32, vp, vp, i32, vp, i32, vp, vp,
                                     C.POINTER(ba_segments), C.c_int, C.c_int, vp]
@@ -171,6 +172,10 @@ def ba_reencode_k_noalloc(cfg, device, k_src, src_off, n_src_rows, k_dst, cu, de
                                                 _ptr(k_dst), _ptr(cu), _ptr(delta), n_blocks, n_rows,
                                                 _ptr(status_word), _stream_ptr(stream)),
            "ba_reencode_k_noalloc")
+
+
+def ba_selftest_wait_expiry(ctx, stream=None) -> None:
+    _check(load_library().ba_selftest_wait_expiry(ctx, _stream_ptr(stream)), "ba_selftest_wait_expiry")
 
 
 def ba_block_prefill(ctx, q, k, v, o, lse, seg, mode, out_dtype, stream=None):

@@ -693,6 +693,28 @@ bool make_map(CUtensorMap *m, const void *ptr, int D, int heads, long long rows,
 
 }  // namespace
 
+// Diagnostic: one CTA waits on an mbarrier that nothing ever arrives on, with the same bounded
+// wait the attention kernel uses, so the expiry path (abort flag, status word, clean return) can be
+// checked on a live device without any fault.
+__global__ void ba_wait_expiry_kernel(int32_t *status) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) { mbar_init(&bar, 1); abort_flag = 0; fence_barrier_init(); }
+  __syncthreads();
+  const bool ok = mbar_wait(&bar, 0, &abort_flag);       // never completes: gives up after the poll limit
+  __syncthreads();
+  if (threadIdx.x == 0 && (!ok || abort_flag)) ba_record_status(status, BA_ERR_TIMEOUT);
+}
+
+extern "C" ba_status ba_selftest_wait_expiry(ba_ctx *ctx, void *stream) {
+  if (!ctx) return BA_ERR_INVALID_ARG;
+  BA_CUDA_TRY(cudaSetDevice(ctx->device));
+  ba_wait_expiry_kernel<<<1, 64, 0, (cudaStream_t)stream>>>(ctx->dev_status);
+  BA_CUDA_TRY(cudaGetLastError());
+  ctx->launches += 1;
+  return BA_OK;
+}
+
 // Heads of one KV group packed into a query tile: the largest of 4, 2, 1 that divides the group size.
 int ba_heads_per_tile(const ba_config &c) {
   int G = c.n_q_heads / c.n_kv_heads;

@@ -375,3 +375,14 @@ def test_runs_are_bit_stable():
     a = run_warm(w, B.BA_MODE_BLOCK)[0]
     b = run_warm(w, B.BA_MODE_BLOCK)[0]
     assert (a == b).all()
+
+
+def test_bounded_wait_expires_into_a_status_and_the_device_stays_usable():
+    w = W.config1()
+    c = ctx_for(w)
+    B.ba_selftest_wait_expiry(c.ctx)
+    assert c.device_status() == B.BA_ERR_TIMEOUT       # the wait gave up; nothing hung, nothing faulted
+    assert c.device_status() == B.BA_OK
+    c.close()
+    o, lse, o_ref, lse_ref = run_prefill(w, B.BA_MODE_BLOCK)   # same process, same device: still works
+    check_attention(o, o_ref, lse, lse_ref)
