@@ -53,17 +53,27 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
   return ok != 0;
 }
 
-// Bounded wait.  Gives up after kSpinLimit polls or as soon as another thread of
-// the CTA has raised *abort_flag (a shared-memory word); the caller then leaves
-// its role loop.  A wait that gives up raises the flag itself.
-constexpr uint32_t kSpinLimit = 1u << 22;
+// Bounded wait.  Gives up after about one second (kWaitLimitNs on the global nanosecond timer)
+// or as soon as another thread of the CTA has raised *abort_flag (a shared-memory word); the
+// caller then leaves its role loop.  A wait that gives up raises the flag itself.  Legitimate
+// waits in these kernels last microseconds.
+constexpr unsigned long long kWaitLimitNs = 1000000000ull;
+__device__ __forceinline__ unsigned long long global_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
 __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag) {
-  for (uint32_t it = 0; it < kSpinLimit; ++it) {
+#pragma unroll 1
+  for (int it = 0; it < 64; ++it)
     if (mbar_try_wait(bar, parity)) return true;
-    if (it > 64) {
-      if (*abort_flag) return false;
-      __nanosleep(it > 4096 ? 256 : 32);
-    }
+  const unsigned long long t0 = global_ns();
+#pragma unroll 1
+  for (uint32_t it = 0;; ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if (global_ns() - t0 > kWaitLimitNs) break;
+    __nanosleep(it > 4096 ? 256 : 32);
   }
   *abort_flag = 1;
   return false;
