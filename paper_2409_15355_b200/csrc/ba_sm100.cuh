@@ -58,6 +58,12 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
 // caller then leaves its role loop.  A wait that gives up raises the flag itself.  Legitimate
 // waits in these kernels last microseconds.
 constexpr unsigned long long kWaitLimitNs = 1000000000ull;
+#ifndef BA_FAST_POLLS
+#define BA_FAST_POLLS 64      // polls before the slow path (timer, abort flag, back-off)
+#endif
+#ifndef BA_SLEEP_NS
+#define BA_SLEEP_NS 32        // back-off between polls on the slow path
+#endif
 __device__ __forceinline__ unsigned long long global_ns() {
   unsigned long long t;
   asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
@@ -65,7 +71,7 @@ __device__ __forceinline__ unsigned long long global_ns() {
 }
 __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag) {
 #pragma unroll 1
-  for (int it = 0; it < 64; ++it)
+  for (int it = 0; it < BA_FAST_POLLS; ++it)
     if (mbar_try_wait(bar, parity)) return true;
   const unsigned long long t0 = global_ns();
 #pragma unroll 1
@@ -73,7 +79,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volati
     if (mbar_try_wait(bar, parity)) return true;
     if (*abort_flag) return false;
     if (global_ns() - t0 > kWaitLimitNs) break;
-    __nanosleep(it > 4096 ? 256 : 32);
+    if (BA_SLEEP_NS > 0) __nanosleep(it > 4096 ? 256 : BA_SLEEP_NS);
   }
   *abort_flag = 1;
   return false;
