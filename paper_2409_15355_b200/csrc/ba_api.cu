@@ -91,7 +91,7 @@ ba_status ba_workspace_bytes(const ba_config *cfg, int32_t max_blocks, int32_t m
   size_t split_rows = (size_t)(max_q_rows < 4096 ? max_q_rows : 4096);
   size_t splits = split_rows * cfg->n_q_heads * (cfg->head_dim + 1) * sizeof(float) * 6;
   size_t stage = stage_bytes_for(max_blocks);
-  if (stage < 128 * 1024) stage = 128 * 1024;   // staging + counter areas
+  if (stage < 64 * 1024) stage = 64 * 1024;
   size_t scratch = table > splits ? table : splits;
   *bytes = stage + ba_align_up(scratch, 256) + 256;
   return BA_OK;
@@ -123,11 +123,9 @@ ba_status ba_create(ba_ctx **out, const ba_config *cfg, int device, size_t works
   ctx->dev_status = nullptr;
   if (cudaMalloc(&ctx->dev_status, 256) != cudaSuccess ||
       cudaMemset(ctx->dev_status, 0, 256) != cudaSuccess ||
-      (workspace_bytes && (cudaMalloc(&ctx->workspace, workspace_bytes) != cudaSuccess ||
-                           cudaMemset(ctx->workspace, 0, workspace_bytes) != cudaSuccess))) {
+      (workspace_bytes && cudaMalloc(&ctx->workspace, workspace_bytes) != cudaSuccess)) {
     cudaGetLastError();
     if (ctx->dev_status) cudaFree(ctx->dev_status);
-    if (ctx->workspace) cudaFree(ctx->workspace);
     delete ctx;
     return BA_ERR_CUDA;
   }
@@ -184,8 +182,7 @@ ba_status ba_segment(ba_ctx *ctx, const int32_t *block_lens, const int32_t *seq_
     for (int q = 0; q < batch; ++q) { if (seq_nblocks[q] < 1) return BA_ERR_INVALID_ARG; nb_sum += seq_nblocks[q]; }
     if (sum != n_tokens || nb_sum != n_blocks) return BA_ERR_INVALID_ARG;
     size_t need = (size_t)(n_blocks + batch) * 4;
-    // host arrays are staged in the first 64 KiB of the workspace (at most 16K lengths)
-    if (!ctx->workspace || need > ctx->workspace_bytes || need > ba_counter_offset()) return BA_ERR_WORKSPACE;
+    if (!ctx->workspace || need > ctx->workspace_bytes) return BA_ERR_WORKSPACE;
     int32_t *stage = (int32_t *)ctx->workspace;
     BA_CUDA_TRY(cudaMemcpyAsync(stage, block_lens, (size_t)n_blocks * 4, cudaMemcpyHostToDevice, s));
     BA_CUDA_TRY(cudaMemcpyAsync(stage + n_blocks, seq_nblocks, (size_t)batch * 4, cudaMemcpyHostToDevice, s));

@@ -75,7 +75,6 @@ struct AttnParams {
   const int32_t *v_src_off;       // non-null: values of cached block c start at pool row v_src_off[c]
   int persistent;                 // 1: CTAs draw work from work_counter; 0: CTA b handles entry b only
   int32_t *work_counter;          // device word, zero at launch: next entry of the work list
-  int32_t *split_counters;        // [2 * items] zero between launches: splits of (item, query tile) finished
   ba_segments seg;
 };
 
@@ -103,8 +102,6 @@ struct Ctrl {
   uint64_t work_full[kWorkSlots];  // work entry published by the scheduler (producer thread)
   uint64_t work_empty[kWorkSlots]; // entry read by the MMA thread and the 8 softmax warps
   int work_ring[kWorkSlots];
-  uint64_t epi_bar[2];            // [query tile] write-out of split-KV partial results (128 arrivals)
-  int epi_last[2];                // this CTA holds the last of the item's splits to finish
   int tile_valid[8];              // pool mode: valid key columns of the cached tiles in flight
   uint32_t tmem_base;
   int abort_flag;
@@ -239,7 +236,7 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
     for (int s = 0; s < kStages; ++s) { mbar_init(&ctrl->kv_full[s], 1); mbar_init(&ctrl->kv_empty[s], 1); }
     for (int t = 0; t < 2; ++t) {
       mbar_init(&ctrl->s_full[t], 1); mbar_init(&ctrl->p_full[t][0], 128); mbar_init(&ctrl->p_full[t][1], 128);
-      mbar_init(&ctrl->o_done[t], 1); mbar_init(&ctrl->o_free[t], 128); mbar_init(&ctrl->epi_bar[t], 128);
+      mbar_init(&ctrl->o_done[t], 1); mbar_init(&ctrl->o_free[t], 128);
     }
     for (int k = 0; k < kWorkSlots; ++k) { mbar_init(&ctrl->work_full[k], 1); mbar_init(&ctrl->work_empty[k], 9); }
     ctrl->abort_flag = 0;
@@ -448,7 +445,6 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
     const float sl = p.scale_log2;
     int s_uses = 0;                       // S tiles of this query tile consumed so far
     int o_uses = 0;                       // items in which this query tile was active
-    int epi_uses = 0;                     // phases of this tile's write-out barrier used so far
     int tiles_before = 0;                 // key tiles of all earlier items (the producer counts the same way)
     bool ok = true;
     Work wk;
@@ -620,74 +616,6 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
           if (partial) p.lse_part[((size_t)wk.split * p.n_q_rows + row_tok) * p.Hq + head] = lse_val;
           else if (p.lse) p.lse[(size_t)row_tok * p.Hq + head] = lse_val;
         }
-        if (partial) {
-          // The last of the item's n_splits entries to finish (on whichever SM) merges all partial
-          // results of this query tile: o = sum_s w_s o_s / sum_s w_s, w_s = exp(lse_s - max lse), in
-          // the fixed order s = 0, 1, ..., so the result does not depend on who finishes last.
-          __threadfence();                                   // this thread's partial row is visible device-wide
-          mbar_arrive(&ctrl->epi_bar[t]);
-          ok = mbar_wait(&ctrl->epi_bar[t], epi_uses & 1, abort_flag);
-          ++epi_uses;
-          if (ok) {
-            if (r == 0) {
-              int32_t *cnt = p.split_counters + 2 * (w / p.n_splits) + t;
-              const int seen = atomicAdd(cnt, 1);
-              const int last = seen == p.n_splits - 1;
-              if (last) *cnt = 0;                            // ready for the next launch
-              ctrl->epi_last[t] = last;
-            }
-            mbar_arrive(&ctrl->epi_bar[t]);
-            ok = mbar_wait(&ctrl->epi_bar[t], epi_uses & 1, abort_flag);
-            ++epi_uses;
-          }
-          if (ok && ctrl->epi_last[t] && row_valid) {
-            __threadfence();
-            const size_t rh = (size_t)row_tok * p.Hq + head, n_rh = (size_t)p.n_q_rows * p.Hq;
-            float mx = -INFINITY;
-            for (int sp = 0; sp < p.n_splits; ++sp) mx = fmaxf(mx, __ldcg(p.lse_part + sp * n_rh + rh));
-            float den = 0.f;
-            for (int sp = 0; sp < p.n_splits; ++sp) {
-              const float ls = __ldcg(p.lse_part + sp * n_rh + rh);
-              den += (ls == -INFINITY) ? 0.f : __expf(ls - mx);
-            }
-            const float inv_den = 1.f / den;
-#pragma unroll 1
-            for (int c = 0; c < D / 16; ++c) {
-              float4 acc[4];
-#pragma unroll
-              for (int i = 0; i < 4; ++i) acc[i] = make_float4(0.f, 0.f, 0.f, 0.f);
-              for (int sp = 0; sp < p.n_splits; ++sp) {
-                const float ls = __ldcg(p.lse_part + sp * n_rh + rh);
-                const float wgt = (ls == -INFINITY) ? 0.f : __expf(ls - mx);
-                const float4 *src = reinterpret_cast<const float4 *>(p.o_part + (sp * n_rh + rh) * D + c * 16);
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                  const float4 x = __ldcg(src + i);
-                  acc[i].x = fmaf(wgt, x.x, acc[i].x); acc[i].y = fmaf(wgt, x.y, acc[i].y);
-                  acc[i].z = fmaf(wgt, x.z, acc[i].z); acc[i].w = fmaf(wgt, x.w, acc[i].w);
-                }
-              }
-              if (p.out_f32) {
-                float4 *dst = reinterpret_cast<float4 *>(reinterpret_cast<float *>(p.o) + rh * D + c * 16);
-#pragma unroll
-                for (int i = 0; i < 4; ++i)
-                  dst[i] = make_float4(acc[i].x * inv_den, acc[i].y * inv_den, acc[i].z * inv_den, acc[i].w * inv_den);
-              } else {
-                uint4 *dst = reinterpret_cast<uint4 *>(reinterpret_cast<__nv_bfloat16 *>(p.o) + rh * D + c * 16);
-                uint32_t wd[8];
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                  __nv_bfloat162 a = __floats2bfloat162_rn(acc[i].x * inv_den, acc[i].y * inv_den);
-                  __nv_bfloat162 b = __floats2bfloat162_rn(acc[i].z * inv_den, acc[i].w * inv_den);
-                  wd[2 * i] = *reinterpret_cast<uint32_t *>(&a); wd[2 * i + 1] = *reinterpret_cast<uint32_t *>(&b);
-                }
-                dst[0] = make_uint4(wd[0], wd[1], wd[2], wd[3]);
-                dst[1] = make_uint4(wd[4], wd[5], wd[6], wd[7]);
-              }
-            }
-            if (p.lse) p.lse[rh] = mx + logf(den);
-          }
-        }
       }
       }
       tiles_before += n_tiles;
@@ -698,6 +626,39 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
   __syncthreads();
   if (tid == 0 && ctrl->abort_flag) ba_record_status(p.status, BA_ERR_TIMEOUT);
   if (warp == 9) tmem_dealloc(tmem, 512);
+}
+
+// Merge of split-KV partial results: o = sum_s w_s o_s / sum_s w_s with w_s = exp(lse_s - max lse).
+// One thread per 4 output columns; the order of the sum is fixed, so results are run-to-run stable.
+template <int D>
+__global__ void __launch_bounds__(256)
+ba_combine_splits_kernel(const float *__restrict__ o_part, const float *__restrict__ lse_part, void *o, float *lse,
+                         int n_rows_heads, int n_splits, int out_f32) {
+  const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+  constexpr int kVec = D / 4;
+  const int rh = idx / kVec, v = idx - rh * kVec;
+  if (rh >= n_rows_heads) return;
+  float mx = -INFINITY;
+  for (int s = 0; s < n_splits; ++s) mx = fmaxf(mx, __ldg(lse_part + (size_t)s * n_rows_heads + rh));
+  float den = 0.f;
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+  for (int s = 0; s < n_splits; ++s) {
+    const float ls = __ldg(lse_part + (size_t)s * n_rows_heads + rh);
+    const float w = (ls == -INFINITY) ? 0.f : __expf(ls - mx);
+    const float4 x = __ldg(reinterpret_cast<const float4 *>(o_part + ((size_t)s * n_rows_heads + rh) * D) + v);
+    den += w;
+    acc.x = fmaf(w, x.x, acc.x); acc.y = fmaf(w, x.y, acc.y); acc.z = fmaf(w, x.z, acc.z); acc.w = fmaf(w, x.w, acc.w);
+  }
+  const float inv = 1.f / den;
+  acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
+  if (out_f32) {
+    reinterpret_cast<float4 *>(reinterpret_cast<float *>(o) + (size_t)rh * D)[v] = acc;
+  } else {
+    __nv_bfloat162 a = __floats2bfloat162_rn(acc.x, acc.y), b = __floats2bfloat162_rn(acc.z, acc.w);
+    uint2 w2 = make_uint2(*reinterpret_cast<uint32_t *>(&a), *reinterpret_cast<uint32_t *>(&b));
+    reinterpret_cast<uint2 *>(reinterpret_cast<__nv_bfloat16 *>(o) + (size_t)rh * D)[v] = w2;
+  }
+  if (lse && v == 0) lse[rh] = mx + logf(den);
 }
 
 // ------------------------------------------------------------------ host side
@@ -807,18 +768,15 @@ ba_status ba_attend_sm100_launch(ba_ctx *ctx, const ba_attend_args &a, const ba_
   p.persistent = work_upper > 2LL * ctx->sm_count;
   p.work_counter = nullptr;
   if (p.persistent) {
-    // the counter lives in the counter area of the workspace and is cleared per launch
+    // the counter lives in the last 256 bytes below the scratch area and is cleared per launch
     if (!ctx->workspace || ctx->workspace_bytes < ba_scratch_offset(ctx)) return BA_ERR_WORKSPACE;
-    p.work_counter = reinterpret_cast<int32_t *>(reinterpret_cast<char *>(ctx->workspace) + ba_counter_offset());
+    p.work_counter = reinterpret_cast<int32_t *>(reinterpret_cast<char *>(ctx->workspace) + ba_scratch_offset(ctx) - 256);
     BA_CUDA_TRY(cudaMemsetAsync(p.work_counter, 0, sizeof(int32_t), stream));
   }
-  p.o_part = nullptr; p.lse_part = nullptr; p.split_counters = nullptr;
+  p.o_part = nullptr; p.lse_part = nullptr;
   if (n_splits > 1) {
     p.o_part = reinterpret_cast<float *>(reinterpret_cast<char *>(ctx->workspace) + ba_scratch_offset(ctx));
     p.lse_part = p.o_part + (size_t)n_splits * a.n_q_rows * Hq * D;
-    // per (item, query tile) counters of finished splits: zero at ba_create, reset by their last user
-    p.split_counters = reinterpret_cast<int32_t *>(reinterpret_cast<char *>(ctx->workspace) + ba_counter_offset() + 256);
-    if (2 * items * sizeof(int32_t) > ba_scratch_offset(ctx) - ba_counter_offset() - 256) n_splits = p.n_splits = 1;
   }
 
   CUtensorMap tq, tk, tv, tkc, tvc;
@@ -845,5 +803,16 @@ ba_status ba_attend_sm100_launch(ba_ctx *ctx, const ba_attend_args &a, const ba_
   }
   BA_CUDA_TRY(cudaGetLastError());
   ctx->launches += 1;
+  if (n_splits > 1) {
+    const int n_rh = a.n_q_rows * Hq;
+    const long long threads = (long long)n_rh * (D / 4);
+    const unsigned cgrid = (unsigned)((threads + 255) / 256);
+    if (D == 128)
+      ba_combine_splits_kernel<128><<<cgrid, 256, 0, stream>>>(p.o_part, p.lse_part, a.o, a.lse, n_rh, n_splits, a.out_f32);
+    else
+      ba_combine_splits_kernel<64><<<cgrid, 256, 0, stream>>>(p.o_part, p.lse_part, a.o, a.lse, n_rh, n_splits, a.out_f32);
+    BA_CUDA_TRY(cudaGetLastError());
+    ctx->launches += 1;
+  }
   return BA_OK;
 }

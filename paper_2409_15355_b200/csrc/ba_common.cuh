@@ -31,15 +31,11 @@ struct ba_ctx {
 
 static inline size_t ba_align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
-// Workspace layout (zero-filled at ba_create):
-//   [0, 64 KiB)        staging of host-side length arrays (ba_segment)
-//   [64 KiB, 128 KiB)  counters of the attention kernel: work-list position (first 256 bytes,
-//                      cleared per launch) and split-KV completion counters (reset by their last user)
-//   [128 KiB, ...)     per-call scratch: split-KV partial results (attention) or, at the very end
-//                      of the workspace, the angle table (re-encode)
-// Calls on one context are stream-ordered, so the regions may be reused from call to call.
-static inline size_t ba_counter_offset() { return 64 * 1024; }
-static inline size_t ba_scratch_offset(const ba_ctx *) { return 128 * 1024; }
+// Workspace layout: [0, 64 KiB) staging of host-side length arrays (ba_segment);
+// [64 KiB, ...) per-call scratch: split-KV partial results (attention) or, at the very end
+// of the workspace, the angle table (re-encode).  Calls on one context are stream-ordered,
+// so the regions may be reused from call to call.
+static inline size_t ba_scratch_offset(const ba_ctx *) { return 64 * 1024; }
 
 // Records the first device-side problem; later ones are dropped.
 __device__ __forceinline__ void ba_record_status(int32_t *status, int32_t code) {

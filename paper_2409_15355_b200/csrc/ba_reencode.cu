@@ -55,11 +55,8 @@ __device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w 
 // HALF layout: the vector at column c (< d/2) pairs with the vector at c + d/2,
 // a thread moves both.
 // A thread owns one vector column (ADJACENT) or one column pair (HALF) of kRows rows.
-#ifndef BA_REENCODE_MINB
-#define BA_REENCODE_MINB 1
-#endif
 template <int kLayout, int kRows>
-__global__ void __launch_bounds__(512, BA_REENCODE_MINB)
+__global__ void __launch_bounds__(512)
 ba_reencode_kernel(const uint4 *src, uint4 *dst,  // may alias (in place): no __restrict__
                    const int32_t *__restrict__ src_off, int n_src_rows,
                    const int32_t *__restrict__ cu, const int32_t *__restrict__ delta, int n_blocks,
