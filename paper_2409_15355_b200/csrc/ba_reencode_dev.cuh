@@ -1,0 +1,152 @@
+// Device-side core of the position re-encoding (Section 2.3, Eq. 1-3 collapsed into one rotation
+// by the block's position delta), shared by the stand-alone kernel and by the attention kernel,
+// whose two spare warps can carry a re-encoding job along in the background.
+#pragma once
+
+#include "ba_common.cuh"
+
+// One re-encoding job: block c of `n_blocks` is read from row src_off[c] (or cu[c]) of `src`,
+// rotated by delta[c] with the (cos, sin) pairs in `table`, and written to rows cu[c].. of `dst`.
+struct ba_reencode_job {
+  const uint4 *src;
+  uint4 *dst;
+  const int32_t *src_off;
+  const int32_t *cu;
+  const int32_t *delta;
+  const float2 *table;      // [n_blocks][head_dim / 2] (cos, sin)
+  int32_t n_src_rows, n_blocks, n_rows;
+  int32_t head_dim, row_vecs /* uint4 per row */, layout;
+};
+
+__device__ __forceinline__ int upper_bound_i32(const int32_t *a, int n, int x) {
+  int lo = 0, hi = n;
+  while (lo < hi) {
+    int mid = (lo + hi) >> 1;
+    if (__ldg(a + mid) <= x) lo = mid + 1; else hi = mid;
+  }
+  return lo;
+}
+
+__device__ __forceinline__ void rot2(float x, float y, float2 cs, float &xo, float &yo) {
+  xo = fmaf(x, cs.x, -y * cs.y);
+  yo = fmaf(x, cs.y, y * cs.x);
+}
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t *>(&v);
+}
+
+__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+
+// ADJACENT layout: a 16-byte vector holds rotary pairs 4v..4v+3 of one head.
+// HALF layout: the vector at column c (< d/2) pairs with the vector at c + d/2, a thread moves both.
+// The calling thread owns unit `u` (one vector column, or one column pair) and handles rows
+// row0, row0 + row_step, ... (kRows of them), all loads first.
+template <int kLayout, int kRows>
+__device__ __forceinline__ void ba_reencode_rows(const ba_reencode_job &job, int u, int row0, int row_step,
+                                                 int32_t *status) {
+  const uint4 *src = job.src;
+  uint4 *dst = job.dst;
+  const int32_t *src_off = job.src_off, *cu = job.cu, *delta = job.delta;
+  const float2 *table = job.table;
+  const int n_src_rows = job.n_src_rows, n_blocks = job.n_blocks, row_vecs = job.row_vecs;
+  const int half_dim = job.head_dim >> 1;
+  const int head_vecs = job.head_dim >> 3;                    // uint4 per head
+  const int total_rows = min(job.n_rows, __ldg(cu + n_blocks));
+  // column of this thread's vector(s) inside the row, and its first rotary pair
+  int vec_x, vec_y, m0;
+  if (kLayout == BA_ROPE_ADJACENT) {
+    vec_x = u; vec_y = u;
+    m0 = (u % head_vecs) * 4;
+  } else {
+    int hv = head_vecs >> 1;                                  // vectors per half head
+    int head = u / hv, v = u - head * hv;
+    vec_x = head * head_vecs + v;
+    vec_y = vec_x + hv;
+    m0 = v * 8;
+  }
+
+  uint4 x[kRows], y[kRows];
+  int blk[kRows];
+  bool live[kRows];
+  // Rows of a thread are close together, so they usually share a block: the block of a row is
+  // looked up again only when the row leaves [c_begin, c_end).
+  int c = 0, c_begin = 0, c_end = -1;
+  long long shift = 0;                                        // source row = row + shift
+#pragma unroll
+  for (int i = 0; i < kRows; ++i) {
+    const int r = row0 + i * row_step;
+    live[i] = r < total_rows;
+    blk[i] = 0;
+    if (live[i]) {
+      if (r < c_begin || r >= c_end) {
+        c = upper_bound_i32(cu, n_blocks + 1, r) - 1;
+        c = min(max(c, 0), n_blocks - 1);
+        c_begin = __ldg(cu + c);
+        c_end = __ldg(cu + c + 1);
+        shift = src_off ? (long long)__ldg(src_off + c) - c_begin : 0;
+      }
+      blk[i] = c;
+      const long long sr = r + shift;
+      if (sr < 0 || sr >= n_src_rows) {
+        ba_record_status(status, BA_ERR_INVALID_ARG);
+        live[i] = false;
+      } else {
+        const uint4 *p = src + sr * row_vecs;
+        x[i] = p[vec_x];
+        if (kLayout == BA_ROPE_HALF) y[i] = p[vec_y];
+      }
+    }
+  }
+  // (cos, sin) of this thread's rotary pairs, reloaded only when the block changes
+  int t_blk = -1, t_delta = 0;
+  float4 tcs[4];
+#pragma unroll
+  for (int i = 0; i < kRows; ++i) {
+    if (!live[i]) continue;
+    int r = row0 + i * row_step;
+    uint4 *q = dst + (long long)r * row_vecs;
+    if (blk[i] != t_blk) {
+      t_blk = blk[i];
+      t_delta = __ldg(delta + t_blk);
+      const float4 *t4 = reinterpret_cast<const float4 *>(table + t_blk * half_dim + m0);
+      tcs[0] = __ldg(t4); tcs[1] = __ldg(t4 + 1);
+      if (kLayout == BA_ROPE_HALF) { tcs[2] = __ldg(t4 + 2); tcs[3] = __ldg(t4 + 3); }
+    }
+    if (t_delta == 0) {                          // identity: copy bit-exactly
+      q[vec_x] = x[i];
+      if (kLayout == BA_ROPE_HALF) q[vec_y] = y[i];
+      continue;
+    }
+    if (kLayout == BA_ROPE_ADJACENT) {
+      const float4 a = tcs[0], b = tcs[1];                      // two (cos,sin) pairs per float4
+      uint32_t w[4] = {x[i].x, x[i].y, x[i].z, x[i].w};
+      float2 cs[4] = {make_float2(a.x, a.y), make_float2(a.z, a.w), make_float2(b.x, b.y), make_float2(b.z, b.w)};
+      uint32_t o[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        float xo, yo;
+        rot2(bf16_lo(w[j]), bf16_hi(w[j]), cs[j], xo, yo);
+        o[j] = pack_bf16x2(xo, yo);
+      }
+      q[vec_x] = make_uint4(o[0], o[1], o[2], o[3]);
+    } else {
+      uint32_t wx[4] = {x[i].x, x[i].y, x[i].z, x[i].w};
+      uint32_t wy[4] = {y[i].x, y[i].y, y[i].z, y[i].w};
+      uint32_t ox[4], oy[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const float4 cs = tcs[j];                             // pairs m0+2j, m0+2j+1
+        float x0, y0, x1, y1;
+        rot2(bf16_lo(wx[j]), bf16_lo(wy[j]), make_float2(cs.x, cs.y), x0, y0);
+        rot2(bf16_hi(wx[j]), bf16_hi(wy[j]), make_float2(cs.z, cs.w), x1, y1);
+        ox[j] = pack_bf16x2(x0, x1);
+        oy[j] = pack_bf16x2(y0, y1);
+      }
+      q[vec_x] = make_uint4(ox[0], ox[1], ox[2], ox[3]);
+      q[vec_y] = make_uint4(oy[0], oy[1], oy[2], oy[3]);
+    }
+  }
+}
