@@ -175,6 +175,24 @@ ba_status ba_reencode_k(ba_ctx *ctx, const void *k_src, const int32_t *src_off, 
                         int32_t n_rows, void *stream);
 
 /*
+ * Section 2.5, across layers: the cached keys of every layer are known the moment the cache is
+ * hit, so the re-encoding of layer l+1 need not wait for the attention of layer l.
+ * ba_reencode_k_deferred queues the job described by its arguments (the same as ba_reencode_k):
+ * the angle table is computed at once on `stream`, the rotation itself is carried out by otherwise
+ * idle warps of the NEXT ba_final_attend / ba_block_prefill launched through this context, in the
+ * background of that kernel, and is complete when that kernel completes (stream order, as usual).
+ * The job must not touch the tensors that attention call reads or writes.  One job can be queued
+ * per context: queuing another, ba_flush() or ba_destroy() run a still-queued job as an ordinary
+ * stand-alone launch.  Results are bit-identical to ba_reencode_k.  The queued job's arguments
+ * (device pointers) must stay valid until it has run.
+ */
+ba_status ba_reencode_k_deferred(ba_ctx *ctx, const void *k_src, const int32_t *src_off, int32_t n_src_rows,
+                                 void *k_dst, const int32_t *cu, const int32_t *delta, int32_t n_blocks,
+                                 int32_t n_rows, void *stream);
+/* Runs a queued re-encoding job now, on `stream`; does nothing when none is queued. */
+ba_status ba_flush(ba_ctx *ctx, void *stream);
+
+/*
  * ba_reencode_k_noalloc -- the same re-encoding as ba_reencode_k for callers that
  * must not allocate device memory.  (The paper has no counterpart to this entry
  * point; it exists for integration reasons only.)

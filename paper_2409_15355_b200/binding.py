@@ -23,7 +23,7 @@ BA_OUT_BF16, BA_OUT_F32 = 0, 1
 EXPORTS = [
     "ba_create", "ba_destroy", "ba_status_string", "ba_workspace_bytes", "ba_last_device_status",
     "ba_launch_count", "ba_segments_bytes", "ba_segment", "ba_reencode_k", "ba_block_prefill",
-    "ba_final_attend", "ba_reencode_k_noalloc", "ba_selftest_wait_expiry",
+    "ba_final_attend", "ba_reencode_k_noalloc", "ba_selftest_wait_expiry", "ba_reencode_k_deferred", "ba_flush",
 ]
 BA_NOALLOC_MAX_BLOCKS = 4096
 
@@ -77,6 +77,8 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.ba_reencode_k.argtypes = [vp, vp, vp, i32, vp, vp, vp, i32, i32, vp]
     lib.ba_reencode_k_noalloc.argtypes = [C.POINTER(ba_config), C.c_int, vp, vp, i32, vp, vp, vp, i32, i32, vp, vp]
     lib.ba_selftest_wait_expiry.argtypes = [vp, vp]
+    lib.ba_reencode_k_deferred.argtypes = [vp, vp, vp, i32, vp, vp, vp, i32, i32, vp]
+    lib.ba_flush.argtypes = [vp, vp]
     lib.ba_block_prefill.argtypes = [vp, vp, vp, vp, vp, vp, C.POINTER(ba_segments), C.c_int, C.c_int, vp]
     lib.ba_final_attend.argtypes = [vp, vp, vp, vp, i32, vp, vp, i32, vp, i32, vp, vp,
                                     C.POINTER(ba_segments), C.c_int, C.c_int, vp]
@@ -163,6 +165,17 @@ def ba_reencode_k(ctx, k_src, src_off, n_src_rows, k_dst, cu, delta, n_blocks, n
     _check(load_library().ba_reencode_k(ctx, _ptr(k_src), _ptr(src_off), n_src_rows, _ptr(k_dst),
                                         _ptr(cu), _ptr(delta), n_blocks, n_rows, _stream_ptr(stream)),
            "ba_reencode_k")
+
+
+def ba_reencode_k_deferred(ctx, k_src, src_off, n_src_rows, k_dst, cu, delta, n_blocks, n_rows, stream=None):
+    """Queues the re-encoding; it runs in the background of the next attention call on this context."""
+    _check(load_library().ba_reencode_k_deferred(ctx, _ptr(k_src), _ptr(src_off), n_src_rows, _ptr(k_dst),
+                                                 _ptr(cu), _ptr(delta), n_blocks, n_rows, _stream_ptr(stream)),
+           "ba_reencode_k_deferred")
+
+
+def ba_flush(ctx, stream=None) -> None:
+    _check(load_library().ba_flush(ctx, _stream_ptr(stream)), "ba_flush")
 
 
 def ba_reencode_k_noalloc(cfg, device, k_src, src_off, n_src_rows, k_dst, cu, delta, n_blocks, n_rows,

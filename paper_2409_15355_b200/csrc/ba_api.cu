@@ -119,6 +119,9 @@ ba_status ba_create(ba_ctx **out, const ba_config *cfg, int device, size_t works
   ctx->scale = cfg->softmax_scale > 0.f ? cfg->softmax_scale : 1.0f / sqrtf((float)cfg->head_dim);
   ctx->workspace_bytes = workspace_bytes;
   ctx->launches = 0;
+  ctx->has_pending = 0;
+  ctx->pending_table_bytes = 0;
+  ctx->pending_stream = nullptr;
   ctx->workspace = nullptr;
   ctx->dev_status = nullptr;
   if (cudaMalloc(&ctx->dev_status, 256) != cudaSuccess ||
@@ -136,6 +139,7 @@ ba_status ba_create(ba_ctx **out, const ba_config *cfg, int device, size_t works
 ba_status ba_destroy(ba_ctx *ctx) {
   if (!ctx) return BA_ERR_INVALID_ARG;
   cudaSetDevice(ctx->device);
+  if (ctx->has_pending) ba_flush_pending(ctx, ctx->pending_stream);   // a queued job is not dropped
   cudaDeviceSynchronize();
   if (ctx->workspace) cudaFree(ctx->workspace);
   if (ctx->dev_status) cudaFree(ctx->dev_status);
@@ -208,22 +212,68 @@ ba_status ba_segment(ba_ctx *ctx, const int32_t *block_lens, const int32_t *seq_
   return ba_segment_launch(ctx, d_lens, d_nb, batch, n_blocks, n_tokens, mode, out, s);
 }
 
-ba_status ba_reencode_k(ba_ctx *ctx, const void *k_src, const int32_t *src_off, int32_t n_src_rows,
-                        void *k_dst, const int32_t *cu, const int32_t *delta, int32_t n_blocks,
-                        int32_t n_rows, void *stream) {
+static ba_status check_reencode_args(ba_ctx *ctx, const void *k_src, const int32_t *src_off, int32_t n_src_rows,
+                                     void *k_dst, const int32_t *cu, const int32_t *delta, int32_t n_blocks,
+                                     int32_t n_rows, bool *nothing_to_do) {
+  *nothing_to_do = false;
   if (!ctx) return BA_ERR_INVALID_ARG;
   if (n_blocks < 0 || n_rows < 0 || n_src_rows < 0) return BA_ERR_INVALID_ARG;
-  if (n_blocks == 0 || n_rows == 0) return BA_OK;            // nothing cached: nothing to do
+  if (n_blocks == 0 || n_rows == 0) { *nothing_to_do = true; return BA_OK; }   // nothing cached
   if (!k_src || !k_dst || !cu || !delta) return BA_ERR_INVALID_ARG;
   if (!aligned16(k_src) || !aligned16(k_dst)) return BA_ERR_INVALID_ARG;
   if (k_src == k_dst && src_off) return BA_ERR_INVALID_ARG;  // a gather cannot run in place
+  return BA_OK;
+}
+
+// The angle table of a call sits at the end of the workspace, below the table of a queued job.
+static ba_status place_table(ba_ctx *ctx, int32_t n_blocks, float2 **table, size_t *bytes) {
+  const size_t need = ba_align_up((size_t)n_blocks * ctx->cfg.head_dim * 4, 256);  // n_blocks * d/2 * sizeof(float2)
+  if (!ctx->workspace || ba_scratch_offset(ctx) + need + ctx->pending_table_bytes > ctx->workspace_bytes)
+    return BA_ERR_WORKSPACE;
+  *table = (float2 *)((char *)ctx->workspace + (ctx->workspace_bytes - ctx->pending_table_bytes - need) / 256 * 256);
+  *bytes = need;
+  return BA_OK;
+}
+
+ba_status ba_reencode_k(ba_ctx *ctx, const void *k_src, const int32_t *src_off, int32_t n_src_rows,
+                        void *k_dst, const int32_t *cu, const int32_t *delta, int32_t n_blocks,
+                        int32_t n_rows, void *stream) {
+  bool nothing;
+  ba_status st = check_reencode_args(ctx, k_src, src_off, n_src_rows, k_dst, cu, delta, n_blocks, n_rows, &nothing);
+  if (st != BA_OK || nothing) return st;
   BA_CUDA_TRY(cudaSetDevice(ctx->device));
-  // scratch: the angle table at the end of the workspace (the staging area is at its start)
-  size_t need = ba_align_up((size_t)n_blocks * ctx->cfg.head_dim * 4, 256);  // n_blocks * d/2 * sizeof(float2)
-  if (!ctx->workspace || ba_scratch_offset(ctx) + need > ctx->workspace_bytes) return BA_ERR_WORKSPACE;
-  float2 *table = (float2 *)((char *)ctx->workspace + (ctx->workspace_bytes - need) / 256 * 256);
+  float2 *table; size_t bytes;
+  st = place_table(ctx, n_blocks, &table, &bytes);
+  if (st != BA_OK) return st;
   return ba_reencode_launch(ctx, k_src, src_off, n_src_rows, k_dst, cu, delta, n_blocks, n_rows, table,
                             (cudaStream_t)stream);
+}
+
+ba_status ba_reencode_k_deferred(ba_ctx *ctx, const void *k_src, const int32_t *src_off, int32_t n_src_rows,
+                                 void *k_dst, const int32_t *cu, const int32_t *delta, int32_t n_blocks,
+                                 int32_t n_rows, void *stream) {
+  bool nothing;
+  ba_status st = check_reencode_args(ctx, k_src, src_off, n_src_rows, k_dst, cu, delta, n_blocks, n_rows, &nothing);
+  if (st != BA_OK || nothing) return st;
+  BA_CUDA_TRY(cudaSetDevice(ctx->device));
+  st = ba_flush_pending(ctx, (cudaStream_t)stream);          // one job may be queued at a time
+  if (st != BA_OK) return st;
+  float2 *table; size_t bytes;
+  st = place_table(ctx, n_blocks, &table, &bytes);
+  if (st != BA_OK) return st;
+  st = ba_reencode_table_launch(ctx, delta, n_blocks, table, (cudaStream_t)stream);
+  if (st != BA_OK) return st;
+  ctx->pending = ba_make_reencode_job(ctx, k_src, src_off, n_src_rows, k_dst, cu, delta, n_blocks, n_rows, table);
+  ctx->has_pending = 1;
+  ctx->pending_table_bytes = bytes;
+  ctx->pending_stream = (cudaStream_t)stream;
+  return BA_OK;
+}
+
+ba_status ba_flush(ba_ctx *ctx, void *stream) {
+  if (!ctx) return BA_ERR_INVALID_ARG;
+  BA_CUDA_TRY(cudaSetDevice(ctx->device));
+  return ba_flush_pending(ctx, (cudaStream_t)stream);
 }
 
 static ba_status check_attend_common(ba_ctx *ctx, const void *q, const void *k, const void *v, void *o,
@@ -280,6 +330,6 @@ ba_status ba_final_attend(ba_ctx *ctx, const void *q_f, const void *k_f, const v
 
 ba_status ba_attend_launch(ba_ctx *ctx, const ba_attend_args &a, const ba_segments *seg,
                            cudaStream_t stream) {
-  if (a.n_q_rows == 0) return BA_OK;
+  if (a.n_q_rows == 0) return ba_flush_pending(ctx, stream);   // no attention launch to ride along with
   return ba_attend_sm100_launch(ctx, a, seg, stream);
 }

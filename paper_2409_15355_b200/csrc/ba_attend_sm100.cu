@@ -24,6 +24,7 @@
 
 #include "ba_common.cuh"
 #include "ba_sm100.cuh"
+#include "ba_reencode_dev.cuh"
 
 using namespace sm100;
 
@@ -75,6 +76,7 @@ struct AttnParams {
   const int32_t *v_src_off;       // non-null: values of cached block c start at pool row v_src_off[c]
   int persistent;                 // 1: CTAs draw work from work_counter; 0: CTA b handles entry b only
   int32_t *work_counter;          // device word, zero at launch: next entry of the work list
+  ba_reencode_job bg;             // bg.n_rows > 0: a re-encoding job the two spare warps carry out meanwhile
   ba_segments seg;
 };
 
@@ -228,7 +230,8 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
   uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   Ctrl *ctrl = reinterpret_cast<Ctrl *>(smem + L::kCtrl);
 
-  if (__ldg(p.seg.totals + 7) != BA_TABLES_VALID) return;
+  // inconsistent tables: no attention work is taken, a background job still runs
+  const bool tables_ok = __ldg(p.seg.totals + 7) == BA_TABLES_VALID;
   const int tid = threadIdx.x, warp = tid >> 5;
 
   if (tid == 0) {
@@ -272,7 +275,7 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
         if (!ok) break;
         // persistent launch: next entry of the global list; one-item launch: this CTA's own entry, then stop
         const int w = p.persistent ? atomicAdd(p.work_counter, 1) : (n_work == 0 ? (int)blockIdx.x : 0x7fffffff);
-        const bool more = next_work(p, w, wk);
+        const bool more = tables_ok && next_work(p, w, wk);
         ctrl->work_ring[slot] = more ? w : -1;
         mbar_arrive(&ctrl->work_full[slot]);
         ++n_work;
@@ -433,7 +436,26 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
       }
     }
   } else if (warp >= 10) {
+    // ------------------------------------------------------------ spare warps: background re-encoding
     asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(BA_SVC_REGS));
+    if (p.bg.n_rows > 0) {
+      // The 64 spare threads of every CTA together act as one wide row-walking engine: thread g
+      // owns one vector column and every rows_per_pass-th row (the host made sure that
+      // gridDim.x * 64 threads cover at least one row).
+      constexpr int kBgRows = 2;
+      const bool adjacent = p.bg.layout == BA_ROPE_ADJACENT;
+      const int upr = adjacent ? p.bg.row_vecs : (p.bg.row_vecs >> 1);
+      const int g = blockIdx.x * 64 + (tid - 320);
+      const int rows_per_pass = (int)(gridDim.x * 64) / upr;
+      if (g < rows_per_pass * upr) {
+        const int u = g % upr;
+        const int total_rows = min(p.bg.n_rows, __ldg(p.bg.cu + p.bg.n_blocks));
+        for (int row0 = g / upr; row0 < total_rows; row0 += rows_per_pass * kBgRows) {
+          if (adjacent) ba_reencode_rows<BA_ROPE_ADJACENT, kBgRows>(p.bg, u, row0, rows_per_pass, p.status);
+          else ba_reencode_rows<BA_ROPE_HALF, kBgRows>(p.bg, u, row0, rows_per_pass, p.status);
+        }
+      }
+    }
   } else {
     // ------------------------------------------------------------ softmax, one thread per tile row
     asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(BA_SMX_REGS));
@@ -790,6 +812,20 @@ ba_status ba_attend_sm100_launch(ba_ctx *ctx, const ba_attend_args &a, const ba_
     tkc = tk; tvc = tv;
   }
   dim3 grid((unsigned)(p.persistent ? ctx->sm_count : work_upper));
+  // a queued re-encoding job rides along if the spare warps of this grid span at least one row;
+  // otherwise it is run on its own first
+  p.bg.n_rows = 0;
+  if (ctx->has_pending) {
+    const int upr = ctx->pending.layout == BA_ROPE_ADJACENT ? ctx->pending.row_vecs : ctx->pending.row_vecs / 2;
+    if ((long long)grid.x * 64 >= upr) {
+      p.bg = ctx->pending;
+      ctx->has_pending = 0;
+      ctx->pending_table_bytes = 0;
+    } else {
+      ba_status fs = ba_flush_pending(ctx, stream);
+      if (fs != BA_OK) return fs;
+    }
+  }
   // ask for more than half of the SM's shared memory so that two CTAs never share an SM
   // (each CTA allocates all 512 tensor-memory columns)
   if (D == 128) {

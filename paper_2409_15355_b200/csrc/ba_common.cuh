@@ -17,6 +17,19 @@
 // Value of ba_segments::totals[7] once ba_segment's kernel has found the lengths consistent.
 #define BA_TABLES_VALID 0x600D
 
+// One re-encoding job: block c of `n_blocks` is read from row src_off[c] (or cu[c]) of `src`,
+// rotated by delta[c] with the (cos, sin) pairs in `table`, and written to rows cu[c].. of `dst`.
+struct ba_reencode_job {
+  const uint4 *src;
+  uint4 *dst;
+  const int32_t *src_off;
+  const int32_t *cu;
+  const int32_t *delta;
+  const float2 *table;      // [n_blocks][head_dim / 2] (cos, sin)
+  int32_t n_src_rows, n_blocks, n_rows;
+  int32_t head_dim, row_vecs /* uint4 per row */, layout;
+};
+
 // Context: configuration, workspace and the device status word.
 struct ba_ctx {
   ba_config cfg;
@@ -27,6 +40,12 @@ struct ba_ctx {
   size_t workspace_bytes;
   int32_t *dev_status;      // device word: first non-zero ba_status recorded by a kernel
   int64_t launches;
+  // a re-encoding job queued by ba_reencode_k_deferred: carried along by the next attention
+  // launch (or run by ba_flush); its angle table sits at the very end of the workspace
+  ba_reencode_job pending;
+  int has_pending;
+  size_t pending_table_bytes;
+  cudaStream_t pending_stream;
 };
 
 static inline size_t ba_align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -47,10 +66,19 @@ ba_status ba_segment_launch(ba_ctx *ctx, const int32_t *d_block_lens, const int3
                             int32_t batch, int32_t n_blocks, int32_t n_tokens, int mode,
                             const ba_segments *seg, cudaStream_t stream);
 
+// Re-encoding in two steps: angle table, then the rotation itself.
+ba_status ba_reencode_table_launch(ba_ctx *ctx, const int32_t *delta, int32_t n_blocks, float2 *table,
+                                   cudaStream_t stream);
+ba_status ba_reencode_main_launch(ba_ctx *ctx, const ba_reencode_job &job, cudaStream_t stream);
 ba_status ba_reencode_launch(ba_ctx *ctx, const void *k_src, const int32_t *src_off,
                              int32_t n_src_rows, void *k_dst, const int32_t *cu,
                              const int32_t *delta, int32_t n_blocks, int32_t n_rows, float2 *table,
                              cudaStream_t stream);
+ba_reencode_job ba_make_reencode_job(const ba_ctx *ctx, const void *k_src, const int32_t *src_off,
+                                     int32_t n_src_rows, void *k_dst, const int32_t *cu, const int32_t *delta,
+                                     int32_t n_blocks, int32_t n_rows, const float2 *table);
+// Runs a pending deferred job as a stand-alone launch (no-op when nothing is pending).
+ba_status ba_flush_pending(ba_ctx *ctx, cudaStream_t stream);
 
 struct ba_attend_args {
   // queries / outputs: rows of the q packing (prompt packing for prefill, final packing for final attend)

@@ -45,40 +45,64 @@ ba_reencode_kernel(const ba_reencode_job job, int32_t *status) {
 
 }  // namespace
 
-ba_status ba_reencode_launch(ba_ctx *ctx, const void *k_src, const int32_t *src_off,
-                             int32_t n_src_rows, void *k_dst, const int32_t *cu,
-                             const int32_t *delta, int32_t n_blocks, int32_t n_rows, float2 *table,
-                             cudaStream_t stream) {
-  const int D = ctx->cfg.head_dim, H = ctx->cfg.n_kv_heads;
-  const int half = D / 2;
+ba_status ba_reencode_table_launch(ba_ctx *ctx, const int32_t *delta, int32_t n_blocks, float2 *table,
+                                   cudaStream_t stream) {
+  const int D = ctx->cfg.head_dim, half = D / 2;
   const double k = -2.0 / (double)D * log2(ctx->cfg.rope_theta);
-  int n = n_blocks * half;
+  const int n = n_blocks * half;
   ba_rope_table_kernel<<<(n + 127) / 128, 128, 0, stream>>>(delta, n_blocks, half, k, table);
   BA_CUDA_TRY(cudaGetLastError());
+  ctx->launches += 1;
+  return BA_OK;
+}
 
+ba_reencode_job ba_make_reencode_job(const ba_ctx *ctx, const void *k_src, const int32_t *src_off,
+                                     int32_t n_src_rows, void *k_dst, const int32_t *cu, const int32_t *delta,
+                                     int32_t n_blocks, int32_t n_rows, const float2 *table) {
+  ba_reencode_job job;
+  job.src = (const uint4 *)k_src; job.dst = (uint4 *)k_dst; job.src_off = src_off; job.cu = cu; job.delta = delta;
+  job.table = table; job.n_src_rows = n_src_rows; job.n_blocks = n_blocks; job.n_rows = n_rows;
+  job.head_dim = ctx->cfg.head_dim; job.row_vecs = ctx->cfg.n_kv_heads * ctx->cfg.head_dim / 8;
+  job.layout = ctx->cfg.rope_layout;
+  return job;
+}
+
+ba_status ba_reencode_main_launch(ba_ctx *ctx, const ba_reencode_job &job, cudaStream_t stream) {
 #ifndef BA_REENCODE_ROWS
 #define BA_REENCODE_ROWS 2
 #endif
   constexpr int kRows = BA_REENCODE_ROWS;   // rows in flight per thread
-  const int row_vecs = H * D / 8;
-  const bool adjacent = ctx->cfg.rope_layout == BA_ROPE_ADJACENT;
-  const int units = adjacent ? row_vecs : row_vecs / 2;
+  const bool adjacent = job.layout == BA_ROPE_ADJACENT;
+  const int units = adjacent ? job.row_vecs : job.row_vecs / 2;
   // threads per CTA: a multiple of the units per row, close to 256
   int threads = units >= 256 ? units : (256 / units) * units;
   if (threads > 512) return BA_ERR_UNSUPPORTED;   // more than 4096 bf16 per row
   const int rows_per_cta = (threads / units) * kRows;
-  const int grid = (n_rows + rows_per_cta - 1) / rows_per_cta;
-  ba_reencode_job job;
-  job.src = (const uint4 *)k_src; job.dst = (uint4 *)k_dst; job.src_off = src_off; job.cu = cu; job.delta = delta;
-  job.table = table; job.n_src_rows = n_src_rows; job.n_blocks = n_blocks; job.n_rows = n_rows;
-  job.head_dim = D; job.row_vecs = row_vecs; job.layout = ctx->cfg.rope_layout;
+  const int grid = (job.n_rows + rows_per_cta - 1) / rows_per_cta;
   if (adjacent)
     ba_reencode_kernel<BA_ROPE_ADJACENT, kRows><<<grid, threads, 0, stream>>>(job, ctx->dev_status);
   else
     ba_reencode_kernel<BA_ROPE_HALF, kRows><<<grid, threads, 0, stream>>>(job, ctx->dev_status);
   BA_CUDA_TRY(cudaGetLastError());
-  ctx->launches += 2;
+  ctx->launches += 1;
   return BA_OK;
+}
+
+ba_status ba_reencode_launch(ba_ctx *ctx, const void *k_src, const int32_t *src_off,
+                             int32_t n_src_rows, void *k_dst, const int32_t *cu,
+                             const int32_t *delta, int32_t n_blocks, int32_t n_rows, float2 *table,
+                             cudaStream_t stream) {
+  ba_status st = ba_reencode_table_launch(ctx, delta, n_blocks, table, stream);
+  if (st != BA_OK) return st;
+  return ba_reencode_main_launch(
+      ctx, ba_make_reencode_job(ctx, k_src, src_off, n_src_rows, k_dst, cu, delta, n_blocks, n_rows, table), stream);
+}
+
+ba_status ba_flush_pending(ba_ctx *ctx, cudaStream_t stream) {
+  if (!ctx->has_pending) return BA_OK;
+  ctx->has_pending = 0;
+  ctx->pending_table_bytes = 0;
+  return ba_reencode_main_launch(ctx, ctx->pending, stream);
 }
 
 // ---------------------------------------------------------------------------
@@ -141,6 +165,9 @@ extern "C" ba_status ba_reencode_k_noalloc(const ba_config *cfg, int device, con
   tmp.workspace_bytes = 0;
   tmp.dev_status = status_word ? status_word : g_noalloc_sink[device];
   tmp.launches = 0;
+  tmp.has_pending = 0;
+  tmp.pending_table_bytes = 0;
+  tmp.pending_stream = nullptr;
   return ba_reencode_launch(&tmp, k_src, src_off, n_src_rows, k_dst, cu, delta, n_blocks, n_rows,
                             g_noalloc_table[device], (cudaStream_t)stream);
 }

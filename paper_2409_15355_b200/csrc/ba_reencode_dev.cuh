@@ -5,19 +5,6 @@
 
 #include "ba_common.cuh"
 
-// One re-encoding job: block c of `n_blocks` is read from row src_off[c] (or cu[c]) of `src`,
-// rotated by delta[c] with the (cos, sin) pairs in `table`, and written to rows cu[c].. of `dst`.
-struct ba_reencode_job {
-  const uint4 *src;
-  uint4 *dst;
-  const int32_t *src_off;
-  const int32_t *cu;
-  const int32_t *delta;
-  const float2 *table;      // [n_blocks][head_dim / 2] (cos, sin)
-  int32_t n_src_rows, n_blocks, n_rows;
-  int32_t head_dim, row_vecs /* uint4 per row */, layout;
-};
-
 __device__ __forceinline__ int upper_bound_i32(const int32_t *a, int n, int x) {
   int lo = 0, hi = n;
   while (lo < hi) {

@@ -386,3 +386,46 @@ def test_bounded_wait_expires_into_a_status_and_the_device_stays_usable():
     c.close()
     o, lse, o_ref, lse_ref = run_prefill(w, B.BA_MODE_BLOCK)   # same process, same device: still works
     check_attention(o, o_ref, lse, lse_ref)
+
+
+@pytest.mark.parametrize("w,layout", [(W.config2(), B.BA_ROPE_ADJACENT), (W.config1(), B.BA_ROPE_HALF),
+                                      (W.config5(4, 64, 6, 32), B.BA_ROPE_ADJACENT)], ids=["rag", "tiny_half", "pool"])
+def test_deferred_reencode_rides_along_with_attention(w, layout):
+    """A queued re-encoding job is carried out by the next attention launch (or by ba_flush) and
+    gives the same bytes as the immediate call; the attention results are unaffected."""
+    c, seg, buf, src, want, ref, t = reencode_case(w, layout=layout)      # `want`: immediate ba_reencode_k
+    off = torch.from_numpy(W.warm_inputs(w)["src_off"]).cuda() if w.pool_lens is not None else None
+    Tc = t["n_cached_tokens"]
+    qb, kb, vb = W.prefill_inputs(w)
+    q, k, v = dev(qb), dev(kb), dev(vb)
+    o_plain = torch.empty(w.n_tokens, w.n_q_heads, w.head_dim, dtype=torch.float32, device="cuda")
+    o_with = torch.empty_like(o_plain)
+    B.ba_block_prefill(c.ctx, q, k, v, o_plain, None, seg, B.BA_MODE_BLOCK, B.BA_OUT_F32)
+    got = torch.zeros_like(want)
+    n0 = c.launches()
+    B.ba_reencode_k_deferred(c.ctx, src, off, src.shape[0], got, seg.cache_cu, seg.cache_delta, seg.n_cached_blocks, Tc)
+    assert c.launches() == n0 + 1                       # only the angle table so far
+    torch.cuda.synchronize()
+    assert not got.any()                                # nothing written yet
+    B.ba_block_prefill(c.ctx, q, k, v, o_with, None, seg, B.BA_MODE_BLOCK, B.BA_OUT_F32)
+    torch.cuda.synchronize()
+    assert c.device_status() == B.BA_OK
+    assert torch.equal(got, want)
+    assert torch.equal(o_with, o_plain)
+    # ba_flush runs a queued job on its own; a second flush is a no-op
+    got2 = torch.zeros_like(want)
+    B.ba_reencode_k_deferred(c.ctx, src, off, src.shape[0], got2, seg.cache_cu, seg.cache_delta, seg.n_cached_blocks, Tc)
+    B.ba_flush(c.ctx)
+    n1 = c.launches()
+    B.ba_flush(c.ctx)
+    assert c.launches() == n1
+    torch.cuda.synchronize()
+    assert torch.equal(got2, want)
+    # an immediate call while a job is queued uses its own table; queuing twice runs the first job
+    got3, got4, got5 = torch.zeros_like(want), torch.zeros_like(want), torch.zeros_like(want)
+    B.ba_reencode_k_deferred(c.ctx, src, off, src.shape[0], got3, seg.cache_cu, seg.cache_delta, seg.n_cached_blocks, Tc)
+    B.ba_reencode_k(c.ctx, src, off, src.shape[0], got4, seg.cache_cu, seg.cache_delta, seg.n_cached_blocks, Tc)
+    B.ba_reencode_k_deferred(c.ctx, src, off, src.shape[0], got5, seg.cache_cu, seg.cache_delta, seg.n_cached_blocks, Tc)
+    c.close()                                           # destroying the context runs what is still queued
+    torch.cuda.synchronize()
+    assert torch.equal(got3, want) and torch.equal(got4, want) and torch.equal(got5, want)
