@@ -49,6 +49,7 @@ constexpr int kBlockN = 128;      // keys per tile
 #endif
 constexpr int kStages = BA_STAGES;   // ring of K/V tiles (K_j, V_j, K_j+1, ...)
 constexpr float kRescaleThreshold = 8.0f;
+constexpr int kBgStageBytes = 16384; // two spare warps x two stages of source rows
 constexpr int kWorkSlots = 4;      // ring of published work entries (power of two)
 // Register split after launch (168 per thread): service warps give registers to the softmax warps.
 // 128 * BA_SVC_REGS + 256 * BA_SMX_REGS <= 384 * 168.
@@ -77,6 +78,8 @@ struct AttnParams {
   int persistent;                 // 1: CTAs draw work from work_counter; 0: CTA b handles entry b only
   int32_t *work_counter;          // device word, zero at launch: next entry of the work list
   ba_reencode_job bg;             // bg.n_rows > 0: a re-encoding job the two spare warps carry out meanwhile
+  int32_t *bg_counter;            // device word, zero at launch: next chunk of that job
+  int bg_rows_per_chunk;
   ba_segments seg;
 };
 
@@ -88,8 +91,9 @@ struct Layout {
   static constexpr int kQ0 = 0;
   static constexpr int kQ1 = kTileBytes;
   static constexpr int kRing = 2 * kTileBytes;
-  static constexpr int kCtrl = kRing + kStages * kTileBytes;
-  static constexpr int kBytes = kCtrl + 1024;
+  static constexpr int kCtrl = kRing + kStages * kTileBytes;   // 2 KB: Ctrl, then two ba_bg_smem
+  static constexpr int kBg = kCtrl + 2048;                     // staging of the background re-encoding
+  static constexpr int kBytes = kBg + 4 * kBgStageBytes;
 };
 
 struct Ctrl {
@@ -439,22 +443,14 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
     // ------------------------------------------------------------ spare warps: background re-encoding
     asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(BA_SVC_REGS));
     if (p.bg.n_rows > 0) {
-      // The 64 spare threads of every CTA together act as one wide row-walking engine: thread g
-      // owns one vector column and every rows_per_pass-th row (the host made sure that
-      // gridDim.x * 64 threads cover at least one row).
-      constexpr int kBgRows = 2;
-      const bool adjacent = p.bg.layout == BA_ROPE_ADJACENT;
-      const int upr = adjacent ? p.bg.row_vecs : (p.bg.row_vecs >> 1);
-      const int g = blockIdx.x * 64 + (tid - 320);
-      const int rows_per_pass = (int)(gridDim.x * 64) / upr;
-      if (g < rows_per_pass * upr) {
-        const int u = g % upr;
-        const int total_rows = min(p.bg.n_rows, __ldg(p.bg.cu + p.bg.n_blocks));
-        for (int row0 = g / upr; row0 < total_rows; row0 += rows_per_pass * kBgRows) {
-          if (adjacent) ba_reencode_rows<BA_ROPE_ADJACENT, kBgRows>(p.bg, u, row0, rows_per_pass, p.status);
-          else ba_reencode_rows<BA_ROPE_HALF, kBgRows>(p.bg, u, row0, rows_per_pass, p.status);
-        }
-      }
+      // each spare warp runs the staged engine with its own two 16 KB stages; chunks are drawn from a
+      // device-wide counter, so the job spreads over every CTA of the launch, early and late ones
+      const int bw = warp - 10;
+      ba_bg_smem *bsm = reinterpret_cast<ba_bg_smem *>(smem + L::kCtrl + 1024) + bw;
+      if ((tid & 31) == 0) { mbar_init(&bsm->bar[0], 1); mbar_init(&bsm->bar[1], 1); fence_barrier_init(); }
+      __syncwarp();
+      ba_reencode_background(p.bg, p.bg_counter, smem + L::kBg + bw * 2 * kBgStageBytes, bsm, p.bg_rows_per_chunk,
+                             p.status, [&](uint64_t *bar, uint32_t parity) { return mbar_wait(bar, parity, abort_flag); });
     }
   } else {
     // ------------------------------------------------------------ softmax, one thread per tile row
@@ -812,15 +808,18 @@ ba_status ba_attend_sm100_launch(ba_ctx *ctx, const ba_attend_args &a, const ba_
     tkc = tk; tvc = tv;
   }
   dim3 grid((unsigned)(p.persistent ? ctx->sm_count : work_upper));
-  // a queued re-encoding job rides along if the spare warps of this grid span at least one row;
-  // otherwise it is run on its own first
-  p.bg.n_rows = 0;
+  // a queued re-encoding job rides along in the spare warps; a job whose rows do not fit the
+  // staging buffers is run on its own first
+  p.bg.n_rows = 0; p.bg_counter = nullptr; p.bg_rows_per_chunk = 0;
   if (ctx->has_pending) {
-    const int upr = ctx->pending.layout == BA_ROPE_ADJACENT ? ctx->pending.row_vecs : ctx->pending.row_vecs / 2;
-    if ((long long)grid.x * 64 >= upr) {
+    const int row_bytes = ctx->pending.row_vecs * 16;
+    if (row_bytes <= kBgStageBytes) {
       p.bg = ctx->pending;
       ctx->has_pending = 0;
       ctx->pending_table_bytes = 0;
+      p.bg_rows_per_chunk = kBgStageBytes / row_bytes < 32 ? kBgStageBytes / row_bytes : 32;
+      p.bg_counter = reinterpret_cast<int32_t *>(reinterpret_cast<char *>(ctx->workspace) + ba_scratch_offset(ctx) - 128);
+      BA_CUDA_TRY(cudaMemsetAsync(p.bg_counter, 0, sizeof(int32_t), stream));
     } else {
       ba_status fs = ba_flush_pending(ctx, stream);
       if (fs != BA_OK) return fs;
