@@ -206,14 +206,24 @@ struct Work {
   int split;
 };
 
-// Decodes work index w: items are ordered heaviest-first (descending pair index: within a
-// sequence an item's cost grows with its index, the final block comes last), then head chunk,
-// then split.  Returns false past the end of the list.
+// Decodes work index w.  Returns false past the end of the list.
+//  Prefill: items heaviest-first (descending pair index: within a sequence an item's cost grows
+//  with its index, the final block comes last), then head chunk, then split.
+//  Final attend: all items cost about the same, so the pair index varies fastest instead: the
+//  CTAs running at the same time then work on the same (KV head, key range) for different query
+//  tiles and each K/V tile comes from HBM once and from L2 for the others.
 __device__ __forceinline__ bool next_work(const AttnParams &p, int w, Work &wk) {
   const int per_pair = p.n_chunks * p.n_splits;
-  const int rank = w / per_pair, rem = w - rank * per_pair;
   const int total_pairs = __ldg(p.seg.totals + (p.final_only ? 3 : 2));
-  if (rank >= total_pairs) return false;
+  int rank, rem;
+  if (p.final_only) {
+    if (total_pairs <= 0) return false;
+    rem = w / total_pairs; rank = w - rem * total_pairs;
+    if (rem >= per_pair) return false;
+  } else {
+    rank = w / per_pair; rem = w - rank * per_pair;
+    if (rank >= total_pairs) return false;
+  }
   if (!resolve_item(p, total_pairs - 1 - rank, wk.it)) return false;
   const int chunk = rem / p.n_splits;
   wk.split = rem - chunk * p.n_splits;
@@ -783,7 +793,7 @@ ba_status ba_attend_sm100_launch(ba_ctx *ctx, const ba_attend_args &a, const ba_
   // most two entries per SM (final block over a long cache) gains nothing from that and is
   // launched one CTA per entry.
   const long long work_upper = (long long)pairs_upper * (Hq / p.hpt) * n_splits;
-  p.persistent = work_upper > 2LL * ctx->sm_count;
+  p.persistent = items * n_splits > 2LL * ctx->sm_count;
   p.work_counter = nullptr;
   if (p.persistent) {
     // the counter lives in the last 256 bytes below the scratch area and is cleared per launch
