@@ -21,6 +21,7 @@
 // running maximum grows by more than 2^8, which keeps every term bounded and the
 // result exact in real arithmetic.
 #include <math.h>
+#include <type_traits>
 
 #include "ba_common.cuh"
 #include "ba_sm100.cuh"
@@ -131,17 +132,30 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
   return d;
 }
 
-// 2^x on the FMA pipe (x <= ~8): round x to the nearest integer n with the 1.5*2^23 trick,
-// evaluate a cubic fit of 2^r on r = x - n in [-0.5, 0.5] (relative error < 8e-5, far below
-// the bf16 rounding applied to the result) and add n to the exponent field.  Can take a
-// fixed share of the columns off the special-function unit (BA_POLY_PERIOD); off by default:
-// the softmax warps are bound by instruction issue, not by that unit, and it measured slower.
-__device__ __forceinline__ float exp2_poly(float x) {
-  x = fmaxf(x, -126.f);
-  const float t = x + 12582912.f;
-  const float r = x - (t - 12582912.f);
-  const float pr = fmaf(fmaf(fmaf(0.055088684f, r, 0.24260405f), r, 0.69327623f), r, 0.99992895f);
-  return __uint_as_float(__float_as_uint(pr) + (__float_as_uint(t) << 23));
+// 2^x for two values on the FMA pipe (x <= ~8): clamp at -126, round x to the nearest integer n
+// with the 1.5*2^23 trick, evaluate a cubic fit of 2^r on r = x - n in [-0.5, 0.5] (relative
+// error < 8e-5, far below the bf16 rounding applied to the result) and add n to the exponent
+// field.  The arithmetic is packed (two fp32 per instruction).  With BA_POLY_PERIOD = n, one
+// column pair in n goes this way and the special-function unit and the FMA pipe work side by
+// side; only tiles without masked columns use it, because a masked column must give exactly 0
+// and this gives 2^-126.  Off by default: at n = 4 the softmax of a tile gets about 6 % shorter
+// in cycles, but the extra instructions cost more clock under the power limit than that (+2.7 %
+// time at 32K context; n = 2, 3 are slower still).
+__device__ __forceinline__ uint64_t exp2_poly2(uint64_t x2) {
+  float x0, x1;
+  unpack2(x2, x0, x1);
+  x2 = pack2(fmaxf(x0, -126.f), fmaxf(x1, -126.f));
+  const uint64_t t2 = add2(x2, pack2(12582912.f, 12582912.f));
+  const uint64_t u2 = add2(t2, pack2(-12582912.f, -12582912.f));
+  const uint64_t r2 = fma2(u2, pack2(-1.f, -1.f), x2);
+  uint64_t q2 = fma2(pack2(0.055088684f, 0.055088684f), r2, pack2(0.24260405f, 0.24260405f));
+  q2 = fma2(q2, r2, pack2(0.69327623f, 0.69327623f));
+  q2 = fma2(q2, r2, pack2(0.99992895f, 0.99992895f));
+  float q0, q1, t0, t1;
+  unpack2(q2, q0, q1);
+  unpack2(t2, t0, t1);
+  return pack2(__uint_as_float(__float_as_uint(q0) + (__float_as_uint(t0) << 23)),
+               __uint_as_float(__float_as_uint(q1) + (__float_as_uint(t1) << 23)));
 }
 #ifndef BA_POLY_PERIOD
 #define BA_POLY_PERIOD 0
@@ -149,12 +163,8 @@ __device__ __forceinline__ float exp2_poly(float x) {
 #ifndef BA_SPLIT_P
 #define BA_SPLIT_P 1
 #endif
-constexpr int kPolyPeriod = BA_POLY_PERIOD;    // one column in kPolyPeriod uses exp2_poly (0: none)
+constexpr int kPolyPeriod = BA_POLY_PERIOD;    // one column pair in kPolyPeriod uses exp2_poly2 (0: none)
 constexpr bool kSplitP = BA_SPLIT_P;             // hand P to the MMA warp in two halves
-#ifndef BA_PACKED
-#define BA_PACKED 1
-#endif
-constexpr bool kPacked = BA_PACKED;              // packed fp32x2 arithmetic in the exponent loop
 
 __device__ __forceinline__ int upper_bound_tbl(const int32_t *a, int n, int x) {
   int lo = 0, hi = n;
@@ -551,46 +561,46 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
           }
         }
         const float neg_m = (m_used == -INFINITY) ? 0.f : -m_used * sl;   // no visible key so far: every p is 0
-        float sum[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
         uint64_t sum2[4] = {0ull, 0ull, 0ull, 0ull};       // packed (0.f, 0.f)
         const uint64_t sl2 = pack2(sl, sl), negm2 = pack2(neg_m, neg_m);
         // P is handed to the MMA warp in two halves so that PV can start on the first 64 keys
-        // while the second 64 are still being exponentiated
+        // while the second 64 are still being exponentiated.  The arithmetic is packed fp32x2.
+        auto exp_halves = [&](auto poly_tag) {
+          constexpr bool kPoly = decltype(poly_tag)::value;
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
-          uint32_t pk[32];
+          for (int h = 0; h < 2; ++h) {
+            uint32_t pk[32];
 #pragma unroll
-          for (int i = 0; i < 32; ++i) {
-            const int e0 = h * 64 + 2 * i, e1 = e0 + 1;
-            float p0, p1;
-            if (kPacked) {
-              float x0, x1;
-              unpack2(fma2(pack2(__uint_as_float(s[e0]), __uint_as_float(s[e1])), sl2, negm2), x0, x1);
-              p0 = ex2(x0); p1 = ex2(x1);
+            for (int i = 0; i < 32; ++i) {
+              const int e0 = h * 64 + 2 * i, e1 = e0 + 1;
+              const uint64_t x2 = fma2(pack2(__uint_as_float(s[e0]), __uint_as_float(s[e1])), sl2, negm2);
+              float p0, p1;
+              if (kPoly && i % (kPolyPeriod > 0 ? kPolyPeriod : 1) == kPolyPeriod - 1) {
+                unpack2(exp2_poly2(x2), p0, p1);
+              } else {
+                float x0, x1;
+                unpack2(x2, x0, x1);
+                p0 = ex2(x0); p1 = ex2(x1);
+              }
               sum2[i & 3] = add2(sum2[i & 3], pack2(p0, p1));
-            } else {
-              const float x0 = fmaf(__uint_as_float(s[e0]), sl, neg_m);
-              const float x1 = fmaf(__uint_as_float(s[e1]), sl, neg_m);
-              p0 = (kPolyPeriod > 0 && e0 % (kPolyPeriod > 0 ? kPolyPeriod : 1) == kPolyPeriod - 1) ? exp2_poly(x0) : ex2(x0);
-              p1 = (kPolyPeriod > 0 && e1 % (kPolyPeriod > 0 ? kPolyPeriod : 1) == kPolyPeriod - 1) ? exp2_poly(x1) : ex2(x1);
-              sum[e0 & 7] += p0; sum[e1 & 7] += p1;
+              __nv_bfloat162 v = __floats2bfloat162_rn(p0, p1);
+              pk[i] = *reinterpret_cast<uint32_t *>(&v);
             }
-            __nv_bfloat162 v = __floats2bfloat162_rn(p0, p1);
-            pk[i] = *reinterpret_cast<uint32_t *>(&v);
+            tmem_st_32x32b_x32(tS + h * 32, pk);
+            if (kSplitP || h == 1) {
+              tmem_wait_st();
+              tc_fence_before();
+              if (!kSplitP) mbar_arrive(&ctrl->p_full[t][0]);
+              mbar_arrive(&ctrl->p_full[t][h]);
+            }
+            if (r == 0) BA_TR(t, j, 4 + h);
           }
-          tmem_st_32x32b_x32(tS + h * 32, pk);
-          if (kSplitP || h == 1) {
-            tmem_wait_st();
-            tc_fence_before();
-            if (!kSplitP) mbar_arrive(&ctrl->p_full[t][0]);
-            mbar_arrive(&ctrl->p_full[t][h]);
-          }
-          if (r == 0) BA_TR(t, j, 4 + h);
-        }
-        if (kPacked) {
+        };
+        if (kPolyPeriod > 0 && __all_sync(0xffffffffu, lim >= kBlockN - 1)) exp_halves(std::true_type{});
+        else exp_halves(std::false_type{});
+        float sum[8];
 #pragma unroll
-          for (int i = 0; i < 4; ++i) unpack2(sum2[i], sum[2 * i], sum[2 * i + 1]);
-        }
+        for (int i = 0; i < 4; ++i) unpack2(sum2[i], sum[2 * i], sum[2 * i + 1]);
         l += ((sum[0] + sum[1]) + (sum[2] + sum[3])) + ((sum[4] + sum[5]) + (sum[6] + sum[7]));
       }
 
