@@ -105,6 +105,9 @@ typedef struct {
   int32_t *cu_ftile;       /* [batch+1] */
   int32_t *cache_tile_cu;  /* [Bc+1] prefix sum of 128-key tiles per cached block (a tile never spans two blocks) */
   int32_t *totals;         /* [8]: cached tokens, final tokens, q tiles, final tiles, ..., [7] = validity word */
+  /* rotation of every cached block, used by ba_final_attend_fused: (cos, sin)(cache_delta[c] * theta_m),
+   * fp32 from fp64 angles, [Bc][head_dim / 2][2] */
+  float *cache_rope;
 } ba_segments;
 
 /* Create a context on CUDA device `device` and allocate `workspace_bytes` of
@@ -258,6 +261,30 @@ ba_status ba_final_attend(ba_ctx *ctx, const void *q_f, const void *k_f, const v
                           int32_t n_cache_rows, const int32_t *v_src_off, int32_t n_v_rows,
                           void *o, float *lse, const ba_segments *seg, ba_mode mode,
                           ba_out_dtype out_dtype, void *stream);
+
+/*
+ * Section 2.5, steps 2 and 3 in one launch: the final block of every sequence attends that
+ * sequence's cached blocks and itself, with the cached keys still at their CACHE-TIME positions
+ * (token t of a block rotated to position t, as Section 2.3 stores them).  The position
+ * re-encoding of Eq. 3 after Eq. 2 -- one rotation by the block's delta -- is applied to the
+ * other side of the dot product: (R(p) q) . (R(delta + t) k) = (R(-delta) R(p) q) . (R(t) k),
+ * so the query tiles are rotated once per cached block on chip and the cached keys are neither
+ * rewritten nor read twice.  The result equals ba_reencode_k followed by ba_final_attend up to
+ * the rounding of the rotated operand to bf16 (queries here, keys there).  Re-encoded keys are
+ * not produced; a later decode phase that wants them calls ba_reencode_k off the critical path.
+ *   q_f, k_f, v_f   as for ba_final_attend
+ *   k_src, v_src    bf16 [n_src_rows, n_kv_heads, head_dim]: cached block c (cache order, as in
+ *                   seg->cache_cu) occupies rows src_off[c] .. src_off[c] + length - 1 of both, or
+ *                   rows cache_cu[c] .. when src_off is NULL (cache packing)
+ *   n_cache_rows    total cached rows of the batch (= cache_cu[Bc])
+ *   seg             tables of ba_segment(); its cache_rope table holds the rotations
+ * A queued ba_reencode_k_deferred job is run as a stand-alone launch first.
+ */
+ba_status ba_final_attend_fused(ba_ctx *ctx, const void *q_f, const void *k_f, const void *v_f,
+                                int32_t n_final_rows, const void *k_src, const void *v_src,
+                                int32_t n_src_rows, const int32_t *src_off, int32_t n_cache_rows,
+                                void *o, float *lse, const ba_segments *seg, ba_mode mode,
+                                ba_out_dtype out_dtype, void *stream);
 
 #ifdef __cplusplus
 }

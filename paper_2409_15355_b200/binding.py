@@ -24,6 +24,7 @@ EXPORTS = [
     "ba_create", "ba_destroy", "ba_status_string", "ba_workspace_bytes", "ba_last_device_status",
     "ba_launch_count", "ba_segments_bytes", "ba_segment", "ba_reencode_k", "ba_block_prefill",
     "ba_final_attend", "ba_reencode_k_noalloc", "ba_selftest_wait_expiry", "ba_reencode_k_deferred", "ba_flush",
+    "ba_final_attend_fused",
 ]
 BA_NOALLOC_MAX_BLOCKS = 4096
 
@@ -41,7 +42,7 @@ class ba_segments(C.Structure):
             "cu_seq", "cu_cache_seq", "cu_final_seq", "cu_seq_block", "cu_block", "block_delta",
             "block_seq", "block_kv_begin", "block_part_off", "block_is_final", "cache_block",
             "cache_cu", "cache_delta", "tok_block", "tok_pos", "tok_pos_local", "cu_qtile",
-            "cu_ftile", "cache_tile_cu", "totals")]
+            "cu_ftile", "cache_tile_cu", "totals", "cache_rope")]
 
 
 class BaError(RuntimeError):
@@ -195,6 +196,14 @@ def ba_block_prefill(ctx, q, k, v, o, lse, seg, mode, out_dtype, stream=None):
     _check(load_library().ba_block_prefill(ctx, _ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(lse),
                                            C.byref(seg), mode, out_dtype, _stream_ptr(stream)),
            "ba_block_prefill")
+
+
+def ba_final_attend_fused(ctx, q_f, k_f, v_f, n_final_rows, k_src, v_src, n_src_rows, src_off,
+                          n_cache_rows, o, lse, seg, mode, out_dtype, stream=None):
+    _check(load_library().ba_final_attend_fused(ctx, _ptr(q_f), _ptr(k_f), _ptr(v_f), n_final_rows,
+                                                _ptr(k_src), _ptr(v_src), n_src_rows, _ptr(src_off),
+                                                n_cache_rows, _ptr(o), _ptr(lse), C.byref(seg), mode,
+                                                out_dtype, _stream_ptr(stream)), "ba_final_attend_fused")
 
 
 def ba_final_attend(ctx, q_f, k_f, v_f, n_final_rows, k_cache, v_cache, n_cache_rows, v_src_off,

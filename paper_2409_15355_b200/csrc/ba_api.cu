@@ -61,6 +61,7 @@ TableLayout table_layout(int32_t batch, int32_t B, int32_t T) {
   take((size_t)(batch + 1) * 4);                              // cu_ftile
   take((size_t)(B + 1) * 4);                                  // cache_tile_cu
   take(8 * 4);                                                // totals
+  take((size_t)B * 64 * 8);                                   // cache_rope: at most 64 rotary pairs per block
   L.bytes = cur;
   return L;
 }
@@ -209,7 +210,11 @@ ba_status ba_segment(ba_ctx *ctx, const int32_t *block_lens, const int32_t *seq_
   out->cache_block = next(); out->cache_cu = next(); out->cache_delta = next();
   out->tok_block = next(); out->tok_pos = next(); out->tok_pos_local = next();
   out->cu_qtile = next(); out->cu_ftile = next(); out->cache_tile_cu = next(); out->totals = next();
-  return ba_segment_launch(ctx, d_lens, d_nb, batch, n_blocks, n_tokens, mode, out, s);
+  out->cache_rope = (float *)next();
+  ba_status st = ba_segment_launch(ctx, d_lens, d_nb, batch, n_blocks, n_tokens, mode, out, s);
+  if (st != BA_OK || out->n_cached_blocks == 0) return st;
+  // rotations of the cached blocks (the same angle table ba_reencode_k builds), once per prompt
+  return ba_reencode_table_launch(ctx, out->cache_delta, out->n_cached_blocks, (float2 *)out->cache_rope, s);
 }
 
 static ba_status check_reencode_args(ba_ctx *ctx, const void *k_src, const int32_t *src_off, int32_t n_src_rows,
@@ -321,6 +326,35 @@ ba_status ba_final_attend(ba_ctx *ctx, const void *q_f, const void *k_f, const v
   a.k_cache = (const __nv_bfloat16 *)k_cache; a.v_cache = (const __nv_bfloat16 *)v_cache;
   a.n_cache_rows = n_cache_rows; a.n_v_rows = v_src_off ? n_v_rows : n_cache_rows;
   a.v_src_off = v_src_off;
+  a.out_f32 = out_dtype == BA_OUT_F32;
+  a.final_only = 1;
+  return ba_attend_launch(ctx, a, seg, (cudaStream_t)stream);
+}
+
+ba_status ba_final_attend_fused(ba_ctx *ctx, const void *q_f, const void *k_f, const void *v_f,
+                                int32_t n_final_rows, const void *k_src, const void *v_src,
+                                int32_t n_src_rows, const int32_t *src_off, int32_t n_cache_rows,
+                                void *o, float *lse, const ba_segments *seg, ba_mode mode,
+                                ba_out_dtype out_dtype, void *stream) {
+  ba_status st = check_attend_common(ctx, q_f, k_f, v_f, o, seg, mode, out_dtype);
+  if (st != BA_OK) return st;
+  if (n_final_rows < 0 || n_cache_rows < 0 || n_src_rows < 0) return BA_ERR_INVALID_ARG;
+  if (n_cache_rows > 0) {
+    if (!k_src || !v_src || !aligned16(k_src) || !aligned16(v_src)) return BA_ERR_INVALID_ARG;
+    if (n_src_rows < 1 || !seg->cache_rope || !seg->cache_tile_cu) return BA_ERR_INVALID_ARG;
+    if (!src_off && n_src_rows < n_cache_rows) return BA_ERR_INVALID_ARG;
+  }
+  BA_CUDA_TRY(cudaSetDevice(ctx->device));
+  ba_attend_args a;
+  memset(&a, 0, sizeof(a));
+  a.q = (const __nv_bfloat16 *)q_f; a.k = (const __nv_bfloat16 *)k_f; a.v = (const __nv_bfloat16 *)v_f;
+  a.o = o; a.lse = lse; a.n_q_rows = n_final_rows; a.n_kv_rows = n_final_rows;
+  a.k_cache = (const __nv_bfloat16 *)k_src; a.v_cache = (const __nv_bfloat16 *)v_src;
+  a.n_cache_rows = n_cache_rows;
+  a.fused = 1;
+  a.k_src_off = src_off; a.n_k_rows = n_src_rows;
+  // values: addressed like the keys.  The kernel's value map covers n_v_rows rows when an offset table is given.
+  a.v_src_off = src_off; a.n_v_rows = n_src_rows;
   a.out_f32 = out_dtype == BA_OUT_F32;
   a.final_only = 1;
   return ba_attend_launch(ctx, a, seg, (cudaStream_t)stream);

@@ -20,6 +20,13 @@
 // operand of the PV product.  O is rescaled in tensor memory only when the
 // running maximum grows by more than 2^8, which keeps every term bounded and the
 // result exact in real arithmetic.
+//
+// Fused warm path (Section 2.5 steps 2 and 3 in one launch): the cached keys stay at their
+// cache-time positions and the position difference of each block (Eq. 3 after Eq. 2) is applied
+// to the other side of the dot product, (R(p) q) . (R(delta + t) k) = (R(-delta) R(p) q) . (R(t) k):
+// warps 10-11 counter-rotate the two query tiles once per cached block into a second pair of
+// buffers, which the QK^T products of that block's key tiles read.  The cached keys are then
+// never rewritten or re-read, and a key tile never spans two blocks.
 #include <math.h>
 #include <type_traits>
 
@@ -76,6 +83,11 @@ struct AttnParams {
   float *o_part;                  // [n_splits, n_q_rows, Hq, D] fp32, each normalised by its own denominator
   float *lse_part;                // [n_splits, n_q_rows, Hq] natural-log denominators (-inf: split saw no key)
   const int32_t *v_src_off;       // non-null: values of cached block c start at pool row v_src_off[c]
+  const int32_t *k_src_off;       // non-null: keys of cached block c start at pool row k_src_off[c] (fused path only)
+  int walk;                       // cached keys are walked block by block (a tile never spans two blocks)
+  int fused;                      // cached keys are at cache-time positions: queries are counter-rotated per block
+  int rope_layout;
+  const float2 *q_rope;           // fused: [cached blocks][D/2] (cos, sin) of delta_c * theta_m
   int persistent;                 // 1: CTAs draw work from work_counter; 0: CTA b handles entry b only
   int32_t *work_counter;          // device word, zero at launch: next entry of the work list
   ba_reencode_job bg;             // bg.n_rows > 0: a re-encoding job the two spare warps carry out meanwhile
@@ -93,7 +105,8 @@ struct Layout {
   static constexpr int kQ1 = kTileBytes;
   static constexpr int kRing = 2 * kTileBytes;
   static constexpr int kCtrl = kRing + kStages * kTileBytes;   // 2 KB: Ctrl, then two ba_bg_smem
-  static constexpr int kBg = kCtrl + 2048;                     // staging of the background re-encoding
+  static constexpr int kBg = kCtrl + 2048;                     // staging of the background re-encoding, or (fused
+                                                               // path) the two counter-rotated query tiles
   static constexpr int kBytes = kBg + 4 * kBgStageBytes;
 };
 
@@ -106,6 +119,8 @@ struct Ctrl {
   uint64_t p_full[2][2];          // [query tile][half of the P tile]
   uint64_t o_done[2];
   uint64_t o_free[2];             // the softmax warps have read O_t out of tensor memory
+  uint64_t qr_full[2];            // fused: counter-rotated query tile t is ready for the current cached block
+  uint64_t qr_empty[2];           // fused: every QK^T reading it has completed
   uint64_t work_full[kWorkSlots];  // work entry published by the scheduler (producer thread)
   uint64_t work_empty[kWorkSlots]; // entry read by the MMA thread and the 8 softmax warps
   int work_ring[kWorkSlots];
@@ -189,7 +204,7 @@ __device__ __forceinline__ bool resolve_item(const AttnParams &p, int pair, Item
     it.own_row0 = f0;
     it.cb0 = __ldg(sg.cu_seq_block + s) - s;           // every earlier sequence has one final block
     it.ctile0 = __ldg(sg.cache_tile_cu + it.cb0);
-    it.n_cache_tiles = p.v_src_off ? __ldg(sg.cache_tile_cu + (__ldg(sg.cu_seq_block + s + 1) - s - 1)) - it.ctile0
+    it.n_cache_tiles = p.walk ? __ldg(sg.cache_tile_cu + (__ldg(sg.cu_seq_block + s + 1) - s - 1)) - it.ctile0
                                    : (it.cache_len + kBlockN - 1) / kBlockN;
   } else {
     if (pair >= __ldg(sg.totals + 2)) return false;
@@ -244,6 +259,76 @@ __device__ __forceinline__ bool next_work(const AttnParams &p, int w, Work &wk) 
   return true;
 }
 
+// Block-by-block walk of the cached keys: index (cache order) of the block that holds key tile
+// `target` (counted over the whole batch); the sequence's blocks follow cb0.
+__device__ __forceinline__ int find_cache_block(const AttnParams &p, const Item &it, int target) {
+  int lo = it.cb0, hi = p.seg.n_cached_blocks;
+  while (lo < hi) {
+    const int mid = (lo + hi + 1) >> 1;
+    if (__ldg(p.seg.cache_tile_cu + mid) <= target) lo = mid; else hi = mid - 1;
+  }
+  return lo;
+}
+
+// Counter-rotation of query rows [row_begin, row_end) of one tile (fused warm path): dst = R(-delta) src,
+// with cs = (cos, sin)(delta * theta_m) of the current cached block.  Both tiles are in the 128-byte
+// swizzled layout the tensor maps produce: 64-column regions of 128 rows x 128 bytes, the 16-byte
+// chunk c of row r stored at chunk position c ^ (r & 7).  Called by one full warp; a lane keeps its
+// chunk column, so its (cos, sin) values are loaded once per block.
+__device__ __forceinline__ uint32_t rot_word_adjacent(uint32_t w, float2 cs) {
+  const float x = __uint_as_float(w << 16), y = __uint_as_float(w & 0xffff0000u);
+  __nv_bfloat162 v = __floats2bfloat162_rn(fmaf(x, cs.x, y * cs.y), fmaf(y, cs.x, -x * cs.y));
+  return *reinterpret_cast<uint32_t *>(&v);
+}
+__device__ __forceinline__ void rot_words_half(uint32_t &a, uint32_t &b, float2 cs0, float2 cs1) {
+  // a holds x of pairs m, m+1; b holds their partners y
+  const float x0 = __uint_as_float(a << 16), x1 = __uint_as_float(a & 0xffff0000u);
+  const float y0 = __uint_as_float(b << 16), y1 = __uint_as_float(b & 0xffff0000u);
+  __nv_bfloat162 va = __floats2bfloat162_rn(fmaf(x0, cs0.x, y0 * cs0.y), fmaf(x1, cs1.x, y1 * cs1.y));
+  __nv_bfloat162 vb = __floats2bfloat162_rn(fmaf(y0, cs0.x, -x0 * cs0.y), fmaf(y1, cs1.x, -x1 * cs1.y));
+  a = *reinterpret_cast<uint32_t *>(&va);
+  b = *reinterpret_cast<uint32_t *>(&vb);
+}
+template <int D>
+__device__ __forceinline__ void rotate_q_rows(const uint8_t *src, uint8_t *dst, const float2 *cs_row, int layout,
+                                              int row_begin, int row_end, int lane) {
+  constexpr int kRegion = 128 * 128;
+  if (layout == BA_ROPE_ADJACENT) {
+    const int chunk = lane & 7;
+#pragma unroll
+    for (int c = 0; c < D / 64; ++c) {
+      float2 cs[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) cs[i] = __ldg(cs_row + c * 32 + chunk * 4 + i);
+      for (int row = row_begin + (lane >> 3); row < row_end; row += 4) {
+        const int off = c * kRegion + row * 128 + ((chunk ^ (row & 7)) << 4);
+        uint4 v = *reinterpret_cast<const uint4 *>(src + off);
+        v.x = rot_word_adjacent(v.x, cs[0]); v.y = rot_word_adjacent(v.y, cs[1]);
+        v.z = rot_word_adjacent(v.z, cs[2]); v.w = rot_word_adjacent(v.w, cs[3]);
+        *reinterpret_cast<uint4 *>(dst + off) = v;
+      }
+    }
+  } else {
+    // pairs (m, m + D/2): D = 128 pairs chunk c of region 0 with chunk c of region 1;
+    // D = 64 pairs chunk c (< 4) with chunk c + 4 of the only region
+    constexpr int kCols = (D == 128) ? 8 : 4;        // chunk columns holding x
+    const int chunk = lane % kCols;
+    float2 cs[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) cs[i] = __ldg(cs_row + chunk * 8 + i);
+    for (int row = row_begin + lane / kCols; row < row_end; row += 32 / kCols) {
+      const int off_x = row * 128 + ((chunk ^ (row & 7)) << 4);
+      const int off_y = (D == 128) ? off_x + kRegion : row * 128 + (((chunk + 4) ^ (row & 7)) << 4);
+      uint4 a = *reinterpret_cast<const uint4 *>(src + off_x);
+      uint4 b = *reinterpret_cast<const uint4 *>(src + off_y);
+      rot_words_half(a.x, b.x, cs[0], cs[1]); rot_words_half(a.y, b.y, cs[2], cs[3]);
+      rot_words_half(a.z, b.z, cs[4], cs[5]); rot_words_half(a.w, b.w, cs[6], cs[7]);
+      *reinterpret_cast<uint4 *>(dst + off_x) = a;
+      *reinterpret_cast<uint4 *>(dst + off_y) = b;
+    }
+  }
+}
+
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
 ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
@@ -264,8 +349,10 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
     for (int t = 0; t < 2; ++t) {
       mbar_init(&ctrl->s_full[t], 1); mbar_init(&ctrl->p_full[t][0], 128); mbar_init(&ctrl->p_full[t][1], 128);
       mbar_init(&ctrl->o_done[t], 1); mbar_init(&ctrl->o_free[t], 128);
+      mbar_init(&ctrl->qr_full[t], 2); mbar_init(&ctrl->qr_empty[t], 1);
     }
-    for (int k = 0; k < kWorkSlots; ++k) { mbar_init(&ctrl->work_full[k], 1); mbar_init(&ctrl->work_empty[k], 9); }
+    // an entry is read by the MMA thread and the 8 softmax warps, on the fused path also by warps 10-11
+    for (int k = 0; k < kWorkSlots; ++k) { mbar_init(&ctrl->work_full[k], 1); mbar_init(&ctrl->work_empty[k], p.fused ? 11 : 9); }
     ctrl->abort_flag = 0;
     fence_barrier_init();
   }
@@ -318,15 +405,9 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
         }
         // pool mode: cached keys are walked block by block (block pc, row offset poff inside it)
         int pc = 0, poff = 0;
-        if (p.v_src_off && wk.tile0 < it.n_cache_tiles) {
+        if (p.walk && wk.tile0 < it.n_cache_tiles) {
           const int target = it.ctile0 + wk.tile0;
-          // last block whose first tile is <= target; the sequence's blocks follow cb0 in cache order
-          int lo = it.cb0, hi = p.seg.n_cached_blocks;
-          while (lo < hi) {
-            const int mid = (lo + hi + 1) >> 1;
-            if (__ldg(p.seg.cache_tile_cu + mid) <= target) lo = mid; else hi = mid - 1;
-          }
-          pc = lo;
+          pc = find_cache_block(p, it, target);
           poff = (target - __ldg(p.seg.cache_tile_cu + pc)) * kBlockN;
         }
         for (int j = 0; j < wk.n_tiles && ok; ++j) {
@@ -335,12 +416,12 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
           int k_row, v_row;
           if (!cached) {
             k_row = v_row = it.own_row0 + (jt - it.n_cache_tiles) * kBlockN;
-          } else if (!p.v_src_off) {
+          } else if (!p.walk) {
             k_row = v_row = it.cache_row0 + jt * kBlockN;
           } else {
             const int c_begin = __ldg(p.seg.cache_cu + pc), c_len = __ldg(p.seg.cache_cu + pc + 1) - c_begin;
-            k_row = c_begin + poff;
-            v_row = __ldg(p.v_src_off + pc) + poff;
+            k_row = (p.k_src_off ? __ldg(p.k_src_off + pc) : c_begin) + poff;
+            v_row = (p.v_src_off ? __ldg(p.v_src_off + pc) : c_begin) + poff;
             ctrl->tile_valid[(gidx >> 1) & 7] = min(kBlockN, c_len - poff);   // read by the softmax warps
             poff += kBlockN;
             if (poff >= c_len) { ++pc; poff = 0; }
@@ -381,12 +462,12 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
       const uint64_t q_desc[2] = {make_smem_desc(q_addr[0], 16, 1024), make_smem_desc(q_addr[1], 16, 1024)};
       const uint64_t k_desc0 = make_smem_desc(ring, 16, 1024);
       const uint64_t v_desc0 = make_smem_desc(ring, L::kRegionBytes, 1024);
-      auto issue_qk = [&](int t, int idx) {
+      auto issue_qk_with = [&](int t, int idx, uint64_t qd) {
         const uint64_t kd = k_desc0 + (uint64_t)(((idx % kStages) * L::kTileBytes) >> 4);
 #pragma unroll
         for (int k = 0; k < D / 16; ++k) {
           const uint64_t off = (uint64_t)(((k >> 2) * L::kRegionBytes + (k & 3) * 32) >> 4);
-          mma_ss(tS[t], q_desc[t] + off, kd + off, idesc_qk, k > 0);
+          mma_ss(tS[t], qd + off, kd + off, idesc_qk, k > 0);
         }
         mma_commit(&ctrl->s_full[t]);
       };
@@ -400,8 +481,33 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
       int gidx = 0;                        // K/V tiles consumed so far (ring position)
       int q_uses[2] = {0, 0};              // items in which query tile t was loaded
       int p_uses[2] = {0, 0};              // P tiles of query tile t consumed
-      Work wk;
+      Work wk = {};
       int n_work = 0;
+      // fused path: the QK^T of a cached key tile reads the query tile counter-rotated for that tile's
+      // block; warps 10-11 rotate once per (block, query tile) and the two sides count those alike
+      const uint64_t qr_desc[2] = {make_smem_desc(smem_u32(smem + L::kBg), 16, 1024),
+                                   make_smem_desc(smem_u32(smem + L::kBg + L::kTileBytes), 16, 1024)};
+      int n_rot[2] = {0, 0};               // rotations of query tile t consumed so far
+      int rot_block[2] = {-1, -1};         // cached block the rotated tile t currently belongs to
+      int walk_pc = -1, walk_end = 0;      // block of the current cached tile and the tile index where it ends
+      // S_t = Q_t K^T for tile `jrel` of the entry, whose keys sit at ring position idx
+      auto issue_qk = [&](int t, int jrel, int idx) -> bool {
+        const int jt = wk.tile0 + jrel;
+        if (!p.fused || jt >= wk.it.n_cache_tiles) { issue_qk_with(t, idx, q_desc[t]); return true; }
+        const int g = wk.it.ctile0 + jt;
+        if (walk_pc < 0) { walk_pc = find_cache_block(p, wk.it, g); walk_end = __ldg(p.seg.cache_tile_cu + walk_pc + 1); }
+        while (g >= walk_end) { ++walk_pc; walk_end = __ldg(p.seg.cache_tile_cu + walk_pc + 1); }
+        if (rot_block[t] != walk_pc) {
+          if (!mbar_wait(&ctrl->qr_full[t], n_rot[t] & 1, abort_flag)) return false;
+          ++n_rot[t];
+          rot_block[t] = walk_pc;
+          tc_fence_after();
+        }
+        issue_qk_with(t, idx, qr_desc[t]);
+        // last key tile of this block within the entry: the rotated tile may be overwritten afterwards
+        if (g + 1 == walk_end || jt + 1 == min(wk.tile0 + wk.n_tiles, wk.it.n_cache_tiles)) mma_commit(&ctrl->qr_empty[t]);
+        return true;
+      };
       for (;;) {
         const int slot = n_work & (kWorkSlots - 1);
         ok = mbar_wait(&ctrl->work_full[slot], (n_work / kWorkSlots) & 1, abort_flag);
@@ -412,11 +518,13 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
         mbar_arrive(&ctrl->work_empty[slot]);          // the entry has been decoded into registers
         const int n_tiles = wk.n_tiles, n_qt = wk.it.n_qt;
         if (n_tiles == 0) continue;
+        walk_pc = -1; rot_block[0] = rot_block[1] = -1;
         for (int t = 0; t < n_qt && ok; ++t) ok = mbar_wait(&ctrl->q_full[t], q_uses[t] & 1, abort_flag);
         if (ok) ok = wait_kv(gidx);
         if (!ok) break;
         tc_fence_after();
-        for (int t = 0; t < n_qt; ++t) issue_qk(t, gidx);
+        for (int t = 0; t < n_qt && ok; ++t) ok = issue_qk(t, 0, gidx);
+        if (!ok) break;
         mma_commit(&ctrl->kv_empty[gidx % kStages]);
         if (n_tiles == 1) mma_commit(&ctrl->q_empty);
         for (int j = 0; j < n_tiles && ok; ++j) {
@@ -446,7 +554,8 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
             if (last) mma_commit(&ctrl->o_done[t]);
             if (t + 1 == n_qt) mma_commit(&ctrl->kv_empty[iv % kStages]);
             if (!last) {
-              issue_qk(t, ik);
+              ok = issue_qk(t, j + 1, ik);
+              if (!ok) break;
               BA_TR(2, j, t * 4 + 3);
               if (t + 1 == n_qt) {
                 mma_commit(&ctrl->kv_empty[ik % kStages]);
@@ -462,7 +571,51 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
   } else if (warp >= 10) {
     // ------------------------------------------------------------ spare warps: background re-encoding
     asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(BA_SVC_REGS));
-    if (p.bg.n_rows > 0) {
+    if (p.fused) {
+      // fused warm path: counter-rotate the query tiles for each cached block of each work entry
+      // (warp 10 rows 0-63, warp 11 rows 64-127 of a tile)
+      const int bw = warp - 10, lane = tid & 31;
+      int n_rot[2] = {0, 0}, q_uses[2] = {0, 0};
+      bool ok = true;
+      Work wk;
+      int n_work = 0;
+      for (;;) {
+        const int slot = n_work & (kWorkSlots - 1);
+        ok = mbar_wait(&ctrl->work_full[slot], (n_work / kWorkSlots) & 1, abort_flag);
+        if (!ok) break;
+        const int w = ctrl->work_ring[slot];
+        ++n_work;
+        if (w < 0 || !next_work(p, w, wk)) break;
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&ctrl->work_empty[slot]);
+        if (wk.n_tiles == 0) continue;
+        const Item &it = wk.it;
+        const int j_end = min(wk.tile0 + wk.n_tiles, it.n_cache_tiles);
+        if (wk.tile0 < j_end) {
+          for (int t = 0; t < it.n_qt && ok; ++t) ok = mbar_wait(&ctrl->q_full[t], q_uses[t] & 1, abort_flag);
+          int g = it.ctile0 + wk.tile0;
+          const int g_end = it.ctile0 + j_end;
+          int pc = ok ? find_cache_block(p, it, g) : 0;
+          while (ok && g < g_end) {
+            const float2 *cs_row = p.q_rope + (size_t)pc * (D / 2);
+            for (int t = 0; t < it.n_qt; ++t) {
+              ok = mbar_wait(&ctrl->qr_empty[t], (n_rot[t] & 1) ^ 1, abort_flag);
+              if (!ok) break;
+              rotate_q_rows<D>(smem + (t ? L::kQ1 : L::kQ0), smem + L::kBg + t * L::kTileBytes, cs_row, p.rope_layout,
+                               bw * 64, bw * 64 + 64, lane);
+              fence_proxy_async();                     // the tensor core reads through the async proxy
+              __syncwarp();
+              if (lane == 0) mbar_arrive(&ctrl->qr_full[t]);
+              ++n_rot[t];
+            }
+            ++pc;
+            g = __ldg(p.seg.cache_tile_cu + pc);
+          }
+          if (!ok) break;
+        }
+        for (int t = 0; t < it.n_qt; ++t) ++q_uses[t];
+      }
+    } else if (p.bg.n_rows > 0) {
       // each spare warp runs the staged engine with its own two 16 KB stages; chunks are drawn from a
       // device-wide counter, so the job spreads over every CTA of the launch, early and late ones
       const int bw = warp - 10;
@@ -521,7 +674,7 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
         // visible columns of this tile for this row: 0 .. lim
         int lim;
         const int jt = tile0 + j;
-        if (jt < it.n_cache_tiles) lim = p.v_src_off ? ctrl->tile_valid[(tiles_before + j) & 7] - 1
+        if (jt < it.n_cache_tiles) lim = p.walk ? ctrl->tile_valid[(tiles_before + j) & 7] - 1
                                                      : it.cache_len - jt * kBlockN - 1;
         else lim = tok_c - (it.own_row0 + (jt - it.n_cache_tiles) * kBlockN);
         if (lim < kBlockN - 1) {
@@ -772,6 +925,12 @@ ba_status ba_attend_sm100_launch(ba_ctx *ctx, const ba_attend_args &a, const ba_
   p.scale_log2 = ctx->scale * 1.4426950408889634f;
   p.final_only = a.final_only;
   p.v_src_off = a.final_only ? a.v_src_off : nullptr;
+  p.fused = a.final_only && a.fused && a.n_cache_rows > 0;
+  p.k_src_off = p.fused ? a.k_src_off : nullptr;
+  p.walk = p.v_src_off != nullptr || p.fused;
+  p.rope_layout = ctx->cfg.rope_layout;
+  p.q_rope = p.fused ? reinterpret_cast<const float2 *>(seg->cache_rope) : nullptr;
+  if (p.fused && !p.q_rope) return BA_ERR_INVALID_ARG;
   p.n_q_rows = a.n_q_rows;
   p.seg = *seg;
   if (seg->q_tile_tokens != 2 * p.tok) return BA_ERR_INVALID_ARG;
@@ -822,7 +981,7 @@ ba_status ba_attend_sm100_launch(ba_ctx *ctx, const ba_attend_args &a, const ba_
   if (!make_map(&tk, a.k, D, Hkv, a.n_kv_rows, 1, kBlockN)) return BA_ERR_CUDA;
   if (!make_map(&tv, a.v, D, Hkv, a.n_kv_rows, 1, kBlockN)) return BA_ERR_CUDA;
   if (a.final_only && a.n_cache_rows > 0) {
-    if (!make_map(&tkc, a.k_cache, D, Hkv, a.n_cache_rows, 1, kBlockN)) return BA_ERR_CUDA;
+    if (!make_map(&tkc, a.k_cache, D, Hkv, p.fused ? a.n_k_rows : a.n_cache_rows, 1, kBlockN)) return BA_ERR_CUDA;
     if (!make_map(&tvc, a.v_cache, D, Hkv, a.v_src_off ? a.n_v_rows : a.n_cache_rows, 1, kBlockN)) return BA_ERR_CUDA;
   } else {
     tkc = tk; tvc = tv;
@@ -833,7 +992,7 @@ ba_status ba_attend_sm100_launch(ba_ctx *ctx, const ba_attend_args &a, const ba_
   p.bg.n_rows = 0; p.bg_counter = nullptr; p.bg_rows_per_chunk = 0;
   if (ctx->has_pending) {
     const int row_bytes = ctx->pending.row_vecs * 16;
-    if (row_bytes <= kBgStageBytes) {
+    if (row_bytes <= kBgStageBytes && !p.fused) {   // the fused path uses the staging area and the spare warps itself
       p.bg = ctx->pending;
       ctx->has_pending = 0;
       ctx->pending_table_bytes = 0;

@@ -94,6 +94,11 @@ struct ba_attend_args {
   const __nv_bfloat16 *k_cache, *v_cache;
   int32_t n_cache_rows, n_v_rows;
   const int32_t *v_src_off;
+  // fused warm path: k_cache holds the cached keys at cache-time positions (n_k_rows rows; block c
+  // at row k_src_off[c], or at its packed offset when k_src_off is null)
+  int fused;
+  const int32_t *k_src_off;
+  int32_t n_k_rows;
   int final_only;  // 1: ba_final_attend, 0: ba_block_prefill
 };
 

@@ -278,10 +278,12 @@ def test_prefill_full_causal_32k_sampled_rows():
 
 
 # --------------------------------------------------------------------------- warm path
-def run_warm(w, mode, out_dtype=B.BA_OUT_F32, layer=0, v_from_pool=True):
-    """ba_segment -> ba_reencode_k -> ba_final_attend, against oracle re-encode + final attend.
-    The oracle attends its own unrounded fp64 re-encoded keys."""
-    c = ctx_for(w)
+def run_warm(w, mode, out_dtype=B.BA_OUT_F32, layer=0, v_from_pool=True, fused=False,
+             layout=B.BA_ROPE_ADJACENT):
+    """ba_segment -> ba_reencode_k -> ba_final_attend (or ba_final_attend_fused on the keys as
+    cached), against oracle re-encode + final attend.  The oracle attends its own unrounded fp64
+    re-encoded keys."""
+    c = ctx_for(w, rope_layout=layout)
     seg, buf = c.segment(w.block_lens, w.seq_nblocks, mode)
     t = ob.segment_tables(w.block_lens, w.seq_nblocks, mode)
     x = W.warm_inputs(w, layer)
@@ -303,14 +305,21 @@ def run_warm(w, mode, out_dtype=B.BA_OUT_F32, layer=0, v_from_pool=True):
             v_cache, v_off, n_v = dev(x["v_pool"]), off, x["v_pool"].shape[0]
         else:
             v_cache, v_off, n_v = dev(W.f32_to_bf16_bits(v_np.astype(np.float32))), None, 0
-    B.ba_reencode_k(c.ctx, k_src, off, k_src.shape[0], k_re, seg.cache_cu, seg.cache_delta,
-                    seg.n_cached_blocks, Tc)
     o = torch.empty(Tf, w.n_q_heads, w.head_dim, device="cuda",
                     dtype=torch.float32 if out_dtype == B.BA_OUT_F32 else torch.bfloat16)
     lse = torch.empty(Tf, w.n_q_heads, dtype=torch.float32, device="cuda")
-    B.ba_final_attend(c.ctx, q_f, k_f, v_f, Tf, k_re, v_cache, Tc, v_off, n_v, o, lse, seg, mode, out_dtype)
+    if fused:
+        # keys and values are addressed alike: both from the pool, or both in cache packing
+        v_src = dev(x["v_pool"]) if w.pool_lens is not None else v_cache
+        B.ba_final_attend_fused(c.ctx, q_f, k_f, v_f, Tf, k_src, v_src, k_src.shape[0], off, Tc, o, lse, seg,
+                                mode, out_dtype)
+    else:
+        B.ba_reencode_k(c.ctx, k_src, off, k_src.shape[0], k_re, seg.cache_cu, seg.cache_delta,
+                        seg.n_cached_blocks, Tc)
+        B.ba_final_attend(c.ctx, q_f, k_f, v_f, Tf, k_re, v_cache, Tc, v_off, n_v, o, lse, seg, mode, out_dtype)
     assert c.device_status() == B.BA_OK
-    k_ref = ob.reencode_blocks(W.bf16_bits_to_f64(k_src_np), off_np, t["cache_cu"], t["cache_delta"], w.rope_theta)
+    k_ref = ob.reencode_blocks(W.bf16_bits_to_f64(k_src_np), off_np, t["cache_cu"], t["cache_delta"], w.rope_theta,
+                               layout)
     o_ref, lse_ref = ob.final_attend(W.bf16_bits_to_f64(x["q_f"]), W.bf16_bits_to_f64(x["k_f"]),
                                      W.bf16_bits_to_f64(x["v_f"]), k_ref, v_np, w.block_lens, w.seq_nblocks, mode)
     c.close()
@@ -352,6 +361,29 @@ def test_warm_path_32k_full_size():
     check_attention(o, round_bf16(o_ref), lse, lse_ref, rel=2e-2, bf16_store=True)
     o2, lse2, _, _ = run_warm(w, B.BA_MODE_BLOCK, B.BA_OUT_F32)
     check_attention(o2, o_ref, lse2, lse_ref)
+
+
+@pytest.mark.parametrize("w", WARM_CASES, ids=lambda w: w.name)
+@pytest.mark.parametrize("mode", [B.BA_MODE_BLOCK, B.BA_MODE_FULL])
+def test_fused_warm_path_parity(w, mode):
+    """Re-encoding applied to the query side inside the attention launch (keys as cached)."""
+    o, lse, o_ref, lse_ref = run_warm(w, mode, fused=True)
+    check_attention(o, o_ref, lse, lse_ref)
+
+
+@pytest.mark.parametrize("w", [W.config1(), W.config2(), W.config5(4, 64, 6, 32)], ids=lambda w: w.name)
+def test_fused_warm_path_half_layout(w):
+    o, lse, o_ref, lse_ref = run_warm(w, B.BA_MODE_BLOCK, fused=True, layout=B.BA_ROPE_HALF)
+    check_attention(o, o_ref, lse, lse_ref)
+
+
+def test_fused_warm_path_32k_full_size_and_pool_serving():
+    w = W.config3(1)
+    o, lse, o_ref, lse_ref = run_warm(w, B.BA_MODE_BLOCK, fused=True)
+    check_attention(o, o_ref, lse, lse_ref)
+    w5 = W.config5()
+    o, lse, o_ref, lse_ref = run_warm(w5, B.BA_MODE_BLOCK, fused=True)
+    check_attention(o, o_ref, lse, lse_ref)
 
 
 def test_attention_rejects_mode_mismatch_and_null():
