@@ -83,7 +83,12 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.ba_block_prefill.argtypes = [vp, vp, vp, vp, vp, vp, C.POINTER(ba_segments), C.c_int, C.c_int, vp]
     lib.ba_final_attend.argtypes = [vp, vp, vp, vp, i32, vp, vp, i32, vp, i32, vp, vp,
                                     C.POINTER(ba_segments), C.c_int, C.c_int, vp]
+    lib.ba_final_attend_fused.argtypes = [vp, vp, vp, vp, i32, vp, vp, i32, vp, i32, vp, vp,
+                                          C.POINTER(ba_segments), C.c_int, C.c_int, vp]
     for name in EXPORTS:
+        # without argtypes ctypes would pass addresses as 32-bit ints
+        if getattr(lib, name).argtypes is None:
+            raise RuntimeError(f"{name}: prototype not declared")
         if name not in ("ba_status_string", "ba_launch_count"):
             getattr(lib, name).restype = C.c_int
     _lib = lib
