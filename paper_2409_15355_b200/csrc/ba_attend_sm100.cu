@@ -289,42 +289,78 @@ __device__ __forceinline__ void rot_words_half(uint32_t &a, uint32_t &b, float2 
   a = *reinterpret_cast<uint32_t *>(&va);
   b = *reinterpret_cast<uint32_t *>(&vb);
 }
+// The lane's (cos, sin) values of one cached block: ADJACENT cs[4 c + i] = pair 32 c + 4 chunk + i of
+// region c; HALF cs[i] = pair 8 chunk + i.
 template <int D>
-__device__ __forceinline__ void rotate_q_rows(const uint8_t *src, uint8_t *dst, const float2 *cs_row, int layout,
-                                              int row_begin, int row_end, int lane) {
+__device__ __forceinline__ void load_q_rope(const float2 *cs_row, int layout, int lane, float2 (&cs)[8]) {
+  if (layout == BA_ROPE_ADJACENT) {
+    const int chunk = lane & 7;
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+      if (i < 4 * (D / 64)) cs[i] = __ldg(cs_row + (i >> 2) * 32 + chunk * 4 + (i & 3));
+  } else {
+    const int chunk = lane % ((D == 128) ? 8 : 4);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) cs[i] = __ldg(cs_row + chunk * 8 + i);
+  }
+}
+// Rows are taken four at a time, all loads first, so that one warp keeps several shared-memory
+// accesses in flight.
+template <int D>
+__device__ __forceinline__ void rotate_q_rows(const uint8_t *__restrict__ src, uint8_t *__restrict__ dst,
+                                              const float2 (&cs)[8], int layout, int row_begin, int row_end, int lane) {
   constexpr int kRegion = 128 * 128;
   if (layout == BA_ROPE_ADJACENT) {
     const int chunk = lane & 7;
 #pragma unroll
     for (int c = 0; c < D / 64; ++c) {
-      float2 cs[4];
+#pragma unroll 1
+      for (int row0 = row_begin + (lane >> 3); row0 < row_end; row0 += 16) {
+        uint4 v[4];
+        int off[4];
 #pragma unroll
-      for (int i = 0; i < 4; ++i) cs[i] = __ldg(cs_row + c * 32 + chunk * 4 + i);
-      for (int row = row_begin + (lane >> 3); row < row_end; row += 4) {
-        const int off = c * kRegion + row * 128 + ((chunk ^ (row & 7)) << 4);
-        uint4 v = *reinterpret_cast<const uint4 *>(src + off);
-        v.x = rot_word_adjacent(v.x, cs[0]); v.y = rot_word_adjacent(v.y, cs[1]);
-        v.z = rot_word_adjacent(v.z, cs[2]); v.w = rot_word_adjacent(v.w, cs[3]);
-        *reinterpret_cast<uint4 *>(dst + off) = v;
+        for (int u = 0; u < 4; ++u) {
+          const int row = row0 + 4 * u;
+          off[u] = c * kRegion + row * 128 + ((chunk ^ (row & 7)) << 4);
+          v[u] = *reinterpret_cast<const uint4 *>(src + off[u]);
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          v[u].x = rot_word_adjacent(v[u].x, cs[4 * c + 0]); v[u].y = rot_word_adjacent(v[u].y, cs[4 * c + 1]);
+          v[u].z = rot_word_adjacent(v[u].z, cs[4 * c + 2]); v[u].w = rot_word_adjacent(v[u].w, cs[4 * c + 3]);
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) *reinterpret_cast<uint4 *>(dst + off[u]) = v[u];
       }
     }
   } else {
     // pairs (m, m + D/2): D = 128 pairs chunk c of region 0 with chunk c of region 1;
     // D = 64 pairs chunk c (< 4) with chunk c + 4 of the only region
     constexpr int kCols = (D == 128) ? 8 : 4;        // chunk columns holding x
+    constexpr int kStep = 32 / kCols;                // rows covered by one pass of the warp
     const int chunk = lane % kCols;
-    float2 cs[8];
+#pragma unroll 1
+    for (int row0 = row_begin + lane / kCols; row0 < row_end; row0 += 2 * kStep) {
+      uint4 a[2], b[2];
+      int off_x[2], off_y[2];
 #pragma unroll
-    for (int i = 0; i < 8; ++i) cs[i] = __ldg(cs_row + chunk * 8 + i);
-    for (int row = row_begin + lane / kCols; row < row_end; row += 32 / kCols) {
-      const int off_x = row * 128 + ((chunk ^ (row & 7)) << 4);
-      const int off_y = (D == 128) ? off_x + kRegion : row * 128 + (((chunk + 4) ^ (row & 7)) << 4);
-      uint4 a = *reinterpret_cast<const uint4 *>(src + off_x);
-      uint4 b = *reinterpret_cast<const uint4 *>(src + off_y);
-      rot_words_half(a.x, b.x, cs[0], cs[1]); rot_words_half(a.y, b.y, cs[2], cs[3]);
-      rot_words_half(a.z, b.z, cs[4], cs[5]); rot_words_half(a.w, b.w, cs[6], cs[7]);
-      *reinterpret_cast<uint4 *>(dst + off_x) = a;
-      *reinterpret_cast<uint4 *>(dst + off_y) = b;
+      for (int u = 0; u < 2; ++u) {
+        const int row = row0 + kStep * u;
+        off_x[u] = row * 128 + ((chunk ^ (row & 7)) << 4);
+        off_y[u] = (D == 128) ? off_x[u] + kRegion : row * 128 + (((chunk + 4) ^ (row & 7)) << 4);
+        a[u] = *reinterpret_cast<const uint4 *>(src + off_x[u]);
+        b[u] = *reinterpret_cast<const uint4 *>(src + off_y[u]);
+      }
+#pragma unroll
+      for (int u = 0; u < 2; ++u) {
+        rot_words_half(a[u].x, b[u].x, cs[0], cs[1]); rot_words_half(a[u].y, b[u].y, cs[2], cs[3]);
+        rot_words_half(a[u].z, b[u].z, cs[4], cs[5]); rot_words_half(a[u].w, b[u].w, cs[6], cs[7]);
+      }
+#pragma unroll
+      for (int u = 0; u < 2; ++u) {
+        *reinterpret_cast<uint4 *>(dst + off_x[u]) = a[u];
+        *reinterpret_cast<uint4 *>(dst + off_y[u]) = b[u];
+      }
     }
   }
 }
@@ -597,11 +633,12 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
           const int g_end = it.ctile0 + j_end;
           int pc = ok ? find_cache_block(p, it, g) : 0;
           while (ok && g < g_end) {
-            const float2 *cs_row = p.q_rope + (size_t)pc * (D / 2);
+            float2 cs[8];                               // fetched before the wait: they depend on the block only
+            load_q_rope<D>(p.q_rope + (size_t)pc * (D / 2), p.rope_layout, lane, cs);
             for (int t = 0; t < it.n_qt; ++t) {
               ok = mbar_wait(&ctrl->qr_empty[t], (n_rot[t] & 1) ^ 1, abort_flag);
               if (!ok) break;
-              rotate_q_rows<D>(smem + (t ? L::kQ1 : L::kQ0), smem + L::kBg + t * L::kTileBytes, cs_row, p.rope_layout,
+              rotate_q_rows<D>(smem + (t ? L::kQ1 : L::kQ0), smem + L::kBg + t * L::kTileBytes, cs, p.rope_layout,
                                bw * 64, bw * 64 + 64, lane);
               fence_proxy_async();                     // the tensor core reads through the async proxy
               __syncwarp();
