@@ -24,9 +24,10 @@
 // Fused warm path (Section 2.5 steps 2 and 3 in one launch): the cached keys stay at their
 // cache-time positions and the position difference of each block (Eq. 3 after Eq. 2) is applied
 // to the other side of the dot product, (R(p) q) . (R(delta + t) k) = (R(-delta) R(p) q) . (R(t) k):
-// warps 10-11 counter-rotate the two query tiles once per cached block into a second pair of
-// buffers, which the QK^T products of that block's key tiles read.  The cached keys are then
-// never rewritten or re-read, and a key tile never spans two blocks.
+// each softmax thread counter-rotates its own row of its query tile once per cached block into a
+// second pair of buffers, which the QK^T products of that block's key tiles read; it does so
+// right after handing over P of the block's last tile, while it would otherwise wait for the next
+// S.  The cached keys are then never rewritten or re-read, and a key tile never spans two blocks.
 #include <math.h>
 #include <type_traits>
 
@@ -38,7 +39,7 @@ using namespace sm100;
 
 // Optional phase timeline of CTA (0,0,0) for tuning: compile with -DBA_TRACE.
 #ifdef BA_TRACE
-__device__ long long g_ba_trace[4][64][8];
+__device__ long long g_ba_trace[6][64][8];
 extern "C" int ba_trace_read(long long *dst) { return (int)cudaMemcpyFromSymbol(dst, g_ba_trace, sizeof(g_ba_trace)); }
 #define BA_TR(role, tile, k)                                                                  \
   do {                                                                                        \
@@ -119,8 +120,7 @@ struct Ctrl {
   uint64_t p_full[2][2];          // [query tile][half of the P tile]
   uint64_t o_done[2];
   uint64_t o_free[2];             // the softmax warps have read O_t out of tensor memory
-  uint64_t qr_full[2];            // fused: counter-rotated query tile t is ready for the current cached block
-  uint64_t qr_empty[2];           // fused: every QK^T reading it has completed
+  uint64_t qr_full[2];            // fused: counter-rotated query tile t is ready for the next cached block
   uint64_t work_full[kWorkSlots];  // work entry published by the scheduler (producer thread)
   uint64_t work_empty[kWorkSlots]; // entry read by the MMA thread and the 8 softmax warps
   int work_ring[kWorkSlots];
@@ -289,78 +289,46 @@ __device__ __forceinline__ void rot_words_half(uint32_t &a, uint32_t &b, float2 
   a = *reinterpret_cast<uint32_t *>(&va);
   b = *reinterpret_cast<uint32_t *>(&vb);
 }
-// The lane's (cos, sin) values of one cached block: ADJACENT cs[4 c + i] = pair 32 c + 4 chunk + i of
-// region c; HALF cs[i] = pair 8 chunk + i.
+// One thread rotates one row of a query tile (row r = TMEM lane r = the row whose softmax the
+// thread computes); the (cos, sin) values are the same for every row, so the loads are warp-wide
+// broadcasts served by L1.
 template <int D>
-__device__ __forceinline__ void load_q_rope(const float2 *cs_row, int layout, int lane, float2 (&cs)[8]) {
-  if (layout == BA_ROPE_ADJACENT) {
-    const int chunk = lane & 7;
-#pragma unroll
-    for (int i = 0; i < 8; ++i)
-      if (i < 4 * (D / 64)) cs[i] = __ldg(cs_row + (i >> 2) * 32 + chunk * 4 + (i & 3));
-  } else {
-    const int chunk = lane % ((D == 128) ? 8 : 4);
-#pragma unroll
-    for (int i = 0; i < 8; ++i) cs[i] = __ldg(cs_row + chunk * 8 + i);
-  }
-}
-// Rows are taken four at a time, all loads first, so that one warp keeps several shared-memory
-// accesses in flight.
-template <int D>
-__device__ __forceinline__ void rotate_q_rows(const uint8_t *__restrict__ src, uint8_t *__restrict__ dst,
-                                              const float2 (&cs)[8], int layout, int row_begin, int row_end, int lane) {
+__device__ __forceinline__ void rotate_q_row(const uint8_t *__restrict__ src, uint8_t *__restrict__ dst,
+                                             const float2 *__restrict__ cs_row, int layout, int r) {
   constexpr int kRegion = 128 * 128;
+  const int rb = r * 128, sw = r & 7;
   if (layout == BA_ROPE_ADJACENT) {
-    const int chunk = lane & 7;
 #pragma unroll
     for (int c = 0; c < D / 64; ++c) {
-#pragma unroll 1
-      for (int row0 = row_begin + (lane >> 3); row0 < row_end; row0 += 16) {
-        uint4 v[4];
-        int off[4];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
-          const int row = row0 + 4 * u;
-          off[u] = c * kRegion + row * 128 + ((chunk ^ (row & 7)) << 4);
-          v[u] = *reinterpret_cast<const uint4 *>(src + off[u]);
-        }
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-          v[u].x = rot_word_adjacent(v[u].x, cs[4 * c + 0]); v[u].y = rot_word_adjacent(v[u].y, cs[4 * c + 1]);
-          v[u].z = rot_word_adjacent(v[u].z, cs[4 * c + 2]); v[u].w = rot_word_adjacent(v[u].w, cs[4 * c + 3]);
-        }
-#pragma unroll
-        for (int u = 0; u < 4; ++u) *reinterpret_cast<uint4 *>(dst + off[u]) = v[u];
+      for (int ch = 0; ch < 8; ++ch) {
+        const int off = c * kRegion + rb + ((ch ^ sw) << 4);
+        uint4 v = *reinterpret_cast<const uint4 *>(src + off);
+        const float4 c01 = __ldg(reinterpret_cast<const float4 *>(cs_row + c * 32 + ch * 4));
+        const float4 c23 = __ldg(reinterpret_cast<const float4 *>(cs_row + c * 32 + ch * 4 + 2));
+        v.x = rot_word_adjacent(v.x, make_float2(c01.x, c01.y)); v.y = rot_word_adjacent(v.y, make_float2(c01.z, c01.w));
+        v.z = rot_word_adjacent(v.z, make_float2(c23.x, c23.y)); v.w = rot_word_adjacent(v.w, make_float2(c23.z, c23.w));
+        *reinterpret_cast<uint4 *>(dst + off) = v;
       }
     }
   } else {
-    // pairs (m, m + D/2): D = 128 pairs chunk c of region 0 with chunk c of region 1;
-    // D = 64 pairs chunk c (< 4) with chunk c + 4 of the only region
-    constexpr int kCols = (D == 128) ? 8 : 4;        // chunk columns holding x
-    constexpr int kStep = 32 / kCols;                // rows covered by one pass of the warp
-    const int chunk = lane % kCols;
-#pragma unroll 1
-    for (int row0 = row_begin + lane / kCols; row0 < row_end; row0 += 2 * kStep) {
-      uint4 a[2], b[2];
-      int off_x[2], off_y[2];
+    // pairs (m, m + D/2): D = 128 pairs chunk ch of region 0 with chunk ch of region 1;
+    // D = 64 pairs chunk ch (< 4) with chunk ch + 4 of the only region
+    constexpr int kCols = (D == 128) ? 8 : 4;
 #pragma unroll
-      for (int u = 0; u < 2; ++u) {
-        const int row = row0 + kStep * u;
-        off_x[u] = row * 128 + ((chunk ^ (row & 7)) << 4);
-        off_y[u] = (D == 128) ? off_x[u] + kRegion : row * 128 + (((chunk + 4) ^ (row & 7)) << 4);
-        a[u] = *reinterpret_cast<const uint4 *>(src + off_x[u]);
-        b[u] = *reinterpret_cast<const uint4 *>(src + off_y[u]);
-      }
-#pragma unroll
-      for (int u = 0; u < 2; ++u) {
-        rot_words_half(a[u].x, b[u].x, cs[0], cs[1]); rot_words_half(a[u].y, b[u].y, cs[2], cs[3]);
-        rot_words_half(a[u].z, b[u].z, cs[4], cs[5]); rot_words_half(a[u].w, b[u].w, cs[6], cs[7]);
-      }
-#pragma unroll
-      for (int u = 0; u < 2; ++u) {
-        *reinterpret_cast<uint4 *>(dst + off_x[u]) = a[u];
-        *reinterpret_cast<uint4 *>(dst + off_y[u]) = b[u];
-      }
+    for (int ch = 0; ch < kCols; ++ch) {
+      const int off_x = rb + ((ch ^ sw) << 4);
+      const int off_y = (D == 128) ? off_x + kRegion : rb + (((ch + 4) ^ sw) << 4);
+      uint4 a = *reinterpret_cast<const uint4 *>(src + off_x);
+      uint4 b = *reinterpret_cast<const uint4 *>(src + off_y);
+      const float4 *cp = reinterpret_cast<const float4 *>(cs_row + ch * 8);
+      const float4 c01 = __ldg(cp), c23 = __ldg(cp + 1), c45 = __ldg(cp + 2), c67 = __ldg(cp + 3);
+      rot_words_half(a.x, b.x, make_float2(c01.x, c01.y), make_float2(c01.z, c01.w));
+      rot_words_half(a.y, b.y, make_float2(c23.x, c23.y), make_float2(c23.z, c23.w));
+      rot_words_half(a.z, b.z, make_float2(c45.x, c45.y), make_float2(c45.z, c45.w));
+      rot_words_half(a.w, b.w, make_float2(c67.x, c67.y), make_float2(c67.z, c67.w));
+      *reinterpret_cast<uint4 *>(dst + off_x) = a;
+      *reinterpret_cast<uint4 *>(dst + off_y) = b;
     }
   }
 }
@@ -385,10 +353,9 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
     for (int t = 0; t < 2; ++t) {
       mbar_init(&ctrl->s_full[t], 1); mbar_init(&ctrl->p_full[t][0], 128); mbar_init(&ctrl->p_full[t][1], 128);
       mbar_init(&ctrl->o_done[t], 1); mbar_init(&ctrl->o_free[t], 128);
-      mbar_init(&ctrl->qr_full[t], 2); mbar_init(&ctrl->qr_empty[t], 1);
+      mbar_init(&ctrl->qr_full[t], 4);
     }
-    // an entry is read by the MMA thread and the 8 softmax warps, on the fused path also by warps 10-11
-    for (int k = 0; k < kWorkSlots; ++k) { mbar_init(&ctrl->work_full[k], 1); mbar_init(&ctrl->work_empty[k], p.fused ? 11 : 9); }
+    for (int k = 0; k < kWorkSlots; ++k) { mbar_init(&ctrl->work_full[k], 1); mbar_init(&ctrl->work_empty[k], 9); }
     ctrl->abort_flag = 0;
     fence_barrier_init();
   }
@@ -519,29 +486,33 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
       int p_uses[2] = {0, 0};              // P tiles of query tile t consumed
       Work wk = {};
       int n_work = 0;
+      // Every loop over the query tile t below is unrolled, so that t is a constant and the small
+      // per-tile arrays live in registers: this thread's issue latency is on the critical path.
       // fused path: the QK^T of a cached key tile reads the query tile counter-rotated for that tile's
-      // block; warps 10-11 rotate once per (block, query tile) and the two sides count those alike
+      // block; the softmax warps rotate once per (block, query tile) and both sides count those alike
       const uint64_t qr_desc[2] = {make_smem_desc(smem_u32(smem + L::kBg), 16, 1024),
                                    make_smem_desc(smem_u32(smem + L::kBg + L::kTileBytes), 16, 1024)};
       int n_rot[2] = {0, 0};               // rotations of query tile t consumed so far
-      int rot_block[2] = {-1, -1};         // cached block the rotated tile t currently belongs to
-      int walk_pc = -1, walk_end = 0;      // block of the current cached tile and the tile index where it ends
+      int rot_end[2] = {-1, -1};           // the rotated tile t is valid for cached key tiles below this index
+      int walk_pc = 0, walk_end = -1;      // block of the current cached tile and the tile index where it ends
+      int cached_end = 0;                  // tiles [tile0, cached_end) of the entry are cached keys
       // S_t = Q_t K^T for tile `jrel` of the entry, whose keys sit at ring position idx
       auto issue_qk = [&](int t, int jrel, int idx) -> bool {
         const int jt = wk.tile0 + jrel;
-        if (!p.fused || jt >= wk.it.n_cache_tiles) { issue_qk_with(t, idx, q_desc[t]); return true; }
+        if (!p.fused || jt >= cached_end) { issue_qk_with(t, idx, q_desc[t]); return true; }
         const int g = wk.it.ctile0 + jt;
-        if (walk_pc < 0) { walk_pc = find_cache_block(p, wk.it, g); walk_end = __ldg(p.seg.cache_tile_cu + walk_pc + 1); }
-        while (g >= walk_end) { ++walk_pc; walk_end = __ldg(p.seg.cache_tile_cu + walk_pc + 1); }
-        if (rot_block[t] != walk_pc) {
+        if (g >= rot_end[t]) {
+          // first key tile of another cached block: take the tile rotated for it
+          if (walk_end < 0) { walk_pc = find_cache_block(p, wk.it, g); walk_end = __ldg(p.seg.cache_tile_cu + walk_pc + 1); }
+          while (g >= walk_end) { ++walk_pc; walk_end = __ldg(p.seg.cache_tile_cu + walk_pc + 1); }
+          BA_TR(5, n_rot[t], t * 2);
           if (!mbar_wait(&ctrl->qr_full[t], n_rot[t] & 1, abort_flag)) return false;
+          BA_TR(5, n_rot[t], t * 2 + 1);
           ++n_rot[t];
-          rot_block[t] = walk_pc;
+          rot_end[t] = walk_end;
           tc_fence_after();
         }
         issue_qk_with(t, idx, qr_desc[t]);
-        // last key tile of this block within the entry: the rotated tile may be overwritten afterwards
-        if (g + 1 == walk_end || jt + 1 == min(wk.tile0 + wk.n_tiles, wk.it.n_cache_tiles)) mma_commit(&ctrl->qr_empty[t]);
         return true;
       };
       for (;;) {
@@ -554,12 +525,17 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
         mbar_arrive(&ctrl->work_empty[slot]);          // the entry has been decoded into registers
         const int n_tiles = wk.n_tiles, n_qt = wk.it.n_qt;
         if (n_tiles == 0) continue;
-        walk_pc = -1; rot_block[0] = rot_block[1] = -1;
-        for (int t = 0; t < n_qt && ok; ++t) ok = mbar_wait(&ctrl->q_full[t], q_uses[t] & 1, abort_flag);
+        walk_end = -1; rot_end[0] = rot_end[1] = -1;
+        cached_end = min(wk.tile0 + n_tiles, wk.it.n_cache_tiles);
+#pragma unroll
+        for (int t = 0; t < 2; ++t)
+          if (t < n_qt && ok) ok = mbar_wait(&ctrl->q_full[t], q_uses[t] & 1, abort_flag);
         if (ok) ok = wait_kv(gidx);
         if (!ok) break;
         tc_fence_after();
-        for (int t = 0; t < n_qt && ok; ++t) ok = issue_qk(t, 0, gidx);
+#pragma unroll
+        for (int t = 0; t < 2; ++t)
+          if (t < n_qt && ok) ok = issue_qk(t, 0, gidx);
         if (!ok) break;
         mma_commit(&ctrl->kv_empty[gidx % kStages]);
         if (n_tiles == 1) mma_commit(&ctrl->q_empty);
@@ -569,20 +545,22 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
           BA_TR(3, j, 0);
           ok = wait_kv(iv);
           BA_TR(3, j, 1);
-          for (int t = 0; t < n_qt && ok; ++t) {
+#pragma unroll
+          for (int t = 0; t < 2; ++t) {
+            if (t >= n_qt || !ok) continue;
             BA_TR(2, j, t * 4 + 0);
             // the first PV of an item overwrites O_t: the previous item's rows must have been read out
-            if (j == 0) { ok = mbar_wait(&ctrl->o_free[t], (q_uses[t] & 1) ^ 1, abort_flag); if (!ok) break; }
+            if (j == 0) { ok = mbar_wait(&ctrl->o_free[t], (q_uses[t] & 1) ^ 1, abort_flag); if (!ok) continue; }
             ok = mbar_wait(&ctrl->p_full[t][0], p_uses[t] & 1, abort_flag);
-            if (!ok) break;
+            if (!ok) continue;
             tc_fence_after();
             BA_TR(2, j, t * 4 + 1);
             issue_pv(t, iv, j == 0, 0);
             // K_(j+1) is needed right after the second half of PV: make sure of it while P is still
             // being finished, off the critical path
-            if (t == 0 && !last) { BA_TR(3, j, 2); ok = wait_kv(ik); if (!ok) break; BA_TR(3, j, 3); }
+            if (t == 0 && !last) { BA_TR(3, j, 2); ok = wait_kv(ik); if (!ok) continue; BA_TR(3, j, 3); }
             ok = mbar_wait(&ctrl->p_full[t][1], p_uses[t] & 1, abort_flag);
-            if (!ok) break;
+            if (!ok) continue;
             tc_fence_after();
             issue_pv(t, iv, j == 0, 1);
             ++p_uses[t];
@@ -591,7 +569,7 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
             if (t + 1 == n_qt) mma_commit(&ctrl->kv_empty[iv % kStages]);
             if (!last) {
               ok = issue_qk(t, j + 1, ik);
-              if (!ok) break;
+              if (!ok) continue;
               BA_TR(2, j, t * 4 + 3);
               if (t + 1 == n_qt) {
                 mma_commit(&ctrl->kv_empty[ik % kStages]);
@@ -601,58 +579,15 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
           }
         }
         gidx += 2 * n_tiles;
-        for (int t = 0; t < n_qt; ++t) ++q_uses[t];
+#pragma unroll
+        for (int t = 0; t < 2; ++t)
+          if (t < n_qt) ++q_uses[t];
       }
     }
   } else if (warp >= 10) {
     // ------------------------------------------------------------ spare warps: background re-encoding
     asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(BA_SVC_REGS));
-    if (p.fused) {
-      // fused warm path: counter-rotate the query tiles for each cached block of each work entry
-      // (warp 10 rows 0-63, warp 11 rows 64-127 of a tile)
-      const int bw = warp - 10, lane = tid & 31;
-      int n_rot[2] = {0, 0}, q_uses[2] = {0, 0};
-      bool ok = true;
-      Work wk;
-      int n_work = 0;
-      for (;;) {
-        const int slot = n_work & (kWorkSlots - 1);
-        ok = mbar_wait(&ctrl->work_full[slot], (n_work / kWorkSlots) & 1, abort_flag);
-        if (!ok) break;
-        const int w = ctrl->work_ring[slot];
-        ++n_work;
-        if (w < 0 || !next_work(p, w, wk)) break;
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&ctrl->work_empty[slot]);
-        if (wk.n_tiles == 0) continue;
-        const Item &it = wk.it;
-        const int j_end = min(wk.tile0 + wk.n_tiles, it.n_cache_tiles);
-        if (wk.tile0 < j_end) {
-          for (int t = 0; t < it.n_qt && ok; ++t) ok = mbar_wait(&ctrl->q_full[t], q_uses[t] & 1, abort_flag);
-          int g = it.ctile0 + wk.tile0;
-          const int g_end = it.ctile0 + j_end;
-          int pc = ok ? find_cache_block(p, it, g) : 0;
-          while (ok && g < g_end) {
-            float2 cs[8];                               // fetched before the wait: they depend on the block only
-            load_q_rope<D>(p.q_rope + (size_t)pc * (D / 2), p.rope_layout, lane, cs);
-            for (int t = 0; t < it.n_qt; ++t) {
-              ok = mbar_wait(&ctrl->qr_empty[t], (n_rot[t] & 1) ^ 1, abort_flag);
-              if (!ok) break;
-              rotate_q_rows<D>(smem + (t ? L::kQ1 : L::kQ0), smem + L::kBg + t * L::kTileBytes, cs, p.rope_layout,
-                               bw * 64, bw * 64 + 64, lane);
-              fence_proxy_async();                     // the tensor core reads through the async proxy
-              __syncwarp();
-              if (lane == 0) mbar_arrive(&ctrl->qr_full[t]);
-              ++n_rot[t];
-            }
-            ++pc;
-            g = __ldg(p.seg.cache_tile_cu + pc);
-          }
-          if (!ok) break;
-        }
-        for (int t = 0; t < it.n_qt; ++t) ++q_uses[t];
-      }
-    } else if (p.bg.n_rows > 0) {
+    if (p.bg.n_rows > 0) {
       // each spare warp runs the staged engine with its own two 16 KB stages; chunks are drawn from a
       // device-wide counter, so the job spreads over every CTA of the launch, early and late ones
       const int bw = warp - 10;
@@ -695,6 +630,25 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
       const int tok_c = min(row_tok, q_last);               // rows past the block behave like its last row
       const int head = head0 + (r & (p.hpt - 1));
       float m_used = -INFINITY, l = 0.f;
+
+      // fused path: this thread counter-rotates row r of query tile t for each cached block of the
+      // entry, first before the entry's first tile, then each time the block's last tile is done
+      const int cached_end = min(tile0 + n_tiles, it.n_cache_tiles);   // tiles [tile0, cached_end) are cached keys
+      int f_pc = 0, f_end = 0;                                         // current cached block and the tile index where it ends
+      auto rotate_for = [&](int pc) {
+        rotate_q_row<D>(smem + (t ? L::kQ1 : L::kQ0), smem + L::kBg + t * L::kTileBytes,
+                        p.q_rope + (size_t)pc * (D / 2), p.rope_layout, r);
+        fence_proxy_async();                               // the tensor core reads through the async proxy
+        __syncwarp();
+        if ((tid & 31) == 0) mbar_arrive(&ctrl->qr_full[t]);
+      };
+      if (p.fused && tile0 < cached_end) {
+        ok = mbar_wait(&ctrl->q_full[t], o_uses & 1, abort_flag);      // the query tile has landed
+        if (!ok) break;
+        f_pc = find_cache_block(p, it, it.ctile0 + tile0);
+        f_end = __ldg(p.seg.cache_tile_cu + f_pc + 1);
+        rotate_for(f_pc);
+      }
 
       for (int j = 0; j < n_tiles; ++j) {
         if (r == 0) BA_TR(t, j, 0);
@@ -788,6 +742,14 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
         };
         if (kPolyPeriod > 0 && __all_sync(0xffffffffu, lim >= kBlockN - 1)) exp_halves(std::true_type{});
         else exp_halves(std::false_type{});
+        // the next tile belongs to another cached block: its rotated queries are due now, while the
+        // tensor core works on PV of this tile (the QK^T that read the old rotation completed
+        // before this tile's S arrived)
+        if (p.fused && tile0 + j + 1 < cached_end && it.ctile0 + tile0 + j + 1 >= f_end) {
+          ++f_pc;
+          f_end = __ldg(p.seg.cache_tile_cu + f_pc + 1);
+          rotate_for(f_pc);
+        }
         float sum[8];
 #pragma unroll
         for (int i = 0; i < 4; ++i) unpack2(sum2[i], sum[2 * i], sum[2 * i + 1]);

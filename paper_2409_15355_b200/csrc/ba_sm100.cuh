@@ -53,6 +53,20 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
   return ok != 0;
 }
 
+// The same with a suspend-time hint: the thread may be parked by the hardware for up to `ns`
+// nanoseconds and resumes as soon as the phase completes.
+__device__ __forceinline__ bool mbar_try_wait_hint(uint64_t *bar, uint32_t parity, uint32_t ns) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}\n"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity), "r"(ns)
+      : "memory");
+  return ok != 0;
+}
+
 // Bounded wait.  Gives up after about one second (kWaitLimitNs on the global nanosecond timer)
 // or as soon as another thread of the CTA has raised *abort_flag (a shared-memory word); the
 // caller then leaves its role loop.  A wait that gives up raises the flag itself.  Legitimate
@@ -60,6 +74,9 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
 constexpr unsigned long long kWaitLimitNs = 1000000000ull;
 #ifndef BA_FAST_POLLS
 #define BA_FAST_POLLS 64      // polls before the slow path (timer, abort flag, back-off)
+#endif
+#ifndef BA_WAIT_HINT_NS
+#define BA_WAIT_HINT_NS 0     // > 0: the slow path parks the thread with this suspend-time hint instead of sleeping
 #endif
 #ifndef BA_SLEEP_NS
 #define BA_SLEEP_NS 32        // back-off between polls on the slow path
@@ -76,10 +93,16 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volati
   const unsigned long long t0 = global_ns();
 #pragma unroll 1
   for (uint32_t it = 0;; ++it) {
+#if BA_WAIT_HINT_NS > 0
+    if (mbar_try_wait_hint(bar, parity, BA_WAIT_HINT_NS)) return true;
+#else
     if (mbar_try_wait(bar, parity)) return true;
+#endif
     if (*abort_flag) return false;
     if (global_ns() - t0 > kWaitLimitNs) break;
+#if BA_WAIT_HINT_NS == 0
     if (BA_SLEEP_NS > 0) __nanosleep(it > 4096 ? 256 : BA_SLEEP_NS);
+#endif
   }
   *abort_flag = 1;
   return false;
