@@ -121,6 +121,7 @@ struct Ctrl {
   uint64_t o_done[2];
   uint64_t o_free[2];             // the softmax warps have read O_t out of tensor memory
   uint64_t qr_full[2];            // fused: counter-rotated query tile t is ready for the next cached block
+  uint64_t cs_full[2];            // fused: the block's (cos, sin) row has been staged for softmax group t
   uint64_t work_full[kWorkSlots];  // work entry published by the scheduler (producer thread)
   uint64_t work_empty[kWorkSlots]; // entry read by the MMA thread and the 8 softmax warps
   int work_ring[kWorkSlots];
@@ -290,47 +291,45 @@ __device__ __forceinline__ void rot_words_half(uint32_t &a, uint32_t &b, float2 
   b = *reinterpret_cast<uint32_t *>(&vb);
 }
 // One thread rotates one row of a query tile (row r = TMEM lane r = the row whose softmax the
-// thread computes); the (cos, sin) values are the same for every row, so the loads are warp-wide
-// broadcasts served by L1.
+// thread computes).  The (cos, sin) values of the block are the same for every row: `cs` points
+// to a copy of them in shared memory, read as warp-wide broadcasts.  The row is loaded in full
+// before the arithmetic starts, so that the shared-memory latency is paid once.
 template <int D>
 __device__ __forceinline__ void rotate_q_row(const uint8_t *__restrict__ src, uint8_t *__restrict__ dst,
-                                             const float2 *__restrict__ cs_row, int layout, int r) {
+                                             const float2 *__restrict__ cs, int layout, int r) {
   constexpr int kRegion = 128 * 128;
+  constexpr int kVec = D / 8;                      // 16-byte chunks per row
   const int rb = r * 128, sw = r & 7;
+  uint4 v[kVec];
+  int off[kVec];
+#pragma unroll
+  for (int i = 0; i < kVec; ++i) {
+    off[i] = (i >> 3) * kRegion + rb + (((i & 7) ^ sw) << 4);     // chunk i of the row: columns 8 i .. 8 i + 7
+    v[i] = *reinterpret_cast<const uint4 *>(src + off[i]);
+  }
   if (layout == BA_ROPE_ADJACENT) {
 #pragma unroll
-    for (int c = 0; c < D / 64; ++c) {
-#pragma unroll
-      for (int ch = 0; ch < 8; ++ch) {
-        const int off = c * kRegion + rb + ((ch ^ sw) << 4);
-        uint4 v = *reinterpret_cast<const uint4 *>(src + off);
-        const float4 c01 = __ldg(reinterpret_cast<const float4 *>(cs_row + c * 32 + ch * 4));
-        const float4 c23 = __ldg(reinterpret_cast<const float4 *>(cs_row + c * 32 + ch * 4 + 2));
-        v.x = rot_word_adjacent(v.x, make_float2(c01.x, c01.y)); v.y = rot_word_adjacent(v.y, make_float2(c01.z, c01.w));
-        v.z = rot_word_adjacent(v.z, make_float2(c23.x, c23.y)); v.w = rot_word_adjacent(v.w, make_float2(c23.z, c23.w));
-        *reinterpret_cast<uint4 *>(dst + off) = v;
-      }
+    for (int i = 0; i < kVec; ++i) {
+      const float4 c01 = *reinterpret_cast<const float4 *>(cs + i * 4);
+      const float4 c23 = *reinterpret_cast<const float4 *>(cs + i * 4 + 2);
+      v[i].x = rot_word_adjacent(v[i].x, make_float2(c01.x, c01.y)); v[i].y = rot_word_adjacent(v[i].y, make_float2(c01.z, c01.w));
+      v[i].z = rot_word_adjacent(v[i].z, make_float2(c23.x, c23.y)); v[i].w = rot_word_adjacent(v[i].w, make_float2(c23.z, c23.w));
     }
   } else {
-    // pairs (m, m + D/2): D = 128 pairs chunk ch of region 0 with chunk ch of region 1;
-    // D = 64 pairs chunk ch (< 4) with chunk ch + 4 of the only region
-    constexpr int kCols = (D == 128) ? 8 : 4;
+    // pairs (m, m + D/2): chunk i (< kVec / 2) holds x of pairs 8 i .. 8 i + 7, chunk i + kVec / 2 their partners
 #pragma unroll
-    for (int ch = 0; ch < kCols; ++ch) {
-      const int off_x = rb + ((ch ^ sw) << 4);
-      const int off_y = (D == 128) ? off_x + kRegion : rb + (((ch + 4) ^ sw) << 4);
-      uint4 a = *reinterpret_cast<const uint4 *>(src + off_x);
-      uint4 b = *reinterpret_cast<const uint4 *>(src + off_y);
-      const float4 *cp = reinterpret_cast<const float4 *>(cs_row + ch * 8);
-      const float4 c01 = __ldg(cp), c23 = __ldg(cp + 1), c45 = __ldg(cp + 2), c67 = __ldg(cp + 3);
+    for (int i = 0; i < kVec / 2; ++i) {
+      const float4 *cp = reinterpret_cast<const float4 *>(cs + i * 8);
+      const float4 c01 = cp[0], c23 = cp[1], c45 = cp[2], c67 = cp[3];
+      uint4 &a = v[i], &b = v[i + kVec / 2];
       rot_words_half(a.x, b.x, make_float2(c01.x, c01.y), make_float2(c01.z, c01.w));
       rot_words_half(a.y, b.y, make_float2(c23.x, c23.y), make_float2(c23.z, c23.w));
       rot_words_half(a.z, b.z, make_float2(c45.x, c45.y), make_float2(c45.z, c45.w));
       rot_words_half(a.w, b.w, make_float2(c67.x, c67.y), make_float2(c67.z, c67.w));
-      *reinterpret_cast<uint4 *>(dst + off_x) = a;
-      *reinterpret_cast<uint4 *>(dst + off_y) = b;
     }
   }
+#pragma unroll
+  for (int i = 0; i < kVec; ++i) *reinterpret_cast<uint4 *>(dst + off[i]) = v[i];
 }
 
 template <int D>
@@ -353,7 +352,7 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
     for (int t = 0; t < 2; ++t) {
       mbar_init(&ctrl->s_full[t], 1); mbar_init(&ctrl->p_full[t][0], 128); mbar_init(&ctrl->p_full[t][1], 128);
       mbar_init(&ctrl->o_done[t], 1); mbar_init(&ctrl->o_free[t], 128);
-      mbar_init(&ctrl->qr_full[t], 4);
+      mbar_init(&ctrl->qr_full[t], 4); mbar_init(&ctrl->cs_full[t], D / 2);
     }
     for (int k = 0; k < kWorkSlots; ++k) { mbar_init(&ctrl->work_full[k], 1); mbar_init(&ctrl->work_empty[k], 9); }
     ctrl->abort_flag = 0;
@@ -608,6 +607,7 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
     const float sl = p.scale_log2;
     int s_uses = 0;                       // S tiles of this query tile consumed so far
     int o_uses = 0;                       // items in which this query tile was active
+    int n_staged = 0;                     // fused: (cos, sin) rows staged so far by this group
     int tiles_before = 0;                 // key tiles of all earlier items (the producer counts the same way)
     bool ok = true;
     Work wk;
@@ -635,19 +635,32 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
       // entry, first before the entry's first tile, then each time the block's last tile is done
       const int cached_end = min(tile0 + n_tiles, it.n_cache_tiles);   // tiles [tile0, cached_end) are cached keys
       int f_pc = 0, f_end = 0;                                         // current cached block and the tile index where it ends
-      auto rotate_for = [&](int pc) {
-        rotate_q_row<D>(smem + (t ? L::kQ1 : L::kQ0), smem + L::kBg + t * L::kTileBytes,
-                        p.q_rope + (size_t)pc * (D / 2), p.rope_layout, r);
+      // The block's (cos, sin) row goes through shared memory: thread r < D/2 of the group holds
+      // pair r, fetched one block ahead (cs_next), and the group's 128 threads wait for all of them.
+      float2 *cs_stage = reinterpret_cast<float2 *>(smem + L::kCtrl + 1024) + t * 64;
+      float2 cs_next = make_float2(1.f, 0.f);
+      auto fetch_cs = [&](int pc) {
+        if (r < D / 2 && pc < p.seg.n_cached_blocks) cs_next = __ldg(p.q_rope + (size_t)pc * (D / 2) + r);
+      };
+      auto rotate_now = [&]() -> bool {
+        if (r < D / 2) { cs_stage[r] = cs_next; mbar_arrive(&ctrl->cs_full[t]); }
+        if (!mbar_wait(&ctrl->cs_full[t], n_staged & 1, abort_flag)) return false;
+        ++n_staged;
+        rotate_q_row<D>(smem + (t ? L::kQ1 : L::kQ0), smem + L::kBg + t * L::kTileBytes, cs_stage, p.rope_layout, r);
         fence_proxy_async();                               // the tensor core reads through the async proxy
         __syncwarp();
         if ((tid & 31) == 0) mbar_arrive(&ctrl->qr_full[t]);
+        return true;
       };
       if (p.fused && tile0 < cached_end) {
         ok = mbar_wait(&ctrl->q_full[t], o_uses & 1, abort_flag);      // the query tile has landed
         if (!ok) break;
         f_pc = find_cache_block(p, it, it.ctile0 + tile0);
         f_end = __ldg(p.seg.cache_tile_cu + f_pc + 1);
-        rotate_for(f_pc);
+        fetch_cs(f_pc);
+        ok = rotate_now();
+        if (!ok) break;
+        fetch_cs(f_pc + 1);
       }
 
       for (int j = 0; j < n_tiles; ++j) {
@@ -748,7 +761,11 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
         if (p.fused && tile0 + j + 1 < cached_end && it.ctile0 + tile0 + j + 1 >= f_end) {
           ++f_pc;
           f_end = __ldg(p.seg.cache_tile_cu + f_pc + 1);
-          rotate_for(f_pc);
+          if (r == 0) BA_TR(t, j, 6);
+          ok = rotate_now();
+          if (!ok) break;
+          if (r == 0) BA_TR(t, j, 7);
+          fetch_cs(f_pc + 1);
         }
         float sum[8];
 #pragma unroll
