@@ -332,7 +332,8 @@ __device__ __forceinline__ void rotate_q_row(const uint8_t *__restrict__ src, ui
   for (int i = 0; i < kVec; ++i) *reinterpret_cast<uint4 *>(dst + off[i]) = v[i];
 }
 
-template <int D>
+// kFused selects the fused warm path at compile time, so that the plain path carries none of its code.
+template <int D, bool kFused>
 __global__ void __launch_bounds__(kThreads, 1)
 ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
                        const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ CUtensorMap tmap_kc,
@@ -405,12 +406,24 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
             tma_load_3d(smem + (t ? L::kQ1 : L::kQ0) + c * L::kRegionBytes, &tmap_q, &ctrl->q_full[t], c * 64,
                         wk.head0, it.q_row0 + t * p.tok);
         }
-        // pool mode: cached keys are walked block by block (block pc, row offset poff inside it)
+        // walk mode: cached keys are taken block by block (block pc, row offset poff inside it).  The
+        // current block's length and first rows sit in registers and the next block's are fetched a
+        // whole block ahead, so that no tile waits for a table look-up.
         int pc = 0, poff = 0;
+        int c_len = 0, k_base = 0, v_base = 0, n_len = 0, n_kbase = 0, n_vbase = 0;
+        auto load_block = [&](int b, int &len, int &kb, int &vb) {
+          if (b >= p.seg.n_cached_blocks) return;
+          const int c0 = __ldg(p.seg.cache_cu + b);
+          len = __ldg(p.seg.cache_cu + b + 1) - c0;
+          kb = p.k_src_off ? __ldg(p.k_src_off + b) : c0;
+          vb = p.v_src_off ? __ldg(p.v_src_off + b) : c0;
+        };
         if (p.walk && wk.tile0 < it.n_cache_tiles) {
           const int target = it.ctile0 + wk.tile0;
           pc = find_cache_block(p, it, target);
           poff = (target - __ldg(p.seg.cache_tile_cu + pc)) * kBlockN;
+          load_block(pc, c_len, k_base, v_base);
+          load_block(pc + 1, n_len, n_kbase, n_vbase);
         }
         for (int j = 0; j < wk.n_tiles && ok; ++j) {
           const int jt = wk.tile0 + j;
@@ -421,12 +434,15 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
           } else if (!p.walk) {
             k_row = v_row = it.cache_row0 + jt * kBlockN;
           } else {
-            const int c_begin = __ldg(p.seg.cache_cu + pc), c_len = __ldg(p.seg.cache_cu + pc + 1) - c_begin;
-            k_row = (p.k_src_off ? __ldg(p.k_src_off + pc) : c_begin) + poff;
-            v_row = (p.v_src_off ? __ldg(p.v_src_off + pc) : c_begin) + poff;
+            k_row = k_base + poff;
+            v_row = v_base + poff;
             ctrl->tile_valid[(gidx >> 1) & 7] = min(kBlockN, c_len - poff);   // read by the softmax warps
             poff += kBlockN;
-            if (poff >= c_len) { ++pc; poff = 0; }
+            if (poff >= c_len) {
+              ++pc; poff = 0;
+              c_len = n_len; k_base = n_kbase; v_base = n_vbase;
+              load_block(pc + 1, n_len, n_kbase, n_vbase);
+            }
           }
           for (int kv = 0; kv < 2; ++kv) {
             const int stage = gidx % kStages;
@@ -498,7 +514,7 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
       // S_t = Q_t K^T for tile `jrel` of the entry, whose keys sit at ring position idx
       auto issue_qk = [&](int t, int jrel, int idx) -> bool {
         const int jt = wk.tile0 + jrel;
-        if (!p.fused || jt >= cached_end) { issue_qk_with(t, idx, q_desc[t]); return true; }
+        if (!kFused || jt >= cached_end) { issue_qk_with(t, idx, q_desc[t]); return true; }
         const int g = wk.it.ctile0 + jt;
         if (g >= rot_end[t]) {
           // first key tile of another cached block: take the tile rotated for it
@@ -652,7 +668,7 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
         if ((tid & 31) == 0) mbar_arrive(&ctrl->qr_full[t]);
         return true;
       };
-      if (p.fused && tile0 < cached_end) {
+      if (kFused && tile0 < cached_end) {
         ok = mbar_wait(&ctrl->q_full[t], o_uses & 1, abort_flag);      // the query tile has landed
         if (!ok) break;
         f_pc = find_cache_block(p, it, it.ctile0 + tile0);
@@ -758,7 +774,7 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
         // the next tile belongs to another cached block: its rotated queries are due now, while the
         // tensor core works on PV of this tile (the QK^T that read the old rotation completed
         // before this tile's S arrived)
-        if (p.fused && tile0 + j + 1 < cached_end && it.ctile0 + tile0 + j + 1 >= f_end) {
+        if (kFused && tile0 + j + 1 < cached_end && it.ctile0 + tile0 + j + 1 >= f_end) {
           ++f_pc;
           f_end = __ldg(p.seg.cache_tile_cu + f_pc + 1);
           if (r == 0) BA_TR(t, j, 6);
@@ -1008,7 +1024,7 @@ ba_status ba_attend_sm100_launch(ba_ctx *ctx, const ba_attend_args &a, const ba_
   p.bg.n_rows = 0; p.bg_counter = nullptr; p.bg_rows_per_chunk = 0;
   if (ctx->has_pending) {
     const int row_bytes = ctx->pending.row_vecs * 16;
-    if (row_bytes <= kBgStageBytes && !p.fused) {   // the fused path uses the staging area and the spare warps itself
+    if (row_bytes <= kBgStageBytes && !p.fused) {   // the fused path keeps its rotated query tiles in the staging area
       p.bg = ctx->pending;
       ctx->has_pending = 0;
       ctx->pending_table_bytes = 0;
@@ -1024,12 +1040,14 @@ ba_status ba_attend_sm100_launch(ba_ctx *ctx, const ba_attend_args &a, const ba_
   // (each CTA allocates all 512 tensor-memory columns)
   if (D == 128) {
     const int smem = Layout<128>::kBytes + 1024;
-    BA_CUDA_TRY(cudaFuncSetAttribute(ba_attend_sm100_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-    ba_attend_sm100_kernel<128><<<grid, kThreads, smem, stream>>>(tq, tk, tv, tkc, tvc, p);
+    auto kern = p.fused ? ba_attend_sm100_kernel<128, true> : ba_attend_sm100_kernel<128, false>;
+    BA_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    kern<<<grid, kThreads, smem, stream>>>(tq, tk, tv, tkc, tvc, p);
   } else {
     const int smem = max(Layout<64>::kBytes + 1024, 120 * 1024);
-    BA_CUDA_TRY(cudaFuncSetAttribute(ba_attend_sm100_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-    ba_attend_sm100_kernel<64><<<grid, kThreads, smem, stream>>>(tq, tk, tv, tkc, tvc, p);
+    auto kern = p.fused ? ba_attend_sm100_kernel<64, true> : ba_attend_sm100_kernel<64, false>;
+    BA_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    kern<<<grid, kThreads, smem, stream>>>(tq, tk, tv, tkc, tvc, p);
   }
   BA_CUDA_TRY(cudaGetLastError());
   ctx->launches += 1;
