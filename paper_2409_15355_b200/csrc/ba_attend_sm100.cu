@@ -65,6 +65,9 @@ constexpr int kWorkSlots = 4;      // ring of published work entries (power of t
 #ifndef BA_SVC_REGS
 #define BA_SVC_REGS 72
 #endif
+#ifndef BA_FUSED_MMA_REGS
+#define BA_FUSED_MMA_REGS 152
+#endif
 #ifndef BA_SMX_REGS
 #define BA_SMX_REGS 216
 #endif
@@ -339,6 +342,12 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
                        const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ CUtensorMap tmap_kc,
                        const __grid_constant__ CUtensorMap tmap_vc, const AttnParams p) {
   using L = Layout<D>;
+  // registers of the service warps after launch (their sum is at most 4 * BA_SVC_REGS): on the fused path the
+  // spare warps have nothing to do and the MMA thread, which also follows the cached blocks, takes their share
+  constexpr int kProdRegs = BA_SVC_REGS;
+  constexpr int kMmaRegs = kFused ? BA_FUSED_MMA_REGS : BA_SVC_REGS;
+  constexpr int kSpareRegs = kFused ? 24 : BA_SVC_REGS;
+  static_assert(kProdRegs + kMmaRegs + 2 * kSpareRegs <= 4 * BA_SVC_REGS && kMmaRegs <= 168, "register split");
   extern __shared__ uint8_t smem_raw[];
   uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   Ctrl *ctrl = reinterpret_cast<Ctrl *>(smem + L::kCtrl);
@@ -373,7 +382,7 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
   // The softmax warps keep a whole 128-column row in registers; the service warps (8-11) need few.
   if (warp == 8) {
     // ------------------------------------------------------------ TMA producer
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(BA_SVC_REGS));
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kProdRegs));
     if (elect_one()) {
       prefetch_tmap(&tmap_q); prefetch_tmap(&tmap_k); prefetch_tmap(&tmap_v);
       prefetch_tmap(&tmap_kc); prefetch_tmap(&tmap_vc);
@@ -466,7 +475,7 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
     }
   } else if (warp == 9) {
     // ------------------------------------------------------------ MMA issuer
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(BA_SVC_REGS));
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kMmaRegs));
     if (elect_one()) {
       const uint32_t tS[2] = {tmem, tmem + 128};
       const uint32_t tO[2] = {tmem + 256, tmem + 384};
@@ -601,7 +610,7 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
     }
   } else if (warp >= 10) {
     // ------------------------------------------------------------ spare warps: background re-encoding
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(BA_SVC_REGS));
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kSpareRegs));
     if (p.bg.n_rows > 0) {
       // each spare warp runs the staged engine with its own two 16 KB stages; chunks are drawn from a
       // device-wide counter, so the job spreads over every CTA of the launch, early and late ones
