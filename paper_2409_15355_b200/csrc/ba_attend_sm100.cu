@@ -65,9 +65,6 @@ constexpr int kWorkSlots = 4;      // ring of published work entries (power of t
 #ifndef BA_SVC_REGS
 #define BA_SVC_REGS 72
 #endif
-#ifndef BA_FUSED_MMA_REGS
-#define BA_FUSED_MMA_REGS 152
-#endif
 #ifndef BA_SMX_REGS
 #define BA_SMX_REGS 216
 #endif
@@ -342,12 +339,8 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
                        const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ CUtensorMap tmap_kc,
                        const __grid_constant__ CUtensorMap tmap_vc, const AttnParams p) {
   using L = Layout<D>;
-  // registers of the service warps after launch (their sum is at most 4 * BA_SVC_REGS): on the fused path the
-  // spare warps have nothing to do and the MMA thread, which also follows the cached blocks, takes their share
-  constexpr int kProdRegs = BA_SVC_REGS;
-  constexpr int kMmaRegs = kFused ? BA_FUSED_MMA_REGS : BA_SVC_REGS;
-  constexpr int kSpareRegs = kFused ? 24 : BA_SVC_REGS;
-  static_assert(kProdRegs + kMmaRegs + 2 * kSpareRegs <= 4 * BA_SVC_REGS && kMmaRegs <= 168, "register split");
+  // setmaxnreg is a warpgroup-wide instruction: the four service warps (8-11) must ask for the same count
+  constexpr int kProdRegs = BA_SVC_REGS, kMmaRegs = BA_SVC_REGS, kSpareRegs = BA_SVC_REGS;
   extern __shared__ uint8_t smem_raw[];
   uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   Ctrl *ctrl = reinterpret_cast<Ctrl *>(smem + L::kCtrl);
