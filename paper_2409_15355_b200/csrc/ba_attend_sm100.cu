@@ -24,10 +24,13 @@
 // Fused warm path (Section 2.5 steps 2 and 3 in one launch): the cached keys stay at their
 // cache-time positions and the position difference of each block (Eq. 3 after Eq. 2) is applied
 // to the other side of the dot product, (R(p) q) . (R(delta + t) k) = (R(-delta) R(p) q) . (R(t) k):
-// each softmax thread counter-rotates its own row of its query tile once per cached block into a
-// second pair of buffers, which the QK^T products of that block's key tiles read; it does so
-// right after handing over P of the block's last tile, while it would otherwise wait for the next
-// S.  The cached keys are then never rewritten or re-read, and a key tile never spans two blocks.
+// each softmax thread owns one row of its query tile and prepares, for every cached block of the
+// work entry, a copy of that row rotated by the block's delta (and a plain copy for the final
+// block's own keys) in one of two buffers per query tile.  The copy for the next block is made
+// while the current block's tiles are worked on -- the raw row is fetched with cp.async after one
+// tile, rotated in place after the next, in time the thread would otherwise spend waiting for S --
+// so the QK^T products switch buffers without a pause.  The cached keys are never rewritten or
+// re-read, and a key tile never spans two blocks.
 #include <math.h>
 #include <type_traits>
 
@@ -89,6 +92,7 @@ struct AttnParams {
   int fused;                      // cached keys are at cache-time positions: queries are counter-rotated per block
   int rope_layout;
   const float2 *q_rope;           // fused: [cached blocks][D/2] (cos, sin) of delta_c * theta_m
+  const __nv_bfloat16 *q;         // fused: the query rows (read by the softmax threads themselves)
   int persistent;                 // 1: CTAs draw work from work_counter; 0: CTA b handles entry b only
   int32_t *work_counter;          // device word, zero at launch: next entry of the work list
   ba_reencode_job bg;             // bg.n_rows > 0: a re-encoding job the two spare warps carry out meanwhile
@@ -107,7 +111,7 @@ struct Layout {
   static constexpr int kRing = 2 * kTileBytes;
   static constexpr int kCtrl = kRing + kStages * kTileBytes;   // 2 KB: Ctrl, then two ba_bg_smem
   static constexpr int kBg = kCtrl + 2048;                     // staging of the background re-encoding, or (fused
-                                                               // path) the two counter-rotated query tiles
+                                                               // path) the second pair of query tile buffers
   static constexpr int kBytes = kBg + 4 * kBgStageBytes;
 };
 
@@ -120,7 +124,7 @@ struct Ctrl {
   uint64_t p_full[2][2];          // [query tile][half of the P tile]
   uint64_t o_done[2];
   uint64_t o_free[2];             // the softmax warps have read O_t out of tensor memory
-  uint64_t qr_full[2];            // fused: counter-rotated query tile t is ready for the next cached block
+  uint64_t qr_full[2][2];         // fused: [query tile][buffer] the tile prepared for the next key range is ready
   uint64_t cs_full[2];            // fused: the block's (cos, sin) row has been staged for softmax group t
   uint64_t work_full[kWorkSlots];  // work entry published by the scheduler (producer thread)
   uint64_t work_empty[kWorkSlots]; // entry read by the MMA thread and the 8 softmax warps
@@ -355,7 +359,7 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
     for (int t = 0; t < 2; ++t) {
       mbar_init(&ctrl->s_full[t], 1); mbar_init(&ctrl->p_full[t][0], 128); mbar_init(&ctrl->p_full[t][1], 128);
       mbar_init(&ctrl->o_done[t], 1); mbar_init(&ctrl->o_free[t], 128);
-      mbar_init(&ctrl->qr_full[t], 4); mbar_init(&ctrl->cs_full[t], D / 2);
+      mbar_init(&ctrl->qr_full[t][0], 4); mbar_init(&ctrl->qr_full[t][1], 4); mbar_init(&ctrl->cs_full[t], D / 2);
     }
     for (int k = 0; k < kWorkSlots; ++k) { mbar_init(&ctrl->work_full[k], 1); mbar_init(&ctrl->work_empty[k], 9); }
     ctrl->abort_flag = 0;
@@ -398,15 +402,17 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
         if (!more) break;
         if (wk.n_tiles == 0) continue;
         const Item &it = wk.it;
-        // the Q buffers are free once every QK^T of the previous item has completed
-        ok = mbar_wait(&ctrl->q_empty, (n_items & 1) ^ 1, abort_flag);
-        if (!ok) break;
-        ++n_items;
-        for (int t = 0; t < it.n_qt; ++t) {
-          mbar_arrive_expect_tx(&ctrl->q_full[t], L::kTileBytes);
-          for (int c = 0; c < L::kChunks; ++c)
-            tma_load_3d(smem + (t ? L::kQ1 : L::kQ0) + c * L::kRegionBytes, &tmap_q, &ctrl->q_full[t], c * 64,
-                        wk.head0, it.q_row0 + t * p.tok);
+        if (!kFused) {      // (on the fused path the softmax threads fetch the query rows themselves)
+          // the Q buffers are free once every QK^T of the previous item has completed
+          ok = mbar_wait(&ctrl->q_empty, (n_items & 1) ^ 1, abort_flag);
+          if (!ok) break;
+          ++n_items;
+          for (int t = 0; t < it.n_qt; ++t) {
+            mbar_arrive_expect_tx(&ctrl->q_full[t], L::kTileBytes);
+            for (int c = 0; c < L::kChunks; ++c)
+              tma_load_3d(smem + (t ? L::kQ1 : L::kQ0) + c * L::kRegionBytes, &tmap_q, &ctrl->q_full[t], c * 64,
+                          wk.head0, it.q_row0 + t * p.tok);
+          }
         }
         // walk mode: cached keys are taken block by block (block pc, row offset poff inside it).  The
         // current block's length and first rows sit in registers and the next block's are fetched a
@@ -505,31 +511,40 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
       int n_work = 0;
       // Every loop over the query tile t below is unrolled, so that t is a constant and the small
       // per-tile arrays live in registers: this thread's issue latency is on the critical path.
-      // fused path: the QK^T of a cached key tile reads the query tile counter-rotated for that tile's
-      // block; the softmax warps rotate once per (block, query tile) and both sides count those alike
-      const uint64_t qr_desc[2] = {make_smem_desc(smem_u32(smem + L::kBg), 16, 1024),
+      // fused path: a "version" of query tile t is the tile prepared for one key range of the entry --
+      // rotated for one cached block, or plain for the final block's own keys.  The softmax threads
+      // prepare versions in order into alternating buffers; both sides count them alike.
+      const uint64_t qb_desc[2] = {make_smem_desc(smem_u32(smem + L::kBg), 16, 1024),         // second buffers
                                    make_smem_desc(smem_u32(smem + L::kBg + L::kTileBytes), 16, 1024)};
-      int n_rot[2] = {0, 0};               // rotations of query tile t consumed so far
-      int rot_end[2] = {-1, -1};           // the rotated tile t is valid for cached key tiles below this index
+      int n_ver[2] = {0, 0};               // versions of query tile t taken so far
+      int ver_end[2] = {-1, -1};           // the current version of tile t serves cached key tiles below this index
       int walk_pc = 0, walk_end = -1;      // block of the current cached tile and the tile index where it ends
       int cached_end = 0;                  // tiles [tile0, cached_end) of the entry are cached keys
       // S_t = Q_t K^T for tile `jrel` of the entry, whose keys sit at ring position idx
       auto issue_qk = [&](int t, int jrel, int idx) -> bool {
+        if (!kFused) { issue_qk_with(t, idx, q_desc[t]); return true; }
         const int jt = wk.tile0 + jrel;
-        if (!kFused || jt >= cached_end) { issue_qk_with(t, idx, q_desc[t]); return true; }
-        const int g = wk.it.ctile0 + jt;
-        if (g >= rot_end[t]) {
-          // first key tile of another cached block: take the tile rotated for it
-          if (walk_end < 0) { walk_pc = find_cache_block(p, wk.it, g); walk_end = __ldg(p.seg.cache_tile_cu + walk_pc + 1); }
-          while (g >= walk_end) { ++walk_pc; walk_end = __ldg(p.seg.cache_tile_cu + walk_pc + 1); }
-          BA_TR(5, n_rot[t], t * 2);
-          if (!mbar_wait(&ctrl->qr_full[t], n_rot[t] & 1, abort_flag)) return false;
-          BA_TR(5, n_rot[t], t * 2 + 1);
-          ++n_rot[t];
-          rot_end[t] = walk_end;
+        bool change = false;
+        if (jt < cached_end) {
+          const int g = wk.it.ctile0 + jt;
+          if (g >= ver_end[t]) {                           // first key tile of another cached block
+            if (walk_end < 0) { walk_pc = find_cache_block(p, wk.it, g); walk_end = __ldg(p.seg.cache_tile_cu + walk_pc + 1); }
+            while (g >= walk_end) { ++walk_pc; walk_end = __ldg(p.seg.cache_tile_cu + walk_pc + 1); }
+            ver_end[t] = walk_end;
+            change = true;
+          }
+        } else if (ver_end[t] != 0x7fffffff) {             // first of the final block's own key tiles
+          ver_end[t] = 0x7fffffff;
+          change = true;
+        }
+        if (change) {
+          BA_TR(5, n_ver[t] & 63, t * 2);
+          if (!mbar_wait(&ctrl->qr_full[t][n_ver[t] & 1], (n_ver[t] >> 1) & 1, abort_flag)) return false;
+          BA_TR(5, n_ver[t] & 63, t * 2 + 1);
+          ++n_ver[t];
           tc_fence_after();
         }
-        issue_qk_with(t, idx, qr_desc[t]);
+        issue_qk_with(t, idx, ((n_ver[t] - 1) & 1) ? qb_desc[t] : q_desc[t]);
         return true;
       };
       for (;;) {
@@ -542,11 +557,13 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
         mbar_arrive(&ctrl->work_empty[slot]);          // the entry has been decoded into registers
         const int n_tiles = wk.n_tiles, n_qt = wk.it.n_qt;
         if (n_tiles == 0) continue;
-        walk_end = -1; rot_end[0] = rot_end[1] = -1;
+        walk_end = -1; ver_end[0] = ver_end[1] = -1;
         cached_end = min(wk.tile0 + n_tiles, wk.it.n_cache_tiles);
+        if (!kFused) {
 #pragma unroll
-        for (int t = 0; t < 2; ++t)
-          if (t < n_qt && ok) ok = mbar_wait(&ctrl->q_full[t], q_uses[t] & 1, abort_flag);
+          for (int t = 0; t < 2; ++t)
+            if (t < n_qt && ok) ok = mbar_wait(&ctrl->q_full[t], q_uses[t] & 1, abort_flag);
+        }
         if (ok) ok = wait_kv(gidx);
         if (!ok) break;
         tc_fence_after();
@@ -626,6 +643,7 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
     int s_uses = 0;                       // S tiles of this query tile consumed so far
     int o_uses = 0;                       // items in which this query tile was active
     int n_staged = 0;                     // fused: (cos, sin) rows staged so far by this group
+    int n_made = 0;                       // fused: versions of this query tile prepared so far
     int tiles_before = 0;                 // key tiles of all earlier items (the producer counts the same way)
     bool ok = true;
     Work wk;
@@ -649,10 +667,16 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
       const int head = head0 + (r & (p.hpt - 1));
       float m_used = -INFINITY, l = 0.f;
 
-      // fused path: this thread counter-rotates row r of query tile t for each cached block of the
-      // entry, first before the entry's first tile, then each time the block's last tile is done
-      const int cached_end = min(tile0 + n_tiles, it.n_cache_tiles);   // tiles [tile0, cached_end) are cached keys
-      int f_pc = 0, f_end = 0;                                         // current cached block and the tile index where it ends
+      // fused path: this thread prepares row r of every version of query tile t (see the MMA warp):
+      // the raw row is fetched with cp.async into the buffer the version will live in and, for a cached
+      // block, rotated there in place.  The first version of an entry is made on the spot; every later
+      // one is begun after one tile of its predecessor and finished after the next, or at the latest
+      // when its first key tile is next.
+      const int tile_end = tile0 + n_tiles;
+      const int cached_end = min(tile_end, it.n_cache_tiles);          // tiles [tile0, cached_end) are cached keys
+      int f_pc = 0;                        // cached block of the version being prepared / in use
+      int next_start = tile_end;           // first tile of the next version (tile_end: there is none)
+      int prep = 0;                        // next version: 0 not begun, 1 row being fetched, 2 ready
       // The block's (cos, sin) row goes through shared memory: thread r < D/2 of the group holds
       // pair r, fetched one block ahead (cs_next), and the group's 128 threads wait for all of them.
       float2 *cs_stage = reinterpret_cast<float2 *>(smem + L::kCtrl + 1024) + t * 64;
@@ -660,25 +684,48 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
       auto fetch_cs = [&](int pc) {
         if (r < D / 2 && pc < p.seg.n_cached_blocks) cs_next = __ldg(p.q_rope + (size_t)pc * (D / 2) + r);
       };
-      auto rotate_now = [&]() -> bool {
-        if (r < D / 2) { cs_stage[r] = cs_next; mbar_arrive(&ctrl->cs_full[t]); }
-        if (!mbar_wait(&ctrl->cs_full[t], n_staged & 1, abort_flag)) return false;
-        ++n_staged;
-        rotate_q_row<D>(smem + (t ? L::kQ1 : L::kQ0), smem + L::kBg + t * L::kTileBytes, cs_stage, p.rope_layout, r);
+      auto ver_buf = [&](int v) { return smem + ((v & 1) ? L::kBg : L::kQ0) + t * L::kTileBytes; };
+      auto begin_version = [&]() {       // raw row r -> buffer of version n_made
+        const int tok_idx = min(row_tok, p.n_q_rows - 1);
+        const uint8_t *src = reinterpret_cast<const uint8_t *>(p.q + ((size_t)tok_idx * p.Hq + head) * D);
+        const uint32_t dst = smem_u32(ver_buf(n_made)) + r * 128;
+#pragma unroll
+        for (int i = 0; i < D / 8; ++i)
+          asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + (i >> 3) * L::kRegionBytes + (((i & 7) ^ (r & 7)) << 4)),
+                       "l"(src + i * 16) : "memory");
+        asm volatile("cp.async.commit_group;" ::: "memory");
+      };
+      auto finish_version = [&](bool rotated) -> bool {
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
+        if (rotated) {
+          if (r < D / 2) { cs_stage[r] = cs_next; mbar_arrive(&ctrl->cs_full[t]); }
+          if (!mbar_wait(&ctrl->cs_full[t], n_staged & 1, abort_flag)) return false;
+          ++n_staged;
+          rotate_q_row<D>(ver_buf(n_made), ver_buf(n_made), cs_stage, p.rope_layout, r);
+        }
         fence_proxy_async();                               // the tensor core reads through the async proxy
         __syncwarp();
-        if ((tid & 31) == 0) mbar_arrive(&ctrl->qr_full[t]);
+        if ((tid & 31) == 0) mbar_arrive(&ctrl->qr_full[t][n_made & 1]);
+        ++n_made;
         return true;
       };
-      if (kFused && tile0 < cached_end) {
-        ok = mbar_wait(&ctrl->q_full[t], o_uses & 1, abort_flag);      // the query tile has landed
+      // where the version after the one for block `pc` (or after the plain one: pc < 0) starts
+      auto plan_next = [&](int pc) {
+        next_start = tile_end;
+        if (pc >= 0) {
+          const int e = __ldg(p.seg.cache_tile_cu + pc + 1) - it.ctile0;   // first tile after the block
+          if (e < tile_end) next_start = min(e, cached_end);
+          if (next_start < cached_end) fetch_cs(pc + 1);
+        }
+        prep = 0;
+      };
+      if (kFused && n_tiles > 0) {
+        const bool first_cached = tile0 < cached_end;
+        if (first_cached) { f_pc = find_cache_block(p, it, it.ctile0 + tile0); fetch_cs(f_pc); }
+        begin_version();
+        ok = finish_version(first_cached);
         if (!ok) break;
-        f_pc = find_cache_block(p, it, it.ctile0 + tile0);
-        f_end = __ldg(p.seg.cache_tile_cu + f_pc + 1);
-        fetch_cs(f_pc);
-        ok = rotate_now();
-        if (!ok) break;
-        fetch_cs(f_pc + 1);
+        plan_next(first_cached ? f_pc : -1);
       }
 
       for (int j = 0; j < n_tiles; ++j) {
@@ -773,17 +820,16 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
         };
         if (kPolyPeriod > 0 && __all_sync(0xffffffffu, lim >= kBlockN - 1)) exp_halves(std::true_type{});
         else exp_halves(std::false_type{});
-        // the next tile belongs to another cached block: its rotated queries are due now, while the
-        // tensor core works on PV of this tile (the QK^T that read the old rotation completed
-        // before this tile's S arrived)
-        if (kFused && tile0 + j + 1 < cached_end && it.ctile0 + tile0 + j + 1 >= f_end) {
-          ++f_pc;
-          f_end = __ldg(p.seg.cache_tile_cu + f_pc + 1);
+        // P of this tile is with the tensor core: time to work on the next version of the query row
+        if (kFused && next_start < tile_end) {
+          const bool due = tile0 + j + 1 == next_start;    // the next tile is the first to need it
+          const bool next_cached = next_start < cached_end;
           if (r == 0) BA_TR(t, j, 6);
-          ok = rotate_now();
+          if (prep == 0) { begin_version(); prep = 1; if (due) { ok = finish_version(next_cached); prep = 2; } }
+          else if (prep == 1) { ok = finish_version(next_cached); prep = 2; }
           if (!ok) break;
           if (r == 0) BA_TR(t, j, 7);
-          fetch_cs(f_pc + 1);
+          if (due) { if (next_cached) ++f_pc; plan_next(next_cached ? f_pc : -1); }
         }
         float sum[8];
 #pragma unroll
@@ -964,6 +1010,7 @@ ba_status ba_attend_sm100_launch(ba_ctx *ctx, const ba_attend_args &a, const ba_
   p.walk = p.v_src_off != nullptr || p.fused;
   p.rope_layout = ctx->cfg.rope_layout;
   p.q_rope = p.fused ? reinterpret_cast<const float2 *>(seg->cache_rope) : nullptr;
+  p.q = a.q;
   if (p.fused && !p.q_rope) return BA_ERR_INVALID_ARG;
   p.n_q_rows = a.n_q_rows;
   p.seg = *seg;
