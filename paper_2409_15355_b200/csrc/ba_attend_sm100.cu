@@ -27,8 +27,8 @@
 // each softmax thread owns one row of its query tile and prepares, for every cached block of the
 // work entry, a copy of that row rotated by the block's delta (and a plain copy for the final
 // block's own keys) in one of two buffers per query tile.  The copy for the next block is made
-// while the current block's tiles are worked on -- the raw row is fetched with cp.async after one
-// tile, rotated in place after the next, in time the thread would otherwise spend waiting for S --
+// while the current block's tiles are worked on -- the plain tile is fetched after one tile and
+// rotated in place after the next, in time the thread would otherwise spend waiting for S --
 // so the QK^T products switch buffers without a pause.  The cached keys are never rewritten or
 // re-read, and a key tile never spans two blocks.
 #include <math.h>
@@ -92,7 +92,6 @@ struct AttnParams {
   int fused;                      // cached keys are at cache-time positions: queries are counter-rotated per block
   int rope_layout;
   const float2 *q_rope;           // fused: [cached blocks][D/2] (cos, sin) of delta_c * theta_m
-  const __nv_bfloat16 *q;         // fused: the query rows (read by the softmax threads themselves)
   int persistent;                 // 1: CTAs draw work from work_counter; 0: CTA b handles entry b only
   int32_t *work_counter;          // device word, zero at launch: next entry of the work list
   ba_reencode_job bg;             // bg.n_rows > 0: a re-encoding job the two spare warps carry out meanwhile
@@ -126,6 +125,7 @@ struct Ctrl {
   uint64_t o_free[2];             // the softmax warps have read O_t out of tensor memory
   uint64_t qr_full[2][2];         // fused: [query tile][buffer] the tile prepared for the next key range is ready
   uint64_t cs_full[2];            // fused: the block's (cos, sin) row has been staged for softmax group t
+  uint64_t qraw_full[2];          // fused: the plain query tile t has landed in the buffer of the version being prepared
   uint64_t work_full[kWorkSlots];  // work entry published by the scheduler (producer thread)
   uint64_t work_empty[kWorkSlots]; // entry read by the MMA thread and the 8 softmax warps
   int work_ring[kWorkSlots];
@@ -360,6 +360,7 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
       mbar_init(&ctrl->s_full[t], 1); mbar_init(&ctrl->p_full[t][0], 128); mbar_init(&ctrl->p_full[t][1], 128);
       mbar_init(&ctrl->o_done[t], 1); mbar_init(&ctrl->o_free[t], 128);
       mbar_init(&ctrl->qr_full[t][0], 4); mbar_init(&ctrl->qr_full[t][1], 4); mbar_init(&ctrl->cs_full[t], D / 2);
+      mbar_init(&ctrl->qraw_full[t], 1);
     }
     for (int k = 0; k < kWorkSlots; ++k) { mbar_init(&ctrl->work_full[k], 1); mbar_init(&ctrl->work_empty[k], 9); }
     ctrl->abort_flag = 0;
@@ -402,7 +403,7 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
         if (!more) break;
         if (wk.n_tiles == 0) continue;
         const Item &it = wk.it;
-        if (!kFused) {      // (on the fused path the softmax threads fetch the query rows themselves)
+        if (!kFused) {      // (on the fused path the softmax warps fetch the query tiles themselves)
           // the Q buffers are free once every QK^T of the previous item has completed
           ok = mbar_wait(&ctrl->q_empty, (n_items & 1) ^ 1, abort_flag);
           if (!ok) break;
@@ -668,8 +669,8 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
       float m_used = -INFINITY, l = 0.f;
 
       // fused path: this thread prepares row r of every version of query tile t (see the MMA warp):
-      // the raw row is fetched with cp.async into the buffer the version will live in and, for a cached
-      // block, rotated there in place.  The first version of an entry is made on the spot; every later
+      // the plain tile is fetched by the copy engine into the buffer the version will live in and, for a
+      // cached block, every thread rotates its row there in place.  The first version of an entry is made on the spot; every later
       // one is begun after one tile of its predecessor and finished after the next, or at the latest
       // when its first key tile is next.
       const int tile_end = tile0 + n_tiles;
@@ -685,18 +686,16 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
         if (r < D / 2 && pc < p.seg.n_cached_blocks) cs_next = __ldg(p.q_rope + (size_t)pc * (D / 2) + r);
       };
       auto ver_buf = [&](int v) { return smem + ((v & 1) ? L::kBg : L::kQ0) + t * L::kTileBytes; };
-      auto begin_version = [&]() {       // raw row r -> buffer of version n_made
-        const int tok_idx = min(row_tok, p.n_q_rows - 1);
-        const uint8_t *src = reinterpret_cast<const uint8_t *>(p.q + ((size_t)tok_idx * p.Hq + head) * D);
-        const uint32_t dst = smem_u32(ver_buf(n_made)) + r * 128;
-#pragma unroll
-        for (int i = 0; i < D / 8; ++i)
-          asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + (i >> 3) * L::kRegionBytes + (((i & 7) ^ (r & 7)) << 4)),
-                       "l"(src + i * 16) : "memory");
-        asm volatile("cp.async.commit_group;" ::: "memory");
+      auto begin_version = [&]() {       // plain query tile -> buffer of version n_made (one thread asks the copy engine)
+        if (r == 0) {
+          mbar_arrive_expect_tx(&ctrl->qraw_full[t], L::kTileBytes);
+          for (int c = 0; c < L::kChunks; ++c)
+            tma_load_3d(ver_buf(n_made) + c * L::kRegionBytes, &tmap_q, &ctrl->qraw_full[t], c * 64, head0,
+                        it.q_row0 + t * p.tok);
+        }
       };
       auto finish_version = [&](bool rotated) -> bool {
-        asm volatile("cp.async.wait_group 0;" ::: "memory");
+        if (!mbar_wait(&ctrl->qraw_full[t], n_made & 1, abort_flag)) return false;
         if (rotated) {
           if (r < D / 2) { cs_stage[r] = cs_next; mbar_arrive(&ctrl->cs_full[t]); }
           if (!mbar_wait(&ctrl->cs_full[t], n_staged & 1, abort_flag)) return false;
@@ -1010,7 +1009,6 @@ ba_status ba_attend_sm100_launch(ba_ctx *ctx, const ba_attend_args &a, const ba_
   p.walk = p.v_src_off != nullptr || p.fused;
   p.rope_layout = ctx->cfg.rope_layout;
   p.q_rope = p.fused ? reinterpret_cast<const float2 *>(seg->cache_rope) : nullptr;
-  p.q = a.q;
   if (p.fused && !p.q_rope) return BA_ERR_INVALID_ARG;
   p.n_q_rows = a.n_q_rows;
   p.seg = *seg;
