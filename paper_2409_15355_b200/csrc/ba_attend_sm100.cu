@@ -68,6 +68,10 @@ constexpr int kWorkSlots = 4;      // ring of published work entries (power of t
 #ifndef BA_SVC_REGS
 #define BA_SVC_REGS 72
 #endif
+// the MMA thread's loops over the two query tiles
+#ifndef BA_T_UNROLL
+#define BA_T_UNROLL _Pragma("unroll")
+#endif
 #ifndef BA_SMX_REGS
 #define BA_SMX_REGS 216
 #endif
@@ -87,17 +91,17 @@ struct AttnParams {
   float *o_part;                  // [n_splits, n_q_rows, Hq, D] fp32, each normalised by its own denominator
   float *lse_part;                // [n_splits, n_q_rows, Hq] natural-log denominators (-inf: split saw no key)
   const int32_t *v_src_off;       // non-null: values of cached block c start at pool row v_src_off[c]
-  const int32_t *k_src_off;       // non-null: keys of cached block c start at pool row k_src_off[c] (fused path only)
-  int walk;                       // cached keys are walked block by block (a tile never spans two blocks)
-  int fused;                      // cached keys are at cache-time positions: queries are counter-rotated per block
-  int rope_layout;
-  const float2 *q_rope;           // fused: [cached blocks][D/2] (cos, sin) of delta_c * theta_m
   int persistent;                 // 1: CTAs draw work from work_counter; 0: CTA b handles entry b only
   int32_t *work_counter;          // device word, zero at launch: next entry of the work list
   ba_reencode_job bg;             // bg.n_rows > 0: a re-encoding job the two spare warps carry out meanwhile
   int32_t *bg_counter;            // device word, zero at launch: next chunk of that job
   int bg_rows_per_chunk;
   ba_segments seg;
+  const int32_t *k_src_off;       // non-null: keys of cached block c start at pool row k_src_off[c] (fused path only)
+  int walk;                       // cached keys are walked block by block (a tile never spans two blocks)
+  int fused;                      // cached keys are at cache-time positions: queries are counter-rotated per block
+  int rope_layout;
+  const float2 *q_rope;           // fused: [cached blocks][D/2] (cos, sin) of delta_c * theta_m
 };
 
 template <int D>
@@ -123,15 +127,15 @@ struct Ctrl {
   uint64_t p_full[2][2];          // [query tile][half of the P tile]
   uint64_t o_done[2];
   uint64_t o_free[2];             // the softmax warps have read O_t out of tensor memory
-  uint64_t qr_full[2][2];         // fused: [query tile][buffer] the tile prepared for the next key range is ready
-  uint64_t cs_full[2];            // fused: the block's (cos, sin) row has been staged for softmax group t
-  uint64_t qraw_full[2];          // fused: the plain query tile t has landed in the buffer of the version being prepared
   uint64_t work_full[kWorkSlots];  // work entry published by the scheduler (producer thread)
   uint64_t work_empty[kWorkSlots]; // entry read by the MMA thread and the 8 softmax warps
   int work_ring[kWorkSlots];
   int tile_valid[8];              // pool mode: valid key columns of the cached tiles in flight
   uint32_t tmem_base;
   int abort_flag;
+  uint64_t qr_full[2][2];         // fused: [query tile][buffer] the tile prepared for the next key range is ready
+  uint64_t cs_full[2];            // fused: the block's (cos, sin) row has been staged for softmax group t
+  uint64_t qraw_full[2];          // fused: the plain query tile t has landed in the buffer of the version being prepared
 };
 
 // One work item: two query tiles of one block (or final block) and the key ranges they see.
@@ -561,14 +565,14 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
         walk_end = -1; ver_end[0] = ver_end[1] = -1;
         cached_end = min(wk.tile0 + n_tiles, wk.it.n_cache_tiles);
         if (!kFused) {
-#pragma unroll
+BA_T_UNROLL
           for (int t = 0; t < 2; ++t)
             if (t < n_qt && ok) ok = mbar_wait(&ctrl->q_full[t], q_uses[t] & 1, abort_flag);
         }
         if (ok) ok = wait_kv(gidx);
         if (!ok) break;
         tc_fence_after();
-#pragma unroll
+BA_T_UNROLL
         for (int t = 0; t < 2; ++t)
           if (t < n_qt && ok) ok = issue_qk(t, 0, gidx);
         if (!ok) break;
@@ -580,7 +584,7 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
           BA_TR(3, j, 0);
           ok = wait_kv(iv);
           BA_TR(3, j, 1);
-#pragma unroll
+BA_T_UNROLL
           for (int t = 0; t < 2; ++t) {
             if (t >= n_qt || !ok) continue;
             BA_TR(2, j, t * 4 + 0);
@@ -614,7 +618,7 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
           }
         }
         gidx += 2 * n_tiles;
-#pragma unroll
+BA_T_UNROLL
         for (int t = 0; t < 2; ++t)
           if (t < n_qt) ++q_uses[t];
       }
