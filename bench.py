@@ -347,6 +347,59 @@ def run_ours(args):
         ctx4.close()
         del q4, k4, v4, o4
 
+    # ---- secondary number: the fused warm path (keys as cached, queries counter-rotated per block in
+    # the attention launch, no re-encoding pass) on the same 32-layer workload, and both paths with a
+    # short final block, where the query side is small and the fused path is the faster one
+    fused = None
+    if rank == 0 and not args.no_fused:
+        def fused_step(inputs):
+            seg = B.ba_segment(ctx.ctx, lens, nb, 1, len(lens), w.n_tokens, B.BA_MODE_BLOCK, tbuf)
+            for l in range(L):
+                x = inputs[l]
+                B.ba_final_attend_fused(ctx.ctx, x["q_f"], x["k_f"], x["v_f"], Tf, x["k_cache"], x["v_cache"], Tc,
+                                        None, Tc, o[l], None, seg, B.BA_MODE_BLOCK, B.BA_OUT_BF16)
+        for _ in range(3):
+            fused_step(d_in)
+        torch.cuda.synchronize()
+        reps = max(1, min(args.steps, 20))
+        ev0.record(stream)
+        for _ in range(reps):
+            fused_step(d_in)
+        ev1.record(stream)
+        torch.cuda.synchronize()
+        fused = {"workload": "the metric's workload through ba_final_attend_fused (no ba_reencode_k pass)",
+                 "us_per_layer": ev0.elapsed_time(ev1) * 1e3 / reps / L}
+        # short final block: 32 x 1000 cached + 64 final tokens, one layer's tensors reused over 4 buffers
+        Ts = 64
+        lens_s = np.asarray([1000] * 32 + [Ts], dtype=np.int32)
+        seg_s = B.ba_segment(ctx.ctx, lens_s, nb, 1, len(lens_s), int(lens_s.sum()), B.BA_MODE_BLOCK, tbuf)
+        nl = min(L, 4)
+        def short_step(use_fused):
+            for l in range(nl):
+                x = d_in[l]
+                if use_fused:
+                    B.ba_final_attend_fused(ctx.ctx, x["q_f"][:Ts], x["k_f"][:Ts], x["v_f"][:Ts], Ts, x["k_cache"],
+                                            x["v_cache"], Tc, None, Tc, o[l][:Ts], None, seg_s, B.BA_MODE_BLOCK,
+                                            B.BA_OUT_BF16)
+                else:
+                    B.ba_reencode_k(ctx.ctx, x["k_cache"], None, Tc, k_re[l], seg_s.cache_cu, seg_s.cache_delta,
+                                    seg_s.n_cached_blocks, Tc)
+                    B.ba_final_attend(ctx.ctx, x["q_f"][:Ts], x["k_f"][:Ts], x["v_f"][:Ts], Ts, k_re[l], x["v_cache"],
+                                      Tc, None, 0, o[l][:Ts], None, seg_s, B.BA_MODE_BLOCK, B.BA_OUT_BF16)
+        short = {}
+        for name, uf in (("unfused_us_per_layer", False), ("fused_us_per_layer", True)):
+            for _ in range(3):
+                short_step(uf)
+            torch.cuda.synchronize()
+            ev0.record(stream)
+            for _ in range(10):
+                short_step(uf)
+            ev1.record(stream)
+            torch.cuda.synchronize()
+            short[name] = ev0.elapsed_time(ev1) * 1e3 / 10 / nl
+        fused["short_final_block"] = dict(final_block=Ts, cached="32 x 1000", **short)
+        assert ctx.device_status() == B.BA_OK
+
     if rank == 0:
         peaks = load_peaks()
         cfg_extra = {"reencode": "queued, in the background of the previous layer's attention launch"} if args.deferred else {}
@@ -374,6 +427,8 @@ def run_ours(args):
                 "e2e": {"value": e2e_us, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                         "steps": e2e_steps},
                 "gpu_launches": launches, "roofline": roofline, "cpu_baseline": cpu}
+        if fused is not None:
+            line["fused_warm_path"] = fused
         if prefill is not None:
             prefill["frac_of_bf16_burst"] = prefill["tflops"] / peaks["bf16_tflops"]
             line["block_prefill"] = prefill
@@ -395,6 +450,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--layers", type=int, default=32, help="layers per step (32 = the metric's workload)")
     ap.add_argument("--no-prefill", action="store_true", help="skip the secondary cold-prefill measurement")
+    ap.add_argument("--no-fused", action="store_true", help="skip the secondary fused-warm-path measurement")
     ap.add_argument("--deferred", action="store_true",
                     help="queue each layer's re-encoding so that it runs in the background of the previous layer's "
                          "attention launch (ba_reencode_k_deferred) instead of as a stand-alone launch")
