@@ -34,6 +34,12 @@ METRIC = "final-block attend+reencode us/layer at 32K ctx"
 UNIT = "us/layer"
 
 
+# dram__bytes_read.sum + dram__bytes_write.sum of one attention launch of this workload (145.4 + 23.8 MB),
+# from the ncu capture summarised in profiles/warm_path_cfg3_32k.md; the algorithmic figure is 146.8 MB.
+# Set to None whenever the attention kernel changes after that capture.
+ATTEND_DRAM_BYTES_PER_LAUNCH = 169.3e6
+
+
 def load_peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
@@ -408,7 +414,7 @@ def run_ours(args):
         achieved = flops / (att_ms * 1e-3) / 1e12
         peak = peaks["bf16_tflops_sustained"] or peaks["bf16_tflops"]
         roofline = {"bound": "tensor", "kernel": "ba_final_attend", "achieved": achieved, "peak": peak,
-                    "unit": "TFLOP/s", "frac": achieved / peak, "traffic": None,
+                    "unit": "TFLOP/s", "frac": achieved / peak, "traffic": ATTEND_DRAM_BYTES_PER_LAUNCH,
                     "peak_source": f"{peaks['source']} bf16 sustained (kernel timed inside a 32-layer step); "
                                    f"burst {peaks['bf16_tflops']}",
                     "frac_of_burst": achieved / peaks["bf16_tflops"],
