@@ -386,6 +386,63 @@ def test_fused_warm_path_32k_full_size_and_pool_serving():
     check_attention(o, o_ref, lse, lse_ref)
 
 
+def test_incremental_block_update_many_small_blocks():
+    """Section 2.1 and Appendix A (prompts of hundreds of small independent blocks): after an edit only
+    the edited blocks are encoded again.  A non-final block sees only itself, so encoding it alone -- as
+    a one-block sequence -- must reproduce its rows of the whole-prompt launch; checked on a prompt of
+    320 small blocks, against the whole launch (bit-identical: same tiles) and against the oracle."""
+    rng = np.random.default_rng(77)
+    lens = [int(x) for x in rng.integers(4, 48, size=320)] + [40]
+    w = W.Workload("many_small_blocks", 8, 2, 128, 5e5, lens, [len(lens)], seed=77)
+    c = ctx_for(w)
+    seg, buf = c.segment(w.block_lens, w.seq_nblocks, B.BA_MODE_BLOCK)
+    qb, kb, vb = W.prefill_inputs(w)
+    q, k, v = dev(qb), dev(kb), dev(vb)
+    o = torch.empty(w.n_tokens, w.n_q_heads, w.head_dim, device="cuda", dtype=torch.float32)
+    B.ba_block_prefill(c.ctx, q, k, v, o, None, seg, B.BA_MODE_BLOCK, B.BA_OUT_F32)
+    cu = np.concatenate([[0], np.cumsum(lens)])
+    edited = [3, 57, 58, 200, 319]
+    rows = np.concatenate([np.arange(cu[b], cu[b + 1]) for b in edited])
+    rt = torch.from_numpy(rows).cuda()
+    # the edited blocks alone: each is a sequence of one block (its final block = causal inside itself)
+    sub_lens = [lens[b] for b in edited]
+    seg2, buf2 = c.segment(sub_lens, [1] * len(edited), B.BA_MODE_BLOCK)
+    q2, k2, v2 = q[rt].contiguous(), k[rt].contiguous(), v[rt].contiguous()
+    o2 = torch.empty(len(rows), w.n_q_heads, w.head_dim, device="cuda", dtype=torch.float32)
+    B.ba_block_prefill(c.ctx, q2, k2, v2, o2, None, seg2, B.BA_MODE_BLOCK, B.BA_OUT_F32)
+    assert c.device_status() == B.BA_OK
+    assert torch.equal(o2, o[rt])
+    o_ref, _ = ob.block_prefill(W.bf16_bits_to_f64(qb), W.bf16_bits_to_f64(kb), W.bf16_bits_to_f64(vb),
+                                w.block_lens, w.seq_nblocks, B.BA_MODE_BLOCK, rows=rows)
+    check_attention(o2.cpu().numpy(), o_ref)
+    c.close()
+
+
+def test_cache_fill_and_no_position_variant():
+    """Section 2.3: after a cold prefill the keys of a block are put into the cache at positions 0..L-1
+    (Eq. 2: rotation by minus the block's start), and re-encoding them later to the same start gives
+    the prompt keys back up to bf16 rounding.  Delta 0 everywhere (the ablation without position
+    re-encoding, Section 3.3) leaves the keys bit-identical."""
+    w = W.config2()
+    c = ctx_for(w)
+    seg, buf = c.segment(w.block_lens, w.seq_nblocks, B.BA_MODE_BLOCK)
+    t = ob.segment_tables(w.block_lens, w.seq_nblocks)
+    x = W.warm_inputs(w)
+    Tc = t["n_cached_tokens"]
+    k_prompt = dev(x["k_cache"])                       # taken as keys at prompt positions
+    neg = torch.from_numpy(-t["cache_delta"]).cuda()
+    k_cached = torch.empty_like(k_prompt)
+    B.ba_reencode_k(c.ctx, k_prompt, None, Tc, k_cached, seg.cache_cu, neg, seg.n_cached_blocks, Tc)
+    ref = ob.reencode_blocks(W.bf16_bits_to_f64(x["k_cache"]), None, t["cache_cu"], -t["cache_delta"], w.rope_theta)
+    check_reencoded(R.device_to_bits(k_cached), ref)
+    zero = torch.zeros_like(neg)
+    same = torch.empty_like(k_prompt)
+    B.ba_reencode_k(c.ctx, k_prompt, None, Tc, same, seg.cache_cu, zero, seg.n_cached_blocks, Tc)
+    assert torch.equal(same, k_prompt)
+    assert c.device_status() == B.BA_OK
+    c.close()
+
+
 def test_attention_rejects_mode_mismatch_and_null():
     w = W.config1()
     c = ctx_for(w)
