@@ -171,7 +171,10 @@ ba_status ba_segment(ba_ctx *ctx, const int32_t *block_lens, const int32_t *seq_
  *            May equal k_src when src_off is NULL (in place).
  *   cu       device int32 [n_blocks+1], delta device int32 [n_blocks], src_off device int32 or NULL
  *   n_rows   rows of k_dst (>= cu[n_blocks]); rows beyond cu[n_blocks] are not touched
- * Uses n_blocks * head_dim * 4 bytes of workspace for the angle table.
+ * Uses n_blocks * head_dim * 4 bytes of workspace for the angle table.  When `delta` is the
+ * cache_delta array of the tables this context's last ba_segment() built (and n_blocks their
+ * cached-block count), the rotation table built with those tables is used instead and no table is
+ * computed; those tables must then still be alive and unchanged.
  */
 ba_status ba_reencode_k(ba_ctx *ctx, const void *k_src, const int32_t *src_off, int32_t n_src_rows,
                         void *k_dst, const int32_t *cu, const int32_t *delta, int32_t n_blocks,

@@ -123,6 +123,7 @@ ba_status ba_create(ba_ctx **out, const ba_config *cfg, int device, size_t works
   ctx->has_pending = 0;
   ctx->pending_table_bytes = 0;
   ctx->pending_stream = nullptr;
+  ctx->seg_delta = nullptr; ctx->seg_rope = nullptr; ctx->seg_rope_blocks = 0;
   ctx->workspace = nullptr;
   ctx->dev_status = nullptr;
   if (cudaMalloc(&ctx->dev_status, 256) != cudaSuccess ||
@@ -211,10 +212,16 @@ ba_status ba_segment(ba_ctx *ctx, const int32_t *block_lens, const int32_t *seq_
   out->tok_block = next(); out->tok_pos = next(); out->tok_pos_local = next();
   out->cu_qtile = next(); out->cu_ftile = next(); out->cache_tile_cu = next(); out->totals = next();
   out->cache_rope = (float *)next();
+  ctx->seg_delta = nullptr; ctx->seg_rope = nullptr; ctx->seg_rope_blocks = 0;
   ba_status st = ba_segment_launch(ctx, d_lens, d_nb, batch, n_blocks, n_tokens, mode, out, s);
   if (st != BA_OK || out->n_cached_blocks == 0) return st;
   // rotations of the cached blocks (the same angle table ba_reencode_k builds), once per prompt
-  return ba_reencode_table_launch(ctx, out->cache_delta, out->n_cached_blocks, (float2 *)out->cache_rope, s);
+  st = ba_reencode_table_launch(ctx, out->cache_delta, out->n_cached_blocks, (float2 *)out->cache_rope, s);
+  if (st == BA_OK) {
+    ctx->seg_delta = out->cache_delta; ctx->seg_rope = (const float2 *)out->cache_rope;
+    ctx->seg_rope_blocks = out->n_cached_blocks;
+  }
+  return st;
 }
 
 static ba_status check_reencode_args(ba_ctx *ctx, const void *k_src, const int32_t *src_off, int32_t n_src_rows,
@@ -247,6 +254,10 @@ ba_status ba_reencode_k(ba_ctx *ctx, const void *k_src, const int32_t *src_off, 
   ba_status st = check_reencode_args(ctx, k_src, src_off, n_src_rows, k_dst, cu, delta, n_blocks, n_rows, &nothing);
   if (st != BA_OK || nothing) return st;
   BA_CUDA_TRY(cudaSetDevice(ctx->device));
+  if (delta == ctx->seg_delta && n_blocks == ctx->seg_rope_blocks)   // the table ba_segment built is for these deltas
+    return ba_reencode_main_launch(
+        ctx, ba_make_reencode_job(ctx, k_src, src_off, n_src_rows, k_dst, cu, delta, n_blocks, n_rows, ctx->seg_rope),
+        (cudaStream_t)stream);
   float2 *table; size_t bytes;
   st = place_table(ctx, n_blocks, &table, &bytes);
   if (st != BA_OK) return st;
@@ -263,12 +274,19 @@ ba_status ba_reencode_k_deferred(ba_ctx *ctx, const void *k_src, const int32_t *
   BA_CUDA_TRY(cudaSetDevice(ctx->device));
   st = ba_flush_pending(ctx, (cudaStream_t)stream);          // one job may be queued at a time
   if (st != BA_OK) return st;
-  float2 *table; size_t bytes;
-  st = place_table(ctx, n_blocks, &table, &bytes);
-  if (st != BA_OK) return st;
-  st = ba_reencode_table_launch(ctx, delta, n_blocks, table, (cudaStream_t)stream);
-  if (st != BA_OK) return st;
-  ctx->pending = ba_make_reencode_job(ctx, k_src, src_off, n_src_rows, k_dst, cu, delta, n_blocks, n_rows, table);
+  const float2 *table_used;
+  size_t bytes = 0;
+  if (delta == ctx->seg_delta && n_blocks == ctx->seg_rope_blocks) {
+    table_used = ctx->seg_rope;
+  } else {
+    float2 *table;
+    st = place_table(ctx, n_blocks, &table, &bytes);
+    if (st != BA_OK) return st;
+    st = ba_reencode_table_launch(ctx, delta, n_blocks, table, (cudaStream_t)stream);
+    if (st != BA_OK) return st;
+    table_used = table;
+  }
+  ctx->pending = ba_make_reencode_job(ctx, k_src, src_off, n_src_rows, k_dst, cu, delta, n_blocks, n_rows, table_used);
   ctx->has_pending = 1;
   ctx->pending_table_bytes = bytes;
   ctx->pending_stream = (cudaStream_t)stream;

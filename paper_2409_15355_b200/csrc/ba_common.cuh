@@ -46,6 +46,11 @@ struct ba_ctx {
   int has_pending;
   size_t pending_table_bytes;
   cudaStream_t pending_stream;
+  // rotation table of the cached blocks built by the last ba_segment (in the caller's table buffer):
+  // a re-encoding call whose delta array is that table's cache_delta reuses it instead of rebuilding it
+  const int32_t *seg_delta;
+  const float2 *seg_rope;
+  int32_t seg_rope_blocks;
 };
 
 static inline size_t ba_align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }

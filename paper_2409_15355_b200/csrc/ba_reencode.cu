@@ -10,7 +10,8 @@
 // Kernel 1 builds that table in fp64 (angles reach tens of thousands of radians,
 // far beyond what fast fp32 sin/cos can reduce) and stores it as fp32.
 // Kernel 2 is a pure bandwidth kernel: every thread moves 16-byte vectors
-// (8 bf16), several rows in flight, rotating in fp32 and rounding once to bf16.
+// (8 bf16) and keeps its column while it walks down a few rows, rotating in fp32 and rounding
+// once to bf16; small CTAs (one row of vectors wide) measured fastest.
 #include "ba_common.cuh"
 #include "ba_reencode_dev.cuh"
 
@@ -30,17 +31,40 @@ ba_rope_table_kernel(const int32_t *__restrict__ delta, int n_blocks, int half_d
   table[i] = make_float2((float)co, (float)s);
 }
 
-#ifndef BA_REENCODE_MINB
-#define BA_REENCODE_MINB 1
+// A CTA takes kPasses consecutive groups of rows; its threads keep their column and walk down the
+// rows, kRows loads in flight each, so the per-thread set-up (column arithmetic, block search, table
+// fetch) is paid once per kPasses * kRows rows.
+#ifndef BA_REENCODE_PASSES
+#define BA_REENCODE_PASSES 4
 #endif
-template <int kLayout, int kRows>
-__global__ void __launch_bounds__(512, BA_REENCODE_MINB)
-ba_reencode_kernel(const ba_reencode_job job, int32_t *status) {
+template <int kLayout, int kRows, int kPasses>
+__global__ void __launch_bounds__(512)
+ba_reencode_kernel(const ba_reencode_job job, int units_shift, int32_t *status) {
+  // units per row is a power of two for every head count that is one (units_shift >= 0): shifts, no divisions
   const int units_per_row = (kLayout == BA_ROPE_ADJACENT) ? job.row_vecs : (job.row_vecs >> 1);
-  const int row_step = blockDim.x / units_per_row;            // blockDim.x is a multiple of units_per_row
-  const int u = threadIdx.x % units_per_row;
-  const int row0 = blockIdx.x * (row_step * kRows) + threadIdx.x / units_per_row;
-  ba_reencode_rows<kLayout, kRows>(job, u, row0, row_step, status);
+  const int row_step = units_shift >= 0 ? (int)(blockDim.x >> units_shift) : (int)(blockDim.x / units_per_row);
+  const int u = units_shift >= 0 ? (int)(threadIdx.x & (units_per_row - 1)) : (int)(threadIdx.x % units_per_row);
+  const int rsub = units_shift >= 0 ? (int)(threadIdx.x >> units_shift) : (int)(threadIdx.x / units_per_row);
+  const int total_rows = min(job.n_rows, __ldg(job.cu + job.n_blocks));
+  const int cta_row0 = blockIdx.x * (row_step * kRows * kPasses);
+  // the block of the CTA's first row is searched once and shared; the threads walk forward from it
+  __shared__ int s_c;
+  if (threadIdx.x == 0) {
+    int c = upper_bound_i32(job.cu, job.n_blocks + 1, min(cta_row0, max(total_rows - 1, 0))) - 1;
+    s_c = min(max(c, 0), job.n_blocks - 1);
+  }
+  __syncthreads();
+  int row0 = cta_row0 + rsub;
+  if (row0 >= total_rows) return;
+  ba_reencode_state st;
+  ba_reencode_state_init<kLayout>(job, u, st);
+  st.c = s_c;
+  st.c_begin = __ldg(job.cu + st.c);
+  st.c_end = __ldg(job.cu + st.c + 1);
+  st.shift = job.src_off ? (long long)__ldg(job.src_off + st.c) - st.c_begin : 0;
+#pragma unroll 1
+  for (int pass = 0; pass < kPasses && row0 < total_rows; ++pass, row0 += row_step * kRows)
+    ba_reencode_rows<kLayout, kRows>(job, st, row0, row_step, total_rows, status);
 }
 
 }  // namespace
@@ -69,20 +93,26 @@ ba_reencode_job ba_make_reencode_job(const ba_ctx *ctx, const void *k_src, const
 
 ba_status ba_reencode_main_launch(ba_ctx *ctx, const ba_reencode_job &job, cudaStream_t stream) {
 #ifndef BA_REENCODE_ROWS
-#define BA_REENCODE_ROWS 2
+#define BA_REENCODE_ROWS 1
 #endif
   constexpr int kRows = BA_REENCODE_ROWS;   // rows in flight per thread
   const bool adjacent = job.layout == BA_ROPE_ADJACENT;
   const int units = adjacent ? job.row_vecs : job.row_vecs / 2;
-  // threads per CTA: a multiple of the units per row, close to 256
-  int threads = units >= 256 ? units : (256 / units) * units;
+  // threads per CTA: a multiple of the units per row, close to BA_REENCODE_THREADS
+#ifndef BA_REENCODE_THREADS
+#define BA_REENCODE_THREADS 128
+#endif
+  int threads = units >= BA_REENCODE_THREADS ? units : (BA_REENCODE_THREADS / units) * units;
+  int units_shift = -1;                       // log2(units) when it is a power of two
+  for (int k = 0; k < 12; ++k) if ((1 << k) == units) units_shift = k;
   if (threads > 512) return BA_ERR_UNSUPPORTED;   // more than 4096 bf16 per row
-  const int rows_per_cta = (threads / units) * kRows;
+  constexpr int kPasses = BA_REENCODE_PASSES;
+  const int rows_per_cta = (threads / units) * kRows * kPasses;
   const int grid = (job.n_rows + rows_per_cta - 1) / rows_per_cta;
   if (adjacent)
-    ba_reencode_kernel<BA_ROPE_ADJACENT, kRows><<<grid, threads, 0, stream>>>(job, ctx->dev_status);
+    ba_reencode_kernel<BA_ROPE_ADJACENT, kRows, kPasses><<<grid, threads, 0, stream>>>(job, units_shift, ctx->dev_status);
   else
-    ba_reencode_kernel<BA_ROPE_HALF, kRows><<<grid, threads, 0, stream>>>(job, ctx->dev_status);
+    ba_reencode_kernel<BA_ROPE_HALF, kRows, kPasses><<<grid, threads, 0, stream>>>(job, units_shift, ctx->dev_status);
   BA_CUDA_TRY(cudaGetLastError());
   ctx->launches += 1;
   return BA_OK;
@@ -168,6 +198,7 @@ extern "C" ba_status ba_reencode_k_noalloc(const ba_config *cfg, int device, con
   tmp.has_pending = 0;
   tmp.pending_table_bytes = 0;
   tmp.pending_stream = nullptr;
+  tmp.seg_delta = nullptr; tmp.seg_rope = nullptr; tmp.seg_rope_blocks = 0;
   return ba_reencode_launch(&tmp, k_src, src_off, n_src_rows, k_dst, cu, delta, n_blocks, n_rows,
                             g_noalloc_table[device], (cudaStream_t)stream);
 }

@@ -29,86 +29,103 @@ __device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w 
 
 // ADJACENT layout: a 16-byte vector holds rotary pairs 4v..4v+3 of one head.
 // HALF layout: the vector at column c (< d/2) pairs with the vector at c + d/2, a thread moves both.
-// The calling thread owns unit `u` (one vector column, or one column pair) and handles rows
-// row0, row0 + row_step, ... (kRows of them), all loads first.
+// A thread owns unit `u` (one vector column, or one column pair) and walks down the rows; what it
+// knows about the block it is in -- bounds, source shift, delta, its (cos, sin) values -- stays in
+// registers from one row to the next and is looked up again only when a row leaves the block.
+// The source rows are read once: streaming loads keep them from displacing the re-encoded keys,
+// which the attention launch that follows reads, in L2.
+#ifndef BA_RE_LOAD
+#define BA_RE_LOAD(p) __ldcs(p)
+#endif
+struct ba_reencode_state {
+  int vec_x, vec_y, m0;              // the thread's vector column(s) and first rotary pair
+  int c, c_begin, c_end;             // block of the last row and its row range
+  long long shift;                   // source row = row + shift
+  int t_blk, t_delta;                // block whose (cos, sin) values are loaded, and its delta
+  float4 tcs[4];
+};
+
+template <int kLayout>
+__device__ __forceinline__ void ba_reencode_state_init(const ba_reencode_job &job, int u, ba_reencode_state &st) {
+  const int head_vecs = job.head_dim >> 3;                    // uint4 per head: 8 or 16
+  if (kLayout == BA_ROPE_ADJACENT) {
+    st.vec_x = u; st.vec_y = u;
+    st.m0 = (u & (head_vecs - 1)) * 4;
+  } else {
+    const int hv = head_vecs >> 1;                            // vectors per half head: 4 or 8
+    const int head = u / hv, v = u & (hv - 1);
+    st.vec_x = head * head_vecs + v;
+    st.vec_y = st.vec_x + hv;
+    st.m0 = v * 8;
+  }
+  st.c = 0; st.c_begin = 0; st.c_end = -1; st.shift = 0;
+  st.t_blk = -1; st.t_delta = 0;
+}
+
+// Rows row0, row0 + row_step, ... (kRows of them, those below total_rows), all loads first.
 template <int kLayout, int kRows>
-__device__ __forceinline__ void ba_reencode_rows(const ba_reencode_job &job, int u, int row0, int row_step,
-                                                 int32_t *status) {
+__device__ __forceinline__ void ba_reencode_rows(const ba_reencode_job &job, ba_reencode_state &st, int row0,
+                                                 int row_step, int total_rows, int32_t *status) {
   const uint4 *src = job.src;
   uint4 *dst = job.dst;
-  const int32_t *src_off = job.src_off, *cu = job.cu, *delta = job.delta;
-  const float2 *table = job.table;
+  const int32_t *src_off = job.src_off, *cu = job.cu;
   const int n_src_rows = job.n_src_rows, n_blocks = job.n_blocks, row_vecs = job.row_vecs;
   const int half_dim = job.head_dim >> 1;
-  const int head_vecs = job.head_dim >> 3;                    // uint4 per head
-  const int total_rows = min(job.n_rows, __ldg(cu + n_blocks));
-  // column of this thread's vector(s) inside the row, and its first rotary pair
-  int vec_x, vec_y, m0;
-  if (kLayout == BA_ROPE_ADJACENT) {
-    vec_x = u; vec_y = u;
-    m0 = (u % head_vecs) * 4;
-  } else {
-    int hv = head_vecs >> 1;                                  // vectors per half head
-    int head = u / hv, v = u - head * hv;
-    vec_x = head * head_vecs + v;
-    vec_y = vec_x + hv;
-    m0 = v * 8;
-  }
+  const int vec_x = st.vec_x, vec_y = st.vec_y;
 
   uint4 x[kRows], y[kRows];
   int blk[kRows];
   bool live[kRows];
-  // Rows of a thread are close together, so they usually share a block: the block of a row is
-  // looked up again only when the row leaves [c_begin, c_end).
-  int c = 0, c_begin = 0, c_end = -1;
-  long long shift = 0;                                        // source row = row + shift
 #pragma unroll
   for (int i = 0; i < kRows; ++i) {
     const int r = row0 + i * row_step;
     live[i] = r < total_rows;
     blk[i] = 0;
     if (live[i]) {
-      if (r < c_begin || r >= c_end) {
-        c = upper_bound_i32(cu, n_blocks + 1, r) - 1;
-        c = min(max(c, 0), n_blocks - 1);
-        c_begin = __ldg(cu + c);
-        c_end = __ldg(cu + c + 1);
-        shift = src_off ? (long long)__ldg(src_off + c) - c_begin : 0;
+      if (r < st.c_begin || r >= st.c_end) {
+        int c;
+        if (r >= st.c_end && st.c + 2 <= n_blocks && r < __ldg(cu + st.c + 2)) {
+          c = st.c + 1;                                       // the usual case: the next block
+        } else {
+          c = upper_bound_i32(cu, n_blocks + 1, r) - 1;
+          c = min(max(c, 0), n_blocks - 1);
+        }
+        st.c = c;
+        st.c_begin = __ldg(cu + c);
+        st.c_end = __ldg(cu + c + 1);
+        st.shift = src_off ? (long long)__ldg(src_off + c) - st.c_begin : 0;
       }
-      blk[i] = c;
-      const long long sr = r + shift;
+      blk[i] = st.c;
+      const long long sr = r + st.shift;
       if (sr < 0 || sr >= n_src_rows) {
         ba_record_status(status, BA_ERR_INVALID_ARG);
         live[i] = false;
       } else {
         const uint4 *p = src + sr * row_vecs;
-        x[i] = p[vec_x];
-        if (kLayout == BA_ROPE_HALF) y[i] = p[vec_y];
+        x[i] = BA_RE_LOAD(p + vec_x);
+        if (kLayout == BA_ROPE_HALF) y[i] = BA_RE_LOAD(p + vec_y);
       }
     }
   }
-  // (cos, sin) of this thread's rotary pairs, reloaded only when the block changes
-  int t_blk = -1, t_delta = 0;
-  float4 tcs[4];
 #pragma unroll
   for (int i = 0; i < kRows; ++i) {
     if (!live[i]) continue;
-    int r = row0 + i * row_step;
+    const int r = row0 + i * row_step;
     uint4 *q = dst + (long long)r * row_vecs;
-    if (blk[i] != t_blk) {
-      t_blk = blk[i];
-      t_delta = __ldg(delta + t_blk);
-      const float4 *t4 = reinterpret_cast<const float4 *>(table + t_blk * half_dim + m0);
-      tcs[0] = __ldg(t4); tcs[1] = __ldg(t4 + 1);
-      if (kLayout == BA_ROPE_HALF) { tcs[2] = __ldg(t4 + 2); tcs[3] = __ldg(t4 + 3); }
+    if (blk[i] != st.t_blk) {                    // (cos, sin) of this thread's rotary pairs in the new block
+      st.t_blk = blk[i];
+      st.t_delta = __ldg(job.delta + st.t_blk);
+      const float4 *t4 = reinterpret_cast<const float4 *>(job.table + st.t_blk * half_dim + st.m0);
+      st.tcs[0] = __ldg(t4); st.tcs[1] = __ldg(t4 + 1);
+      if (kLayout == BA_ROPE_HALF) { st.tcs[2] = __ldg(t4 + 2); st.tcs[3] = __ldg(t4 + 3); }
     }
-    if (t_delta == 0) {                          // identity: copy bit-exactly
+    if (st.t_delta == 0) {                       // identity: copy bit-exactly
       q[vec_x] = x[i];
       if (kLayout == BA_ROPE_HALF) q[vec_y] = y[i];
       continue;
     }
     if (kLayout == BA_ROPE_ADJACENT) {
-      const float4 a = tcs[0], b = tcs[1];                      // two (cos,sin) pairs per float4
+      const float4 a = st.tcs[0], b = st.tcs[1];              // two (cos,sin) pairs per float4
       uint32_t w[4] = {x[i].x, x[i].y, x[i].z, x[i].w};
       float2 cs[4] = {make_float2(a.x, a.y), make_float2(a.z, a.w), make_float2(b.x, b.y), make_float2(b.z, b.w)};
       uint32_t o[4];
@@ -125,7 +142,7 @@ __device__ __forceinline__ void ba_reencode_rows(const ba_reencode_job &job, int
       uint32_t ox[4], oy[4];
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
-        const float4 cs = tcs[j];                             // pairs m0+2j, m0+2j+1
+        const float4 cs = st.tcs[j];                          // pairs m0+2j, m0+2j+1
         float x0, y0, x1, y1;
         rot2(bf16_lo(wx[j]), bf16_lo(wy[j]), make_float2(cs.x, cs.y), x0, y0);
         rot2(bf16_hi(wx[j]), bf16_hi(wy[j]), make_float2(cs.z, cs.w), x1, y1);
