@@ -492,7 +492,8 @@ def test_deferred_reencode_rides_along_with_attention(w, layout):
     B.ba_block_prefill(c.ctx, q, k, v, o_plain, None, seg, B.BA_MODE_BLOCK, B.BA_OUT_F32)
     got = torch.zeros_like(want)
     n0 = c.launches()
-    B.ba_reencode_k_deferred(c.ctx, src, off, src.shape[0], got, seg.cache_cu, seg.cache_delta, seg.n_cached_blocks, Tc)
+    own_delta = torch.from_numpy(t["cache_delta"]).cuda()  # not the tables' array: the call builds its own angle table
+    B.ba_reencode_k_deferred(c.ctx, src, off, src.shape[0], got, seg.cache_cu, own_delta, seg.n_cached_blocks, Tc)
     assert c.launches() == n0 + 1                       # only the angle table so far
     torch.cuda.synchronize()
     assert not got.any()                                # nothing written yet
@@ -503,7 +504,9 @@ def test_deferred_reencode_rides_along_with_attention(w, layout):
     assert torch.equal(o_with, o_plain)
     # ba_flush runs a queued job on its own; a second flush is a no-op
     got2 = torch.zeros_like(want)
+    n2 = c.launches()
     B.ba_reencode_k_deferred(c.ctx, src, off, src.shape[0], got2, seg.cache_cu, seg.cache_delta, seg.n_cached_blocks, Tc)
+    assert c.launches() == n2                           # with the tables' own deltas the table ba_segment built is reused
     B.ba_flush(c.ctx)
     n1 = c.launches()
     B.ba_flush(c.ctx)
