@@ -68,12 +68,6 @@ constexpr int kWorkSlots = 4;      // ring of published work entries (power of t
 #ifndef BA_SVC_REGS
 #define BA_SVC_REGS 72
 #endif
-// BA_SPLIT_S = 1: S of a query tile is computed, exponentiated and consumed in two halves of 64 keys,
-// each with its own tensor-memory columns and barriers, so that QK^T of one half runs while the other
-// half is in the softmax (plain path only).
-#ifndef BA_SPLIT_S
-#define BA_SPLIT_S 0
-#endif
 // the MMA thread's loops over the two query tiles
 #ifndef BA_T_UNROLL
 #define BA_T_UNROLL _Pragma("unroll")
@@ -129,7 +123,7 @@ struct Ctrl {
   uint64_t q_empty;               // every QK^T of the current item has completed: Q may be reloaded
   uint64_t kv_full[kStages];
   uint64_t kv_empty[kStages];
-  uint64_t s_full[2][2];          // [query tile][half of the key tile] (only [t][0] unless S is split)
+  uint64_t s_full[2];
   uint64_t p_full[2][2];          // [query tile][half of the P tile]
   uint64_t o_done[2];
   uint64_t o_free[2];             // the softmax warps have read O_t out of tensor memory
@@ -140,7 +134,6 @@ struct Ctrl {
   uint32_t tmem_base;
   int abort_flag;
   uint64_t qr_full[2][2];         // fused: [query tile][buffer] the tile prepared for the next key range is ready
-  uint64_t pv_done[2];            // split S: one arrival per PV half of query tile t completed
   uint64_t cs_full[2];            // fused: the block's (cos, sin) row has been staged for softmax group t
   uint64_t qraw_full[2];          // fused: the plain query tile t has landed in the buffer of the version being prepared
 };
@@ -354,7 +347,6 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
                        const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ CUtensorMap tmap_kc,
                        const __grid_constant__ CUtensorMap tmap_vc, const AttnParams p) {
   using L = Layout<D>;
-  constexpr bool kSplitS = BA_SPLIT_S && !kFused;
   // setmaxnreg is a warpgroup-wide instruction: the four service warps (8-11) must ask for the same count
   constexpr int kProdRegs = BA_SVC_REGS, kMmaRegs = BA_SVC_REGS, kSpareRegs = BA_SVC_REGS;
   extern __shared__ uint8_t smem_raw[];
@@ -369,10 +361,9 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
     mbar_init(&ctrl->q_full[0], 1); mbar_init(&ctrl->q_full[1], 1); mbar_init(&ctrl->q_empty, 1);
     for (int s = 0; s < kStages; ++s) { mbar_init(&ctrl->kv_full[s], 1); mbar_init(&ctrl->kv_empty[s], 1); }
     for (int t = 0; t < 2; ++t) {
-      mbar_init(&ctrl->s_full[t][0], 1); mbar_init(&ctrl->s_full[t][1], 1); mbar_init(&ctrl->p_full[t][0], 128); mbar_init(&ctrl->p_full[t][1], 128);
+      mbar_init(&ctrl->s_full[t], 1); mbar_init(&ctrl->p_full[t][0], 128); mbar_init(&ctrl->p_full[t][1], 128);
       mbar_init(&ctrl->o_done[t], 1); mbar_init(&ctrl->o_free[t], 128);
       mbar_init(&ctrl->qr_full[t][0], 4); mbar_init(&ctrl->qr_full[t][1], 4); mbar_init(&ctrl->cs_full[t], D / 2);
-      mbar_init(&ctrl->pv_done[t], 1);
       mbar_init(&ctrl->qraw_full[t], 1);
     }
     for (int k = 0; k < kWorkSlots; ++k) { mbar_init(&ctrl->work_full[k], 1); mbar_init(&ctrl->work_empty[k], 9); }
@@ -492,7 +483,7 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
     if (elect_one()) {
       const uint32_t tS[2] = {tmem, tmem + 128};
       const uint32_t tO[2] = {tmem + 256, tmem + 384};
-      constexpr uint32_t idesc_qk = make_idesc_bf16(128, kSplitS ? kBlockN / 2 : kBlockN, 0);
+      constexpr uint32_t idesc_qk = make_idesc_bf16(128, kBlockN, 0);
       constexpr uint32_t idesc_pv = make_idesc_bf16(128, D, 1);
       const uint32_t q_addr[2] = {smem_u32(smem + L::kQ0), smem_u32(smem + L::kQ1)};
       const uint32_t ring = smem_u32(smem + L::kRing);
@@ -502,24 +493,21 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
       const uint64_t q_desc[2] = {make_smem_desc(q_addr[0], 16, 1024), make_smem_desc(q_addr[1], 16, 1024)};
       const uint64_t k_desc0 = make_smem_desc(ring, 16, 1024);
       const uint64_t v_desc0 = make_smem_desc(ring, L::kRegionBytes, 1024);
-      // h: half of the key tile when S is split (keys 64 h .. 64 h + 63, S columns 64 h ..), else 0
-      auto issue_qk_with = [&](int t, int h, int idx, uint64_t qd) {
-        const uint64_t kd = k_desc0 + (uint64_t)(((idx % kStages) * L::kTileBytes + h * 64 * 128) >> 4);
+      auto issue_qk_with = [&](int t, int idx, uint64_t qd) {
+        const uint64_t kd = k_desc0 + (uint64_t)(((idx % kStages) * L::kTileBytes) >> 4);
 #pragma unroll
         for (int k = 0; k < D / 16; ++k) {
           const uint64_t off = (uint64_t)(((k >> 2) * L::kRegionBytes + (k & 3) * 32) >> 4);
-          mma_ss(tS[t] + h * 64, qd + off, kd + off, idesc_qk, k > 0);
+          mma_ss(tS[t], qd + off, kd + off, idesc_qk, k > 0);
         }
-        mma_commit(&ctrl->s_full[t][h]);
+        mma_commit(&ctrl->s_full[t]);
       };
-      // half = 0: keys 0..63 of the tile, half = 1: keys 64..127; P of a half sits at the start of the
-      // S columns it was computed from
+      // half = 0: keys 0..63 of the tile, half = 1: keys 64..127
       auto issue_pv = [&](int t, int idx, bool first, int half) {
         const uint64_t vd = v_desc0 + (uint64_t)(((idx % kStages) * L::kTileBytes) >> 4);
 #pragma unroll
         for (int k = half * 4; k < half * 4 + 4; ++k)
-          mma_ts(tO[t], tS[t] + (kSplitS ? half * 64 + (k - half * 4) * 8 : k * 8), vd + (uint64_t)((k * 2048) >> 4), idesc_pv,
-                 (!first || k > 0) ? 1u : 0u);
+          mma_ts(tO[t], tS[t] + k * 8, vd + (uint64_t)((k * 2048) >> 4), idesc_pv, (!first || k > 0) ? 1u : 0u);
       };
       int gidx = 0;                        // K/V tiles consumed so far (ring position)
       int q_uses[2] = {0, 0};              // items in which query tile t was loaded
@@ -539,11 +527,7 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
       int cached_end = 0;                  // tiles [tile0, cached_end) of the entry are cached keys
       // S_t = Q_t K^T for tile `jrel` of the entry, whose keys sit at ring position idx
       auto issue_qk = [&](int t, int jrel, int idx) -> bool {
-        if (!kFused) {
-          issue_qk_with(t, 0, idx, q_desc[t]);
-          if (kSplitS) issue_qk_with(t, 1, idx, q_desc[t]);     // entry start: both halves at once
-          return true;
-        }
+        if (!kFused) { issue_qk_with(t, idx, q_desc[t]); return true; }
         const int jt = wk.tile0 + jrel;
         bool change = false;
         if (jt < cached_end) {
@@ -565,7 +549,7 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
           ++n_ver[t];
           tc_fence_after();
         }
-        issue_qk_with(t, 0, idx, ((n_ver[t] - 1) & 1) ? qb_desc[t] : q_desc[t]);
+        issue_qk_with(t, idx, ((n_ver[t] - 1) & 1) ? qb_desc[t] : q_desc[t]);
         return true;
       };
       for (;;) {
@@ -611,23 +595,19 @@ BA_T_UNROLL
             tc_fence_after();
             BA_TR(2, j, t * 4 + 1);
             issue_pv(t, iv, j == 0, 0);
-            if (kSplitS) mma_commit(&ctrl->pv_done[t]);
             // K_(j+1) is needed right after the second half of PV: make sure of it while P is still
             // being finished, off the critical path
             if (t == 0 && !last) { BA_TR(3, j, 2); ok = wait_kv(ik); if (!ok) continue; BA_TR(3, j, 3); }
-            if (kSplitS && !last) issue_qk_with(t, 0, ik, q_desc[t]);   // its S columns are free again
             ok = mbar_wait(&ctrl->p_full[t][1], p_uses[t] & 1, abort_flag);
             if (!ok) continue;
             tc_fence_after();
             issue_pv(t, iv, j == 0, 1);
-            if (kSplitS) mma_commit(&ctrl->pv_done[t]);
             ++p_uses[t];
             BA_TR(2, j, t * 4 + 2);
             if (last) mma_commit(&ctrl->o_done[t]);
             if (t + 1 == n_qt) mma_commit(&ctrl->kv_empty[iv % kStages]);
             if (!last) {
-              if (kSplitS) issue_qk_with(t, 1, ik, q_desc[t]);
-              else ok = issue_qk(t, j + 1, ik);
+              ok = issue_qk(t, j + 1, ik);
               if (!ok) continue;
               BA_TR(2, j, t * 4 + 3);
               if (t + 1 == n_qt) {
@@ -669,7 +649,6 @@ BA_T_UNROLL
     int o_uses = 0;                       // items in which this query tile was active
     int n_staged = 0;                     // fused: (cos, sin) rows staged so far by this group
     int n_made = 0;                       // fused: versions of this query tile prepared so far
-    int n_handed = 0;                     // split S: halves of P handed to the MMA thread so far
     int tiles_before = 0;                 // key tiles of all earlier items (the producer counts the same way)
     bool ok = true;
     Work wk;
@@ -753,89 +732,8 @@ BA_T_UNROLL
       }
 
       for (int j = 0; j < n_tiles; ++j) {
-        if (kSplitS) {
-          // S arrives, is exponentiated and handed back in two halves of 64 keys, each a small tile of
-          // the online softmax.  O may only be rescaled once the PV products handed over so far have
-          // completed (at most one is outstanding when a half of S arrives).
-          int lim;
-          const int jt = tile0 + j;
-          if (jt < it.n_cache_tiles) lim = p.walk ? ctrl->tile_valid[(tiles_before + j) & 7] - 1
-                                                  : it.cache_len - jt * kBlockN - 1;
-          else lim = tok_c - (it.own_row0 + (jt - it.n_cache_tiles) * kBlockN);
-#pragma unroll
-          for (int h = 0; h < 2; ++h) {
-            ok = mbar_wait(&ctrl->s_full[t][h], s_uses & 1, abort_flag);
-            if (!ok) break;
-            tc_fence_after();
-            uint32_t s[64];
-            tmem_ld_32x32b_x32(tS + h * 64, *reinterpret_cast<uint32_t(*)[32]>(&s[0]));
-            tmem_ld_32x32b_x32(tS + h * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&s[32]));
-            tmem_wait_ld();
-            const int limh = lim - h * 64;
-            if (limh < 63) {
-#pragma unroll
-              for (int c = 0; c < 64; ++c)
-                if (c > limh) s[c] = 0xff800000u;               // -inf
-            }
-            float mx8[8];
-#pragma unroll
-            for (int i = 0; i < 8; ++i) mx8[i] = fmaxf(__uint_as_float(s[i]), __uint_as_float(s[8 + i]));
-#pragma unroll
-            for (int c = 16; c < 64; c += 16)
-#pragma unroll
-              for (int i = 0; i < 8; ++i) mx8[i] = max3(mx8[i], __uint_as_float(s[c + i]), __uint_as_float(s[c + 8 + i]));
-            const float mx = fmaxf(max3(mx8[0], mx8[1], mx8[2]), max3(max3(mx8[3], mx8[4], mx8[5]), mx8[6], mx8[7]));
-            const float m_new = fmaxf(m_used, mx);
-            if (j == 0 && h == 0) {
-              m_used = m_new;
-            } else {
-              const bool grow = (m_new - m_used) * sl > kRescaleThreshold;
-              if (__any_sync(0xffffffffu, grow)) {
-                ok = mbar_wait(&ctrl->pv_done[t], (n_handed - 1) & 1, abort_flag);   // the last PV handed over
-                if (!ok) break;
-                tc_fence_after();
-                const float alpha = (m_new == -INFINITY) ? 1.f : ex2((m_used - m_new) * sl);
-                m_used = m_new;
-                l *= alpha;
-#pragma unroll
-                for (int c = 0; c < D / 32; ++c) {
-                  uint32_t o[32];
-                  tmem_ld_32x32b_x32(tO + c * 32, o);
-                  tmem_wait_ld();
-#pragma unroll
-                  for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
-                  tmem_st_32x32b_x32(tO + c * 32, o);
-                }
-              }
-            }
-            const float neg_m = (m_used == -INFINITY) ? 0.f : -m_used * sl;
-            uint64_t sum2[4] = {0ull, 0ull, 0ull, 0ull};
-            const uint64_t sl2 = pack2(sl, sl), negm2 = pack2(neg_m, neg_m);
-            uint32_t pk[32];
-#pragma unroll
-            for (int i = 0; i < 32; ++i) {
-              float x0, x1;
-              unpack2(fma2(pack2(__uint_as_float(s[2 * i]), __uint_as_float(s[2 * i + 1])), sl2, negm2), x0, x1);
-              const float p0 = ex2(x0), p1 = ex2(x1);
-              sum2[i & 3] = add2(sum2[i & 3], pack2(p0, p1));
-              __nv_bfloat162 v = __floats2bfloat162_rn(p0, p1);
-              pk[i] = *reinterpret_cast<uint32_t *>(&v);
-            }
-            tmem_st_32x32b_x32(tS + h * 64, pk);
-            tmem_wait_st();
-            tc_fence_before();
-            mbar_arrive(&ctrl->p_full[t][h]);
-            ++n_handed;
-            float sa, sb;
-#pragma unroll
-            for (int i = 0; i < 4; ++i) { unpack2(sum2[i], sa, sb); l += sa + sb; }
-          }
-          if (!ok) break;
-          ++s_uses;
-          continue;
-        }
         if (r == 0) BA_TR(t, j, 0);
-        ok = mbar_wait(&ctrl->s_full[t][0], s_uses & 1, abort_flag);
+        ok = mbar_wait(&ctrl->s_full[t], s_uses & 1, abort_flag);
         if (!ok) break;
         ++s_uses;
         tc_fence_after();
