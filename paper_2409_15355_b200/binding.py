@@ -60,7 +60,7 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     if _lib is not None and path is None:
         return _lib
     if path is None:
-        path = _build.build()
+        path = os.environ.get("BA_LIBRARY") or _build.build()   # BA_LIBRARY: use this prebuilt library as it is
     if not os.path.exists(path):
         raise FileNotFoundError(f"CUDA library not found: {path}")
     lib = C.CDLL(path)
