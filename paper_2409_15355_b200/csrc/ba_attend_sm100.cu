@@ -184,12 +184,6 @@ __device__ __forceinline__ uint64_t exp2_poly2(uint64_t x2) {
 #ifndef BA_POLY_PERIOD
 #define BA_POLY_PERIOD 0
 #endif
-// BA_SPEC_MAX = 1: from an item's second key tile on, the exponentials of the first half of a row start
-// against the running maximum in use, beside the row-maximum reduction, instead of after it.
-#ifndef BA_SPEC_MAX
-#define BA_SPEC_MAX 1
-#endif
-constexpr bool kSpecMax = BA_SPEC_MAX;
 #ifndef BA_SPLIT_P
 #define BA_SPLIT_P 1
 #endif
@@ -761,104 +755,74 @@ BA_T_UNROLL
             if (c > lim) s[c] = 0xff800000u;                 // -inf
         }
         // eight independent running maxima (three-input max) keep the dependency chains short
-        auto row_max = [&]() {
-          float mx8[8];
+        float mx8[8];
 #pragma unroll
-          for (int i = 0; i < 8; ++i) mx8[i] = fmaxf(__uint_as_float(s[i]), __uint_as_float(s[8 + i]));
+        for (int i = 0; i < 8; ++i) mx8[i] = fmaxf(__uint_as_float(s[i]), __uint_as_float(s[8 + i]));
 #pragma unroll
-          for (int c = 16; c < 128; c += 16)
+        for (int c = 16; c < 128; c += 16)
 #pragma unroll
-            for (int i = 0; i < 8; ++i) mx8[i] = max3(mx8[i], __uint_as_float(s[c + i]), __uint_as_float(s[c + 8 + i]));
-          return fmaxf(max3(mx8[0], mx8[1], mx8[2]), max3(max3(mx8[3], mx8[4], mx8[5]), mx8[6], mx8[7]));
-        };
-        // the running maximum moves to m_new: rescale what has been accumulated (l here, O in tensor memory)
-        auto rescale_to = [&](float m_new) {
-          // 1 when this row's maximum did not move (also when the row has seen no key yet)
-          const float alpha = (m_new == -INFINITY) ? 1.f : ex2((m_used - m_new) * sl);
+          for (int i = 0; i < 8; ++i) mx8[i] = max3(mx8[i], __uint_as_float(s[c + i]), __uint_as_float(s[c + 8 + i]));
+        const float mx = fmaxf(max3(mx8[0], mx8[1], mx8[2]), max3(max3(mx8[3], mx8[4], mx8[5]), mx8[6], mx8[7]));
+        const float m_new = fmaxf(m_used, mx);
+        if (r == 0) BA_TR(t, j, 3);
+        if (j == 0) {
           m_used = m_new;
-          l *= alpha;
+        } else {
+          const bool grow = (m_new - m_used) * sl > kRescaleThreshold;
+          if (__any_sync(0xffffffffu, grow)) {
+            // 1 when this row's maximum did not move (also when the row has seen no key yet)
+            const float alpha = (m_new == -INFINITY) ? 1.f : ex2((m_used - m_new) * sl);
+            m_used = m_new;
+            l *= alpha;
 #pragma unroll
-          for (int c = 0; c < D / 32; ++c) {
-            uint32_t o[32];
-            tmem_ld_32x32b_x32(tO + c * 32, o);
-            tmem_wait_ld();
+            for (int c = 0; c < D / 32; ++c) {
+              uint32_t o[32];
+              tmem_ld_32x32b_x32(tO + c * 32, o);
+              tmem_wait_ld();
 #pragma unroll
-            for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
-            tmem_st_32x32b_x32(tO + c * 32, o);
+              for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+              tmem_st_32x32b_x32(tO + c * 32, o);
+            }
           }
-        };
+        }
+        const float neg_m = (m_used == -INFINITY) ? 0.f : -m_used * sl;   // no visible key so far: every p is 0
         uint64_t sum2[4] = {0ull, 0ull, 0ull, 0ull};       // packed (0.f, 0.f)
-        const uint64_t sl2 = pack2(sl, sl);
-        // exponentials of one half of the row (keys 64 h ..), packed fp32x2 arithmetic
-        auto exp_half = [&](auto poly_tag, int h, uint64_t negm2, uint32_t (&pk)[32], uint64_t (&acc)[4]) {
+        const uint64_t sl2 = pack2(sl, sl), negm2 = pack2(neg_m, neg_m);
+        // P is handed to the MMA warp in two halves so that PV can start on the first 64 keys
+        // while the second 64 are still being exponentiated.  The arithmetic is packed fp32x2.
+        auto exp_halves = [&](auto poly_tag) {
           constexpr bool kPoly = decltype(poly_tag)::value;
 #pragma unroll
-          for (int i = 0; i < 32; ++i) {
-            const int e0 = h * 64 + 2 * i, e1 = e0 + 1;
-            const uint64_t x2 = fma2(pack2(__uint_as_float(s[e0]), __uint_as_float(s[e1])), sl2, negm2);
-            float p0, p1;
-            if (kPoly && i % (kPolyPeriod > 0 ? kPolyPeriod : 1) == kPolyPeriod - 1) {
-              unpack2(exp2_poly2(x2), p0, p1);
-            } else {
-              float x0, x1;
-              unpack2(x2, x0, x1);
-              p0 = ex2(x0); p1 = ex2(x1);
-            }
-            acc[i & 3] = add2(acc[i & 3], pack2(p0, p1));
-            __nv_bfloat162 v = __floats2bfloat162_rn(p0, p1);
-            pk[i] = *reinterpret_cast<uint32_t *>(&v);
-          }
-        };
-        // P is handed to the MMA warp in two halves so that PV can start on the first 64 keys
-        // while the second 64 are still being exponentiated.
-        auto hand_over = [&](int h, const uint32_t (&pk)[32]) {
-          tmem_st_32x32b_x32(tS + h * 32, pk);
-          if (kSplitP || h == 1) {
-            tmem_wait_st();
-            tc_fence_before();
-            if (!kSplitP) mbar_arrive(&ctrl->p_full[t][0]);
-            mbar_arrive(&ctrl->p_full[t][h]);
-          }
-          if (r == 0) BA_TR(t, j, 4 + h);
-        };
-        auto neg_of = [&](float m) { return (m == -INFINITY) ? 0.f : -m * sl; };   // no visible key so far: every p is 0
-        auto tile = [&](auto poly_tag) {
-          uint32_t pk[32];
-          if (j == 0 || !kSpecMax) {
-            // the maximum first, then the exponentials
-            const float m_new = fmaxf(m_used, row_max());
-            if (r == 0) BA_TR(t, j, 3);
-            if (j == 0) m_used = m_new;
-            else if (__any_sync(0xffffffffu, (m_new - m_used) * sl > kRescaleThreshold)) rescale_to(m_new);
-            const float neg_m = neg_of(m_used);
-            exp_half(poly_tag, 0, pack2(neg_m, neg_m), pk, sum2);
-          } else {
-            // The maximum rarely moves by more than the threshold: the first half is exponentiated
-            // against the maximum in use while the row maximum is formed beside it (independent
-            // work, so the two interleave); if some row of the warp does need the rescaling, that
-            // half is done again.  The results are the same as with the maximum taken first.
-            uint64_t acc[4] = {0ull, 0ull, 0ull, 0ull};
-            const float neg_old = neg_of(m_used);
-            exp_half(poly_tag, 0, pack2(neg_old, neg_old), pk, acc);
-            const float m_new = fmaxf(m_used, row_max());
-            if (r == 0) BA_TR(t, j, 3);
-            if (__any_sync(0xffffffffu, (m_new - m_used) * sl > kRescaleThreshold)) {
-              rescale_to(m_new);
-              const float neg_m = neg_of(m_used);
+          for (int h = 0; h < 2; ++h) {
+            uint32_t pk[32];
 #pragma unroll
-              for (int i = 0; i < 4; ++i) acc[i] = 0ull;
-              exp_half(poly_tag, 0, pack2(neg_m, neg_m), pk, acc);
+            for (int i = 0; i < 32; ++i) {
+              const int e0 = h * 64 + 2 * i, e1 = e0 + 1;
+              const uint64_t x2 = fma2(pack2(__uint_as_float(s[e0]), __uint_as_float(s[e1])), sl2, negm2);
+              float p0, p1;
+              if (kPoly && i % (kPolyPeriod > 0 ? kPolyPeriod : 1) == kPolyPeriod - 1) {
+                unpack2(exp2_poly2(x2), p0, p1);
+              } else {
+                float x0, x1;
+                unpack2(x2, x0, x1);
+                p0 = ex2(x0); p1 = ex2(x1);
+              }
+              sum2[i & 3] = add2(sum2[i & 3], pack2(p0, p1));
+              __nv_bfloat162 v = __floats2bfloat162_rn(p0, p1);
+              pk[i] = *reinterpret_cast<uint32_t *>(&v);
             }
-#pragma unroll
-            for (int i = 0; i < 4; ++i) sum2[i] = add2(sum2[i], acc[i]);
+            tmem_st_32x32b_x32(tS + h * 32, pk);
+            if (kSplitP || h == 1) {
+              tmem_wait_st();
+              tc_fence_before();
+              if (!kSplitP) mbar_arrive(&ctrl->p_full[t][0]);
+              mbar_arrive(&ctrl->p_full[t][h]);
+            }
+            if (r == 0) BA_TR(t, j, 4 + h);
           }
-          hand_over(0, pk);
-          const float neg_m = neg_of(m_used);
-          exp_half(poly_tag, 1, pack2(neg_m, neg_m), pk, sum2);
-          hand_over(1, pk);
         };
-        if (kPolyPeriod > 0 && __all_sync(0xffffffffu, lim >= kBlockN - 1)) tile(std::true_type{});
-        else tile(std::false_type{});
+        if (kPolyPeriod > 0 && __all_sync(0xffffffffu, lim >= kBlockN - 1)) exp_halves(std::true_type{});
+        else exp_halves(std::false_type{});
         // P of this tile is with the tensor core: time to work on the next version of the query row
         if (kFused && next_start < tile_end) {
           const bool due = tile0 + j + 1 == next_start;    // the next tile is the first to need it
