@@ -352,6 +352,31 @@ def run_ours(args):
         assert ctx4.device_status() == B.BA_OK
         ctx4.close()
         del q4, k4, v4, o4
+        # the 32K prompt of the metric's workload encoded cold, under the full causal mask and under the
+        # Block-attention mask (same tensors, one launch each): the paper's FLOPs / latency comparison
+        T3 = w.n_tokens
+        g.manual_seed(3003)
+        q3 = torch.randn(T3, w.n_q_heads, w.head_dim, device=dev, generator=g).bfloat16()
+        k3 = torch.randn(T3, w.n_kv_heads, w.head_dim, device=dev, generator=g).bfloat16()
+        v3 = torch.randn(T3, w.n_kv_heads, w.head_dim, device=dev, generator=g).bfloat16()
+        o3 = torch.empty_like(q3)
+        p32 = {"workload": "cfg3 prompt (32 x 1000 + 768 tokens) encoded cold, one ba_block_prefill launch per mode"}
+        for name, mode, omode in (("full_causal", B.BA_MODE_FULL, ob.MODE_FULL), ("block", B.BA_MODE_BLOCK, ob.MODE_BLOCK)):
+            seg3 = B.ba_segment(ctx.ctx, lens, nb, 1, len(lens), T3, mode, tbuf)
+            for _ in range(2):
+                B.ba_block_prefill(ctx.ctx, q3, k3, v3, o3, None, seg3, mode, B.BA_OUT_BF16)
+            torch.cuda.synchronize()
+            ev0.record(stream)
+            for _ in range(5):
+                B.ba_block_prefill(ctx.ctx, q3, k3, v3, o3, None, seg3, mode, B.BA_OUT_BF16)
+            ev1.record(stream)
+            torch.cuda.synchronize()
+            ms3 = ev0.elapsed_time(ev1) / 5
+            fl3 = 4.0 * w.head_dim * w.n_q_heads * ob.allowed_pairs(w.block_lens, w.seq_nblocks, omode)
+            p32[name] = {"ms": ms3, "algorithmic_flops": fl3, "tflops": fl3 / ms3 / 1e9}
+        prefill["prompt_32k"] = p32
+        assert ctx.device_status() == B.BA_OK
+        del q3, k3, v3, o3
 
     # ---- secondary number: the fused warm path (keys as cached, queries counter-rotated per block in
     # the attention launch, no re-encoding pass) on the same 32-layer workload, and both paths with a
