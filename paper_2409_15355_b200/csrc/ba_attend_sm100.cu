@@ -904,7 +904,8 @@ BA_T_UNROLL
 
 // Merge of split-KV partial results: o = sum_s w_s o_s / sum_s w_s with w_s = exp(lse_s - max lse).
 // One thread per 4 output columns; the order of the sum is fixed, so results are run-to-run stable.
-template <int D>
+// kNS > 0: the number of splits is known at compile time and every load is issued before the first use.
+template <int D, int kNS>
 __global__ void __launch_bounds__(256)
 ba_combine_splits_kernel(const float *__restrict__ o_part, const float *__restrict__ lse_part, void *o, float *lse,
                          int n_rows_heads, int n_splits, int out_f32) {
@@ -912,16 +913,33 @@ ba_combine_splits_kernel(const float *__restrict__ o_part, const float *__restri
   constexpr int kVec = D / 4;
   const int rh = idx / kVec, v = idx - rh * kVec;
   if (rh >= n_rows_heads) return;
-  float mx = -INFINITY;
-  for (int s = 0; s < n_splits; ++s) mx = fmaxf(mx, __ldg(lse_part + (size_t)s * n_rows_heads + rh));
-  float den = 0.f;
+  float den = 0.f, mx = -INFINITY;
   float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-  for (int s = 0; s < n_splits; ++s) {
-    const float ls = __ldg(lse_part + (size_t)s * n_rows_heads + rh);
-    const float w = (ls == -INFINITY) ? 0.f : __expf(ls - mx);
-    const float4 x = __ldg(reinterpret_cast<const float4 *>(o_part + ((size_t)s * n_rows_heads + rh) * D) + v);
-    den += w;
-    acc.x = fmaf(w, x.x, acc.x); acc.y = fmaf(w, x.y, acc.y); acc.z = fmaf(w, x.z, acc.z); acc.w = fmaf(w, x.w, acc.w);
+  if (kNS > 0) {
+    float ls[kNS > 0 ? kNS : 1];
+    float4 x[kNS > 0 ? kNS : 1];
+#pragma unroll
+    for (int s = 0; s < kNS; ++s) {
+      ls[s] = __ldg(lse_part + (size_t)s * n_rows_heads + rh);
+      x[s] = __ldcs(reinterpret_cast<const float4 *>(o_part + ((size_t)s * n_rows_heads + rh) * D) + v);
+    }
+#pragma unroll
+    for (int s = 0; s < kNS; ++s) mx = fmaxf(mx, ls[s]);
+#pragma unroll
+    for (int s = 0; s < kNS; ++s) {
+      const float w = (ls[s] == -INFINITY) ? 0.f : __expf(ls[s] - mx);
+      den += w;
+      acc.x = fmaf(w, x[s].x, acc.x); acc.y = fmaf(w, x[s].y, acc.y); acc.z = fmaf(w, x[s].z, acc.z); acc.w = fmaf(w, x[s].w, acc.w);
+    }
+  } else {
+    for (int s = 0; s < n_splits; ++s) mx = fmaxf(mx, __ldg(lse_part + (size_t)s * n_rows_heads + rh));
+    for (int s = 0; s < n_splits; ++s) {
+      const float ls = __ldg(lse_part + (size_t)s * n_rows_heads + rh);
+      const float w = (ls == -INFINITY) ? 0.f : __expf(ls - mx);
+      const float4 x = __ldg(reinterpret_cast<const float4 *>(o_part + ((size_t)s * n_rows_heads + rh) * D) + v);
+      den += w;
+      acc.x = fmaf(w, x.x, acc.x); acc.y = fmaf(w, x.y, acc.y); acc.z = fmaf(w, x.z, acc.z); acc.w = fmaf(w, x.w, acc.w);
+    }
   }
   const float inv = 1.f / den;
   acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
@@ -1106,10 +1124,20 @@ ba_status ba_attend_sm100_launch(ba_ctx *ctx, const ba_attend_args &a, const ba_
     const int n_rh = a.n_q_rows * Hq;
     const long long threads = (long long)n_rh * (D / 4);
     const unsigned cgrid = (unsigned)((threads + 255) / 256);
-    if (D == 128)
-      ba_combine_splits_kernel<128><<<cgrid, 256, 0, stream>>>(p.o_part, p.lse_part, a.o, a.lse, n_rh, n_splits, a.out_f32);
-    else
-      ba_combine_splits_kernel<64><<<cgrid, 256, 0, stream>>>(p.o_part, p.lse_part, a.o, a.lse, n_rh, n_splits, a.out_f32);
+    auto launch = [&](auto kern) {
+      kern<<<cgrid, 256, 0, stream>>>(p.o_part, p.lse_part, a.o, a.lse, n_rh, n_splits, a.out_f32);
+    };
+    if (D == 128) {
+      if (n_splits == 2) launch(ba_combine_splits_kernel<128, 2>);
+      else if (n_splits == 3) launch(ba_combine_splits_kernel<128, 3>);
+      else if (n_splits == 4) launch(ba_combine_splits_kernel<128, 4>);
+      else launch(ba_combine_splits_kernel<128, 0>);
+    } else {
+      if (n_splits == 2) launch(ba_combine_splits_kernel<64, 2>);
+      else if (n_splits == 3) launch(ba_combine_splits_kernel<64, 3>);
+      else if (n_splits == 4) launch(ba_combine_splits_kernel<64, 4>);
+      else launch(ba_combine_splits_kernel<64, 0>);
+    }
     BA_CUDA_TRY(cudaGetLastError());
     ctx->launches += 1;
   }
