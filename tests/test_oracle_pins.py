@@ -330,6 +330,21 @@ def test_warm_path_equals_prefill_with_direct_rope():
     np.testing.assert_allclose(o_warm, o_cold[fin], atol=1e-12)
 
 
+def test_reencoding_may_be_applied_to_the_query_side():
+    # Eq. 3 after Eq. 2 is one rotation R(delta) of the cached key; rotations are orthogonal, so
+    # q . (R(delta) k) = (R(-delta) q) . k: the logits of a cached block against the re-encoded keys
+    # equal those of the counter-rotated queries against the keys as cached (both RoPE layouts).
+    d, base = 8, 10000.0
+    for layout in (ob.ROPE_ADJACENT, ob.ROPE_HALF):
+        q, k = rnd(41, 5, 2, d), rnd(42, 7, 2, d)
+        for delta in (0, 3, 250, 31000):
+            k_re = ob.reencode_delta(k, delta, base, layout)
+            q_rot = ob.rotate(q, np.full((5, 1), float(delta)), base, layout, inverse=True)
+            lhs = np.einsum("ihd,jhd->hij", q, k_re)
+            rhs = np.einsum("ihd,jhd->hij", q_rot, k)
+            np.testing.assert_allclose(lhs, rhs, atol=1e-10)
+
+
 # --------------------------------------------------------------------------- Table 3
 def test_table3_flops_exclude_attention_scores():
     # FLOPs-TFT = 2 * (about 7.5e9 parameters) * (tokens encoded): 50 tokens under
