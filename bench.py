@@ -250,6 +250,7 @@ def run_ours(args):
     stream = torch.cuda.current_stream()
 
     att_events = []
+    re_events = []
 
     def step(inputs, record=False):
         seg = B.ba_segment(ctx.ctx, lens, nb, 1, len(lens), w.n_tokens, B.BA_MODE_BLOCK, tbuf)
@@ -263,8 +264,13 @@ def run_ours(args):
                 B.ba_reencode_k_deferred(ctx.ctx, inputs[l + 1]["k_cache"], None, Tc, k_re[l + 1], seg.cache_cu,
                                          seg.cache_delta, seg.n_cached_blocks, Tc)
             elif l + 1 < L:
+                if record:
+                    r0 = torch.cuda.Event(enable_timing=True); r0.record(stream)
                 B.ba_reencode_k(ctx.ctx, inputs[l + 1]["k_cache"], None, Tc, k_re[l + 1], seg.cache_cu,
                                 seg.cache_delta, seg.n_cached_blocks, Tc)
+                if record:
+                    r1 = torch.cuda.Event(enable_timing=True); r1.record(stream)
+                    re_events.append((r0, r1))
             if record:
                 e0 = torch.cuda.Event(enable_timing=True); e0.record(stream)
             B.ba_final_attend(ctx.ctx, x["q_f"], x["k_f"], x["v_f"], Tf, k_re[l], x["v_cache"], Tc, None, 0,
@@ -298,6 +304,7 @@ def run_ours(args):
     ms, us_per_layer = aggregate(ms_local, float(L), dev)
 
     att_ms = statistics.mean(a.elapsed_time(b) for a, b in att_events)
+    re_ms = statistics.mean(a.elapsed_time(b) for a, b in re_events) if re_events else None
 
     # ---- end to end: host buffers in, host result out, copies inside the timed region
     e2e_steps = max(1, min(args.steps, 3))
@@ -458,6 +465,13 @@ def run_ours(args):
                 "e2e": {"value": e2e_us, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                         "steps": e2e_steps},
                 "gpu_launches": launches, "roofline": roofline, "cpu_baseline": cpu}
+        if re_ms is not None:
+            re_bytes = 2.0 * Tc * w.n_kv_heads * w.head_dim * 2        # cached K read once + re-encoded K written once
+            line["reencode"] = {"bound": "hbm", "kernel": "ba_reencode_k", "us_per_launch": re_ms * 1e3,
+                                "algorithmic_bytes_per_launch": re_bytes, "achieved": re_bytes / (re_ms * 1e-3) / 1e9,
+                                "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                                "frac": re_bytes / (re_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                                "peak_source": f"{peaks['source']} copy bandwidth"}
         if fused is not None:
             line["fused_warm_path"] = fused
         if prefill is not None:
