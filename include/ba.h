@@ -26,7 +26,15 @@
  *   Problems only the device can see (inconsistent tables, a bounded wait that
  *   ran out) are recorded in a status word read by ba_last_device_status().
  * - Nothing is allocated after ba_create(); a workspace that is too small for a
- *   call yields BA_ERR_WORKSPACE.  One context serves one stream at a time.
+ *   call yields BA_ERR_WORKSPACE.  Calls on one context share its workspace, so
+ *   they must be ordered on the device (one stream, or events between streams);
+ *   the one exception is ba_reencode_k with the cache_delta array of the
+ *   context's current tables, which uses no workspace and may run on another
+ *   stream beside an attention call that does not read or write its tensors.
+ *   All calls on a context come from one host thread at a time.
+ * - Every call that takes a context makes that context's device the calling
+ *   thread's current CUDA device (cudaSetDevice) and leaves it current on return;
+ *   ba_reencode_k_noalloc does the same with its `device` argument.
  * - No C++ exceptions cross this boundary.  There is no CPU fallback: on a
  *   machine without a usable sm_100 device ba_create() fails.
  */
@@ -80,6 +88,8 @@ typedef struct {
   int32_t batch, n_blocks, n_tokens, n_cached_blocks;
   int32_t mode;            /* ba_mode the tables were built for */
   int32_t q_tile_tokens;   /* tokens per query tile of the attention kernels */
+  int32_t n_prompt_items;  /* work items of ba_block_prefill / ba_final_attend for these tables when the */
+  int32_t n_final_items;   /* lengths were host arrays (exact launch size); 0 when they were on the device */
   /* per sequence, [batch + 1] */
   int32_t *cu_seq;         /* first row of the sequence, prompt packing */
   int32_t *cu_cache_seq;   /* first row of the sequence, cache packing */
@@ -123,7 +133,10 @@ ba_status ba_workspace_bytes(const ba_config *cfg, int32_t max_blocks, int32_t m
 
 /* Synchronises the context's device and returns (then clears) the first
  * problem a kernel recorded since the last call: BA_OK, BA_ERR_INVALID_ARG
- * (tables inconsistent with the lengths given) or BA_ERR_TIMEOUT. */
+ * (tables inconsistent with the lengths given; a gather index outside its source;
+ * a rotation table that no longer belongs to the tables it was stored with),
+ * BA_ERR_SHAPE (the tables describe more query rows than the tensors passed to an
+ * attention call hold: the surplus rows are not written) or BA_ERR_TIMEOUT. */
 ba_status ba_last_device_status(ba_ctx *ctx);
 
 /* Diagnostic (no counterpart in the paper): launches one CTA that waits, with the library's
@@ -174,7 +187,9 @@ ba_status ba_segment(ba_ctx *ctx, const int32_t *block_lens, const int32_t *seq_
  * Uses n_blocks * head_dim * 4 bytes of workspace for the angle table.  When `delta` is the
  * cache_delta array of the tables this context's last ba_segment() built (and n_blocks their
  * cached-block count), the rotation table built with those tables is used instead and no table is
- * computed; those tables must then still be alive and unchanged.
+ * computed; those tables must then still be alive and unchanged.  (ba_segment() stamps its tables;
+ * if the buffer was rebuilt or overwritten in the meantime the call rotates nothing and
+ * ba_last_device_status() reports BA_ERR_INVALID_ARG.)
  */
 ba_status ba_reencode_k(ba_ctx *ctx, const void *k_src, const int32_t *src_off, int32_t n_src_rows,
                         void *k_dst, const int32_t *cu, const int32_t *delta, int32_t n_blocks,
@@ -215,7 +230,9 @@ ba_status ba_flush(ba_ctx *ctx, void *stream);
  * call itself performs no cudaMalloc/cudaFree and uses no allocating library
  * routine.
  *
- *   cfg, device    as for ba_create (head_dim, n_kv_heads, rope_theta, rope_layout are used)
+ *   cfg, device    as for ba_create (head_dim, n_kv_heads, rope_theta, rope_layout are used); the
+ *                  device must exist (BA_ERR_CUDA otherwise), becomes the thread's current device,
+ *                  and gets a CUDA context if it had none
  *   status_word    device int32 owned by the caller, or NULL.  A source row out of range is
  *                  skipped and BA_ERR_INVALID_ARG is stored there if the word is still 0
  *                  (clear it yourself); with NULL such rows are skipped silently.

@@ -37,7 +37,8 @@ class ba_config(C.Structure):
 
 class ba_segments(C.Structure):
     _fields_ = [("batch", C.c_int32), ("n_blocks", C.c_int32), ("n_tokens", C.c_int32),
-                ("n_cached_blocks", C.c_int32), ("mode", C.c_int32), ("q_tile_tokens", C.c_int32)] + [
+                ("n_cached_blocks", C.c_int32), ("mode", C.c_int32), ("q_tile_tokens", C.c_int32),
+                ("n_prompt_items", C.c_int32), ("n_final_items", C.c_int32)] + [
         (n, C.c_void_p) for n in (
             "cu_seq", "cu_cache_seq", "cu_final_seq", "cu_seq_block", "cu_block", "block_delta",
             "block_seq", "block_kv_begin", "block_part_off", "block_is_final", "cache_block",

@@ -7,6 +7,8 @@
 
 ba_status ba_attend_sm100_launch(ba_ctx *ctx, const ba_attend_args &a, const ba_segments *seg,
                                  cudaStream_t stream);
+ba_status ba_attend_sm100_setup(ba_ctx *ctx);
+void ba_attend_sm100_teardown(ba_ctx *ctx);
 int ba_heads_per_tile(const ba_config &c);
 
 namespace {
@@ -124,12 +126,16 @@ ba_status ba_create(ba_ctx **out, const ba_config *cfg, int device, size_t works
   ctx->pending_table_bytes = 0;
   ctx->pending_stream = nullptr;
   ctx->seg_delta = nullptr; ctx->seg_rope = nullptr; ctx->seg_rope_blocks = 0;
+  ctx->seg_gen = nullptr; ctx->seg_gen_value = 0; ctx->seg_counter = 0;
+  ctx->maps = nullptr;
   ctx->workspace = nullptr;
   ctx->dev_status = nullptr;
   if (cudaMalloc(&ctx->dev_status, 256) != cudaSuccess ||
       cudaMemset(ctx->dev_status, 0, 256) != cudaSuccess ||
-      (workspace_bytes && cudaMalloc(&ctx->workspace, workspace_bytes) != cudaSuccess)) {
+      (workspace_bytes && cudaMalloc(&ctx->workspace, workspace_bytes) != cudaSuccess) ||
+      ba_attend_sm100_setup(ctx) != BA_OK) {
     cudaGetLastError();
+    if (ctx->workspace) cudaFree(ctx->workspace);
     if (ctx->dev_status) cudaFree(ctx->dev_status);
     delete ctx;
     return BA_ERR_CUDA;
@@ -145,6 +151,7 @@ ba_status ba_destroy(ba_ctx *ctx) {
   cudaDeviceSynchronize();
   if (ctx->workspace) cudaFree(ctx->workspace);
   if (ctx->dev_status) cudaFree(ctx->dev_status);
+  ba_attend_sm100_teardown(ctx);
   delete ctx;
   return BA_OK;
 }
@@ -203,6 +210,13 @@ ba_status ba_segment(ba_ctx *ctx, const int32_t *block_lens, const int32_t *seq_
   out->n_cached_blocks = n_blocks - batch;
   out->mode = mode;
   out->q_tile_tokens = q_tile_tokens(ctx->cfg);
+  if (host_lens) {   // lengths known here: the attention launches can be sized exactly
+    const int tt = out->q_tile_tokens;
+    long long items = 0, fitems = 0;
+    for (int b = 0; b < n_blocks; ++b) items += (block_lens[b] + tt - 1) / tt;
+    for (int q = 0, b = 0; q < batch; ++q) { b += seq_nblocks[q]; fitems += (block_lens[b - 1] + tt - 1) / tt; }
+    out->n_prompt_items = (int32_t)items; out->n_final_items = (int32_t)fitems;
+  }
   auto next = [&]() { return (int32_t *)(base + L.off[i++]); };
   out->cu_seq = next(); out->cu_cache_seq = next(); out->cu_final_seq = next(); out->cu_seq_block = next();
   out->cu_block = next();
@@ -212,14 +226,21 @@ ba_status ba_segment(ba_ctx *ctx, const int32_t *block_lens, const int32_t *seq_
   out->tok_block = next(); out->tok_pos = next(); out->tok_pos_local = next();
   out->cu_qtile = next(); out->cu_ftile = next(); out->cache_tile_cu = next(); out->totals = next();
   out->cache_rope = (float *)next();
-  ctx->seg_delta = nullptr; ctx->seg_rope = nullptr; ctx->seg_rope_blocks = 0;
-  ba_status st = ba_segment_launch(ctx, d_lens, d_nb, batch, n_blocks, n_tokens, mode, out, s);
+  ctx->seg_delta = nullptr; ctx->seg_rope = nullptr; ctx->seg_rope_blocks = 0; ctx->seg_gen = nullptr;
+  // Every call stamps its tables (totals[6]) with a value that differs from call to call and from
+  // context to context: a later re-encoding that wants to reuse the rotation table stored with the
+  // tables can tell on the device whether the buffer still holds this call's tables.
+  ctx->seg_counter += 1;
+  const int32_t gen = (int32_t)((((uint32_t)((uintptr_t)ctx >> 6)) * 0x9E3779B1u +
+                                 (uint32_t)ctx->seg_counter * 0x85EBCA6Bu) | 1u);
+  ba_status st = ba_segment_launch(ctx, d_lens, d_nb, batch, n_blocks, n_tokens, mode, gen, out, s);
   if (st != BA_OK || out->n_cached_blocks == 0) return st;
   // rotations of the cached blocks (the same angle table ba_reencode_k builds), once per prompt
   st = ba_reencode_table_launch(ctx, out->cache_delta, out->n_cached_blocks, (float2 *)out->cache_rope, s);
   if (st == BA_OK) {
     ctx->seg_delta = out->cache_delta; ctx->seg_rope = (const float2 *)out->cache_rope;
     ctx->seg_rope_blocks = out->n_cached_blocks;
+    ctx->seg_gen = out->totals + 6; ctx->seg_gen_value = gen;
   }
   return st;
 }
@@ -254,10 +275,12 @@ ba_status ba_reencode_k(ba_ctx *ctx, const void *k_src, const int32_t *src_off, 
   ba_status st = check_reencode_args(ctx, k_src, src_off, n_src_rows, k_dst, cu, delta, n_blocks, n_rows, &nothing);
   if (st != BA_OK || nothing) return st;
   BA_CUDA_TRY(cudaSetDevice(ctx->device));
-  if (delta == ctx->seg_delta && n_blocks == ctx->seg_rope_blocks)   // the table ba_segment built is for these deltas
-    return ba_reencode_main_launch(
-        ctx, ba_make_reencode_job(ctx, k_src, src_off, n_src_rows, k_dst, cu, delta, n_blocks, n_rows, ctx->seg_rope),
-        (cudaStream_t)stream);
+  if (delta == ctx->seg_delta && n_blocks == ctx->seg_rope_blocks) {   // the table ba_segment built is for these deltas
+    ba_reencode_job job =
+        ba_make_reencode_job(ctx, k_src, src_off, n_src_rows, k_dst, cu, delta, n_blocks, n_rows, ctx->seg_rope);
+    job.gen = ctx->seg_gen; job.gen_expected = ctx->seg_gen_value;
+    return ba_reencode_main_launch(ctx, job, (cudaStream_t)stream);
+  }
   float2 *table; size_t bytes;
   st = place_table(ctx, n_blocks, &table, &bytes);
   if (st != BA_OK) return st;
@@ -287,6 +310,7 @@ ba_status ba_reencode_k_deferred(ba_ctx *ctx, const void *k_src, const int32_t *
     table_used = table;
   }
   ctx->pending = ba_make_reencode_job(ctx, k_src, src_off, n_src_rows, k_dst, cu, delta, n_blocks, n_rows, table_used);
+  if (table_used == ctx->seg_rope) { ctx->pending.gen = ctx->seg_gen; ctx->pending.gen_expected = ctx->seg_gen_value; }
   ctx->has_pending = 1;
   ctx->pending_table_bytes = bytes;
   ctx->pending_stream = (cudaStream_t)stream;
@@ -336,6 +360,8 @@ ba_status ba_final_attend(ba_ctx *ctx, const void *q_f, const void *k_f, const v
   if (n_cache_rows > 0 && (!k_cache || !v_cache || !aligned16(k_cache) || !aligned16(v_cache)))
     return BA_ERR_INVALID_ARG;
   if (v_src_off && n_v_rows < 1) return BA_ERR_INVALID_ARG;
+  // the tables describe n_tokens rows: the caller's final and cached tensors must add up to them
+  if ((long long)n_final_rows + n_cache_rows != seg->n_tokens) return BA_ERR_SHAPE;
   BA_CUDA_TRY(cudaSetDevice(ctx->device));
   ba_attend_args a;
   memset(&a, 0, sizeof(a));
@@ -362,6 +388,7 @@ ba_status ba_final_attend_fused(ba_ctx *ctx, const void *q_f, const void *k_f, c
     if (n_src_rows < 1 || !seg->cache_rope || !seg->cache_tile_cu) return BA_ERR_INVALID_ARG;
     if (!src_off && n_src_rows < n_cache_rows) return BA_ERR_INVALID_ARG;
   }
+  if ((long long)n_final_rows + n_cache_rows != seg->n_tokens) return BA_ERR_SHAPE;
   BA_CUDA_TRY(cudaSetDevice(ctx->device));
   ba_attend_args a;
   memset(&a, 0, sizeof(a));

@@ -32,6 +32,7 @@
 // so the QK^T products switch buffers without a pause.  The cached keys are never rewritten or
 // re-read, and a key tile never spans two blocks.
 #include <math.h>
+#include <new>
 #include <type_traits>
 
 #include "ba_common.cuh"
@@ -40,7 +41,9 @@
 
 using namespace sm100;
 
-// Optional phase timeline of CTA (0,0,0) for tuning: compile with -DBA_TRACE.
+// Tuning aid, absent from ordinary builds: with -DBA_TRACE the roles of CTA 0 stamp clock64() at the
+// phases of their first 64 key tiles into a device array that a developer build reads back
+// (roles 0/1: softmax groups, 2: MMA thread per query tile, 3: MMA thread's K/V waits, 5: fused query versions).
 #ifdef BA_TRACE
 __device__ long long g_ba_trace[6][64][8];
 extern "C" int ba_trace_read(long long *dst) { return (int)cudaMemcpyFromSymbol(dst, g_ba_trace, sizeof(g_ba_trace)); }
@@ -56,25 +59,14 @@ namespace {
 
 constexpr int kThreads = 384;
 constexpr int kBlockN = 128;      // keys per tile
-#ifndef BA_STAGES
-#define BA_STAGES 3
-#endif
-constexpr int kStages = BA_STAGES;   // ring of K/V tiles (K_j, V_j, K_j+1, ...)
+constexpr int kStages = 3;           // ring of K/V tiles (K_j, V_j, K_j+1, ...)
 constexpr float kRescaleThreshold = 8.0f;
 constexpr int kBgStageBytes = 16384; // two spare warps x two stages of source rows
 constexpr int kWorkSlots = 4;      // ring of published work entries (power of two)
-// Register split after launch (168 per thread): service warps give registers to the softmax warps.
-// 128 * BA_SVC_REGS + 256 * BA_SMX_REGS <= 384 * 168.
-#ifndef BA_SVC_REGS
-#define BA_SVC_REGS 72
-#endif
-// the MMA thread's loops over the two query tiles
-#ifndef BA_T_UNROLL
-#define BA_T_UNROLL _Pragma("unroll")
-#endif
-#ifndef BA_SMX_REGS
-#define BA_SMX_REGS 216
-#endif
+// Register split after launch (168 per thread): the service warps give registers to the softmax warps.
+// 128 * kServiceRegs + 256 * kSoftmaxRegs <= 384 * 168.
+constexpr int kServiceRegs = 72;
+constexpr int kSoftmaxRegs = 216;
 
 struct AttnParams {
   void *o;
@@ -155,40 +147,6 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
   asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
   return d;
 }
-
-// 2^x for two values on the FMA pipe (x <= ~8): clamp at -126, round x to the nearest integer n
-// with the 1.5*2^23 trick, evaluate a cubic fit of 2^r on r = x - n in [-0.5, 0.5] (relative
-// error < 8e-5, far below the bf16 rounding applied to the result) and add n to the exponent
-// field.  The arithmetic is packed (two fp32 per instruction).  With BA_POLY_PERIOD = n, one
-// column pair in n goes this way and the special-function unit and the FMA pipe work side by
-// side; only tiles without masked columns use it, because a masked column must give exactly 0
-// and this gives 2^-126.  Off by default: at n = 4 the softmax of a tile gets about 6 % shorter
-// in cycles, but the extra instructions cost more clock under the power limit than that (+2.7 %
-// time at 32K context; n = 2, 3 are slower still).
-__device__ __forceinline__ uint64_t exp2_poly2(uint64_t x2) {
-  float x0, x1;
-  unpack2(x2, x0, x1);
-  x2 = pack2(fmaxf(x0, -126.f), fmaxf(x1, -126.f));
-  const uint64_t t2 = add2(x2, pack2(12582912.f, 12582912.f));
-  const uint64_t u2 = add2(t2, pack2(-12582912.f, -12582912.f));
-  const uint64_t r2 = fma2(u2, pack2(-1.f, -1.f), x2);
-  uint64_t q2 = fma2(pack2(0.055088684f, 0.055088684f), r2, pack2(0.24260405f, 0.24260405f));
-  q2 = fma2(q2, r2, pack2(0.69327623f, 0.69327623f));
-  q2 = fma2(q2, r2, pack2(0.99992895f, 0.99992895f));
-  float q0, q1, t0, t1;
-  unpack2(q2, q0, q1);
-  unpack2(t2, t0, t1);
-  return pack2(__uint_as_float(__float_as_uint(q0) + (__float_as_uint(t0) << 23)),
-               __uint_as_float(__float_as_uint(q1) + (__float_as_uint(t1) << 23)));
-}
-#ifndef BA_POLY_PERIOD
-#define BA_POLY_PERIOD 0
-#endif
-#ifndef BA_SPLIT_P
-#define BA_SPLIT_P 1
-#endif
-constexpr int kPolyPeriod = BA_POLY_PERIOD;    // one column pair in kPolyPeriod uses exp2_poly2 (0: none)
-constexpr bool kSplitP = BA_SPLIT_P;             // hand P to the MMA warp in two halves
 
 __device__ __forceinline__ int upper_bound_tbl(const int32_t *a, int n, int x) {
   int lo = 0, hi = n;
@@ -348,7 +306,7 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
                        const __grid_constant__ CUtensorMap tmap_vc, const AttnParams p) {
   using L = Layout<D>;
   // setmaxnreg is a warpgroup-wide instruction: the four service warps (8-11) must ask for the same count
-  constexpr int kProdRegs = BA_SVC_REGS, kMmaRegs = BA_SVC_REGS, kSpareRegs = BA_SVC_REGS;
+  constexpr int kProdRegs = kServiceRegs, kMmaRegs = kServiceRegs, kSpareRegs = kServiceRegs;
   extern __shared__ uint8_t smem_raw[];
   uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   Ctrl *ctrl = reinterpret_cast<Ctrl *>(smem + L::kCtrl);
@@ -565,14 +523,14 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
         walk_end = -1; ver_end[0] = ver_end[1] = -1;
         cached_end = min(wk.tile0 + n_tiles, wk.it.n_cache_tiles);
         if (!kFused) {
-BA_T_UNROLL
+#pragma unroll
           for (int t = 0; t < 2; ++t)
             if (t < n_qt && ok) ok = mbar_wait(&ctrl->q_full[t], q_uses[t] & 1, abort_flag);
         }
         if (ok) ok = wait_kv(gidx);
         if (!ok) break;
         tc_fence_after();
-BA_T_UNROLL
+#pragma unroll
         for (int t = 0; t < 2; ++t)
           if (t < n_qt && ok) ok = issue_qk(t, 0, gidx);
         if (!ok) break;
@@ -584,7 +542,7 @@ BA_T_UNROLL
           BA_TR(3, j, 0);
           ok = wait_kv(iv);
           BA_TR(3, j, 1);
-BA_T_UNROLL
+#pragma unroll
           for (int t = 0; t < 2; ++t) {
             if (t >= n_qt || !ok) continue;
             BA_TR(2, j, t * 4 + 0);
@@ -618,7 +576,7 @@ BA_T_UNROLL
           }
         }
         gidx += 2 * n_tiles;
-BA_T_UNROLL
+#pragma unroll
         for (int t = 0; t < 2; ++t)
           if (t < n_qt) ++q_uses[t];
       }
@@ -638,7 +596,7 @@ BA_T_UNROLL
     }
   } else {
     // ------------------------------------------------------------ softmax, one thread per tile row
-    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(BA_SMX_REGS));
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kSoftmaxRegs));
     const int t = warp >> 2;
     const int r = tid & 127;
     const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
@@ -667,7 +625,10 @@ BA_T_UNROLL
       if (t < it.n_qt) {
       const int q_last = it.q_row0 + it.q_rows - 1;
       const int row_tok = it.q_row0 + t * p.tok + (r >> p.hpt_log2);
-      const bool row_valid = row_tok <= q_last;
+      // a row is stored only if it belongs to the item and lies inside the caller's tensors; tables that
+      // describe more rows than the caller gave are reported, nothing is written past the end
+      const bool row_valid = row_tok <= q_last && row_tok < p.n_q_rows;
+      if (row_tok <= q_last && row_tok >= p.n_q_rows) ba_record_status(p.status, BA_ERR_SHAPE);
       const int tok_c = min(row_tok, q_last);               // rows past the block behave like its last row
       const int head = head0 + (r & (p.hpt - 1));
       float m_used = -INFINITY, l = 0.f;
@@ -790,39 +751,26 @@ BA_T_UNROLL
         const uint64_t sl2 = pack2(sl, sl), negm2 = pack2(neg_m, neg_m);
         // P is handed to the MMA warp in two halves so that PV can start on the first 64 keys
         // while the second 64 are still being exponentiated.  The arithmetic is packed fp32x2.
-        auto exp_halves = [&](auto poly_tag) {
-          constexpr bool kPoly = decltype(poly_tag)::value;
 #pragma unroll
-          for (int h = 0; h < 2; ++h) {
-            uint32_t pk[32];
+        for (int h = 0; h < 2; ++h) {
+          uint32_t pk[32];
 #pragma unroll
-            for (int i = 0; i < 32; ++i) {
-              const int e0 = h * 64 + 2 * i, e1 = e0 + 1;
-              const uint64_t x2 = fma2(pack2(__uint_as_float(s[e0]), __uint_as_float(s[e1])), sl2, negm2);
-              float p0, p1;
-              if (kPoly && i % (kPolyPeriod > 0 ? kPolyPeriod : 1) == kPolyPeriod - 1) {
-                unpack2(exp2_poly2(x2), p0, p1);
-              } else {
-                float x0, x1;
-                unpack2(x2, x0, x1);
-                p0 = ex2(x0); p1 = ex2(x1);
-              }
-              sum2[i & 3] = add2(sum2[i & 3], pack2(p0, p1));
-              __nv_bfloat162 v = __floats2bfloat162_rn(p0, p1);
-              pk[i] = *reinterpret_cast<uint32_t *>(&v);
-            }
-            tmem_st_32x32b_x32(tS + h * 32, pk);
-            if (kSplitP || h == 1) {
-              tmem_wait_st();
-              tc_fence_before();
-              if (!kSplitP) mbar_arrive(&ctrl->p_full[t][0]);
-              mbar_arrive(&ctrl->p_full[t][h]);
-            }
-            if (r == 0) BA_TR(t, j, 4 + h);
+          for (int i = 0; i < 32; ++i) {
+            const int e0 = h * 64 + 2 * i, e1 = e0 + 1;
+            const uint64_t x2 = fma2(pack2(__uint_as_float(s[e0]), __uint_as_float(s[e1])), sl2, negm2);
+            float x0, x1;
+            unpack2(x2, x0, x1);
+            const float p0 = ex2(x0), p1 = ex2(x1);
+            sum2[i & 3] = add2(sum2[i & 3], pack2(p0, p1));
+            __nv_bfloat162 v = __floats2bfloat162_rn(p0, p1);
+            pk[i] = *reinterpret_cast<uint32_t *>(&v);
           }
-        };
-        if (kPolyPeriod > 0 && __all_sync(0xffffffffu, lim >= kBlockN - 1)) exp_halves(std::true_type{});
-        else exp_halves(std::false_type{});
+          tmem_st_32x32b_x32(tS + h * 32, pk);
+          tmem_wait_st();
+          tc_fence_before();
+          mbar_arrive(&ctrl->p_full[t][h]);
+          if (r == 0) BA_TR(t, j, 4 + h);
+        }
         // P of this tile is with the tensor core: time to work on the next version of the query row
         if (kFused && next_start < tile_end) {
           const bool due = tile0 + j + 1 == next_start;    // the next tile is the first to need it
@@ -985,6 +933,66 @@ bool make_map(CUtensorMap *m, const void *ptr, int D, int heads, long long rows,
 
 }  // namespace
 
+// Tensor maps of the tensors recently passed to the attention calls.  A serving loop hands the same
+// few buffers to the library layer after layer; encoding a map costs a driver call each time, so
+// the maps are kept in a small direct-mapped table keyed by everything that goes into them.
+struct ba_map_cache {
+  static constexpr int kSlots = 512;
+  struct Slot {
+    const void *ptr;
+    long long rows;
+    int D, heads, box_heads, box_rows;
+    alignas(64) CUtensorMap map;
+  } slot[kSlots];
+};
+
+namespace {
+
+const CUtensorMap *cached_map(ba_ctx *ctx, const void *ptr, int D, int heads, long long rows, int box_heads,
+                              int box_rows) {
+  uint64_t h = (uint64_t)(uintptr_t)ptr * 0x9E3779B97F4A7C15ull;
+  h ^= (uint64_t)rows * 0xC2B2AE3D27D4EB4Full + (uint64_t)(box_heads * 131 + box_rows);
+  ba_map_cache::Slot &sl = ctx->maps->slot[(h >> 40) & (ba_map_cache::kSlots - 1)];
+  if (sl.ptr == ptr && sl.rows == rows && sl.D == D && sl.heads == heads && sl.box_heads == box_heads &&
+      sl.box_rows == box_rows)
+    return &sl.map;
+  sl.ptr = nullptr;
+  if (!make_map(&sl.map, ptr, D, heads, rows, box_heads, box_rows)) return nullptr;
+  sl.ptr = ptr; sl.rows = rows; sl.D = D; sl.heads = heads; sl.box_heads = box_heads; sl.box_rows = box_rows;
+  return &sl.map;
+}
+
+template <int D>
+constexpr int attend_smem_bytes() {
+  // ask for more than half of the SM's shared memory so that two CTAs never share an SM
+  // (each CTA allocates all 512 tensor-memory columns)
+  return Layout<D>::kBytes + 1024 > 120 * 1024 ? Layout<D>::kBytes + 1024 : 120 * 1024;
+}
+
+}  // namespace
+
+// Per-context set-up of the attention path, with the context's device current: the kernels' shared-memory
+// limit is raised once here instead of on every launch, and the tensor-map table is created.
+ba_status ba_attend_sm100_setup(ba_ctx *ctx) {
+  BA_CUDA_TRY(cudaFuncSetAttribute(ba_attend_sm100_kernel<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                   attend_smem_bytes<128>()));
+  BA_CUDA_TRY(cudaFuncSetAttribute(ba_attend_sm100_kernel<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                   attend_smem_bytes<128>()));
+  BA_CUDA_TRY(cudaFuncSetAttribute(ba_attend_sm100_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                   attend_smem_bytes<64>()));
+  BA_CUDA_TRY(cudaFuncSetAttribute(ba_attend_sm100_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                   attend_smem_bytes<64>()));
+  ctx->maps = new (std::nothrow) ba_map_cache();
+  if (!ctx->maps) return BA_ERR_CUDA;
+  for (auto &sl : ctx->maps->slot) sl.ptr = nullptr;
+  return BA_OK;
+}
+
+void ba_attend_sm100_teardown(ba_ctx *ctx) {
+  delete ctx->maps;
+  ctx->maps = nullptr;
+}
+
 // Diagnostic: one CTA waits on an mbarrier that nothing ever arrives on, with the same bounded
 // wait the attention kernel uses, so the expiry path (abort flag, status word, clean return) can be
 // checked on a live device without any fault.
@@ -1041,13 +1049,18 @@ ba_status ba_attend_sm100_launch(ba_ctx *ctx, const ba_attend_args &a, const ba_
   // waves x (tiles per CTA + a fixed per-CTA cost) and is capped by the workspace.
   const int pair_tok = 2 * p.tok;
   const int n_units = a.final_only ? seg->batch : seg->n_blocks;
-  const unsigned pairs_upper = (unsigned)(a.n_q_rows / pair_tok + n_units);
+  // work items: the exact count when ba_segment() saw the lengths on the host, else an upper bound
+  const int pairs_known = a.final_only ? seg->n_final_items : seg->n_prompt_items;
+  const unsigned pairs_upper = pairs_known > 0 ? (unsigned)pairs_known : (unsigned)(a.n_q_rows / pair_tok + n_units);
   const long long items = (long long)((a.n_q_rows + pair_tok - 1) / pair_tok) * (Hq / p.hpt);
   int n_splits = 1;
   if (a.final_only && items < 2LL * ctx->sm_count) {
     const long long avg_tiles = ((long long)a.n_cache_rows / seg->batch + pair_tok) / kBlockN + 1;
     const size_t per_split = (size_t)a.n_q_rows * Hq * (D + 1) * sizeof(float);
-    const size_t avail = ctx->workspace_bytes > ba_scratch_offset(ctx) ? ctx->workspace_bytes - ba_scratch_offset(ctx) : 0;
+    // the angle table of a queued re-encoding job sits at the end of the workspace and is read by
+    // this very launch: the partial results must stay below it
+    const size_t taken = ba_scratch_offset(ctx) + ctx->pending_table_bytes;
+    const size_t avail = ctx->workspace_bytes > taken ? ctx->workspace_bytes - taken : 0;
     const int cap = (int)min((size_t)16, per_split ? avail / per_split : 0);
     long long best = -1;
     for (int ns = 1; ns <= cap && ns <= avg_tiles; ++ns) {
@@ -1077,15 +1090,18 @@ ba_status ba_attend_sm100_launch(ba_ctx *ctx, const ba_attend_args &a, const ba_
     p.lse_part = p.o_part + (size_t)n_splits * a.n_q_rows * Hq * D;
   }
 
-  CUtensorMap tq, tk, tv, tkc, tvc;
-  if (!make_map(&tq, a.q, D, Hq, a.n_q_rows, p.hpt, p.tok)) return BA_ERR_CUDA;
-  if (!make_map(&tk, a.k, D, Hkv, a.n_kv_rows, 1, kBlockN)) return BA_ERR_CUDA;
-  if (!make_map(&tv, a.v, D, Hkv, a.n_kv_rows, 1, kBlockN)) return BA_ERR_CUDA;
+  const CUtensorMap *mq = cached_map(ctx, a.q, D, Hq, a.n_q_rows, p.hpt, p.tok);
+  const CUtensorMap *mk = cached_map(ctx, a.k, D, Hkv, a.n_kv_rows, 1, kBlockN);
+  const CUtensorMap *mv = cached_map(ctx, a.v, D, Hkv, a.n_kv_rows, 1, kBlockN);
+  if (!mq || !mk || !mv) return BA_ERR_CUDA;
+  CUtensorMap tq = *mq, tk = *mk, tv = *mv, tkc = *mk, tvc = *mv;   // (a slot may be reused by a later look-up)
   if (a.final_only && a.n_cache_rows > 0) {
-    if (!make_map(&tkc, a.k_cache, D, Hkv, p.fused ? a.n_k_rows : a.n_cache_rows, 1, kBlockN)) return BA_ERR_CUDA;
-    if (!make_map(&tvc, a.v_cache, D, Hkv, a.v_src_off ? a.n_v_rows : a.n_cache_rows, 1, kBlockN)) return BA_ERR_CUDA;
-  } else {
-    tkc = tk; tvc = tv;
+    const CUtensorMap *mkc = cached_map(ctx, a.k_cache, D, Hkv, p.fused ? a.n_k_rows : a.n_cache_rows, 1, kBlockN);
+    if (!mkc) return BA_ERR_CUDA;
+    tkc = *mkc;
+    const CUtensorMap *mvc = cached_map(ctx, a.v_cache, D, Hkv, a.v_src_off ? a.n_v_rows : a.n_cache_rows, 1, kBlockN);
+    if (!mvc) return BA_ERR_CUDA;
+    tvc = *mvc;
   }
   dim3 grid((unsigned)(p.persistent ? ctx->sm_count : work_upper));
   // a queued re-encoding job rides along in the spare warps; a job whose rows do not fit the
@@ -1105,18 +1121,12 @@ ba_status ba_attend_sm100_launch(ba_ctx *ctx, const ba_attend_args &a, const ba_
       if (fs != BA_OK) return fs;
     }
   }
-  // ask for more than half of the SM's shared memory so that two CTAs never share an SM
-  // (each CTA allocates all 512 tensor-memory columns)
   if (D == 128) {
-    const int smem = Layout<128>::kBytes + 1024;
     auto kern = p.fused ? ba_attend_sm100_kernel<128, true> : ba_attend_sm100_kernel<128, false>;
-    BA_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-    kern<<<grid, kThreads, smem, stream>>>(tq, tk, tv, tkc, tvc, p);
+    kern<<<grid, kThreads, attend_smem_bytes<128>(), stream>>>(tq, tk, tv, tkc, tvc, p);
   } else {
-    const int smem = max(Layout<64>::kBytes + 1024, 120 * 1024);
     auto kern = p.fused ? ba_attend_sm100_kernel<64, true> : ba_attend_sm100_kernel<64, false>;
-    BA_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-    kern<<<grid, kThreads, smem, stream>>>(tq, tk, tv, tkc, tvc, p);
+    kern<<<grid, kThreads, attend_smem_bytes<64>(), stream>>>(tq, tk, tv, tkc, tvc, p);
   }
   BA_CUDA_TRY(cudaGetLastError());
   ctx->launches += 1;

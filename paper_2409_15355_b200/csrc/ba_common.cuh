@@ -8,10 +8,12 @@
 
 #include "ba.h"
 
-#define BA_CUDA_TRY(expr)                          \
-  do {                                             \
-    cudaError_t _e = (expr);                       \
-    if (_e != cudaSuccess) { return BA_ERR_CUDA; } \
+// A failed runtime call also leaves its code in the runtime's per-thread "last error" slot; it is
+// cleared here so that a later, healthy launch does not trip over it.
+#define BA_CUDA_TRY(expr)                                              \
+  do {                                                                 \
+    cudaError_t _e = (expr);                                           \
+    if (_e != cudaSuccess) { cudaGetLastError(); return BA_ERR_CUDA; } \
   } while (0)
 
 // Value of ba_segments::totals[7] once ba_segment's kernel has found the lengths consistent.
@@ -28,6 +30,11 @@ struct ba_reencode_job {
   const float2 *table;      // [n_blocks][head_dim / 2] (cos, sin)
   int32_t n_src_rows, n_blocks, n_rows;
   int32_t head_dim, row_vecs /* uint4 per row */, layout;
+  // non-null: `table` is the rotation table ba_segment() stored with its tables; *gen must still hold
+  // gen_expected (the stamp that call wrote), else the tables were rebuilt or overwritten since and
+  // the job reports BA_ERR_INVALID_ARG instead of rotating with a foreign table
+  const int32_t *gen;
+  int32_t gen_expected;
 };
 
 // Context: configuration, workspace and the device status word.
@@ -51,6 +58,11 @@ struct ba_ctx {
   const int32_t *seg_delta;
   const float2 *seg_rope;
   int32_t seg_rope_blocks;
+  const int32_t *seg_gen;   // device word the same ba_segment stamped with seg_gen_value (totals[6])
+  int32_t seg_gen_value;
+  int32_t seg_counter;      // ba_segment calls so far on this context
+  // tensor maps of recently used tensors (attention launches re-use a handful of buffers)
+  struct ba_map_cache *maps;
 };
 
 static inline size_t ba_align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -68,7 +80,7 @@ __device__ __forceinline__ void ba_record_status(int32_t *status, int32_t code) 
 
 // Entry points implemented in the individual .cu files.
 ba_status ba_segment_launch(ba_ctx *ctx, const int32_t *d_block_lens, const int32_t *d_seq_nblocks,
-                            int32_t batch, int32_t n_blocks, int32_t n_tokens, int mode,
+                            int32_t batch, int32_t n_blocks, int32_t n_tokens, int mode, int32_t gen,
                             const ba_segments *seg, cudaStream_t stream);
 
 // Re-encoding in two steps: angle table, then the rotation itself.

@@ -34,9 +34,6 @@ ba_rope_table_kernel(const int32_t *__restrict__ delta, int n_blocks, int half_d
 // A CTA takes kPasses consecutive groups of rows; its threads keep their column and walk down the
 // rows, kRows loads in flight each, so the per-thread set-up (column arithmetic, block search, table
 // fetch) is paid once per kPasses * kRows rows.
-#ifndef BA_REENCODE_PASSES
-#define BA_REENCODE_PASSES 4
-#endif
 template <int kLayout, int kRows, int kPasses>
 __global__ void __launch_bounds__(512)
 ba_reencode_kernel(const ba_reencode_job job, int units_shift, int32_t *status) {
@@ -47,6 +44,10 @@ ba_reencode_kernel(const ba_reencode_job job, int units_shift, int32_t *status) 
   const int rsub = units_shift >= 0 ? (int)(threadIdx.x >> units_shift) : (int)(threadIdx.x / units_per_row);
   const int total_rows = min(job.n_rows, __ldg(job.cu + job.n_blocks));
   const int cta_row0 = blockIdx.x * (row_step * kRows * kPasses);
+  if (job.gen && __ldg(job.gen) != job.gen_expected) {     // the rotation table is not the one this job was given
+    if (threadIdx.x == 0) ba_record_status(status, BA_ERR_INVALID_ARG);
+    return;
+  }
   // the block of the CTA's first row is searched once and shared; the threads walk forward from it
   __shared__ int s_c;
   if (threadIdx.x == 0) {
@@ -88,25 +89,20 @@ ba_reencode_job ba_make_reencode_job(const ba_ctx *ctx, const void *k_src, const
   job.table = table; job.n_src_rows = n_src_rows; job.n_blocks = n_blocks; job.n_rows = n_rows;
   job.head_dim = ctx->cfg.head_dim; job.row_vecs = ctx->cfg.n_kv_heads * ctx->cfg.head_dim / 8;
   job.layout = ctx->cfg.rope_layout;
+  job.gen = nullptr; job.gen_expected = 0;
   return job;
 }
 
 ba_status ba_reencode_main_launch(ba_ctx *ctx, const ba_reencode_job &job, cudaStream_t stream) {
-#ifndef BA_REENCODE_ROWS
-#define BA_REENCODE_ROWS 1
-#endif
-  constexpr int kRows = BA_REENCODE_ROWS;   // rows in flight per thread
+  constexpr int kRows = 1;                  // rows in flight per thread
   const bool adjacent = job.layout == BA_ROPE_ADJACENT;
   const int units = adjacent ? job.row_vecs : job.row_vecs / 2;
-  // threads per CTA: a multiple of the units per row, close to BA_REENCODE_THREADS
-#ifndef BA_REENCODE_THREADS
-#define BA_REENCODE_THREADS 128
-#endif
-  int threads = units >= BA_REENCODE_THREADS ? units : (BA_REENCODE_THREADS / units) * units;
+  // threads per CTA: a multiple of the units per row, close to 128
+  int threads = units >= 128 ? units : (128 / units) * units;
   int units_shift = -1;                       // log2(units) when it is a power of two
   for (int k = 0; k < 12; ++k) if ((1 << k) == units) units_shift = k;
   if (threads > 512) return BA_ERR_UNSUPPORTED;   // more than 4096 bf16 per row
-  constexpr int kPasses = BA_REENCODE_PASSES;
+  constexpr int kPasses = 4;                // consecutive row groups per CTA
   const int rows_per_cta = (threads / units) * kRows * kPasses;
   const int grid = (job.n_rows + rows_per_cta - 1) / rows_per_cta;
   if (adjacent)
@@ -167,6 +163,10 @@ extern "C" ba_status ba_reencode_k_noalloc(const ba_config *cfg, int device, con
   if (cfg->rope_layout != BA_ROPE_ADJACENT && cfg->rope_layout != BA_ROPE_HALF) return BA_ERR_INVALID_ARG;
   if (!(cfg->rope_theta > 1.0)) return BA_ERR_INVALID_ARG;
   if (device < 0 || device >= kNoallocMaxDevices) return BA_ERR_INVALID_ARG;
+  {
+    int n_dev = 0;
+    if (cudaGetDeviceCount(&n_dev) != cudaSuccess || device >= n_dev) { cudaGetLastError(); return BA_ERR_CUDA; }
+  }
   if (n_blocks < 0 || n_rows < 0 || n_src_rows < 0) return BA_ERR_INVALID_ARG;
   if (n_blocks > BA_NOALLOC_MAX_BLOCKS) return BA_ERR_WORKSPACE;   // built-in table too small
   if (n_blocks == 0 || n_rows == 0) return BA_OK;
@@ -199,6 +199,7 @@ extern "C" ba_status ba_reencode_k_noalloc(const ba_config *cfg, int device, con
   tmp.pending_table_bytes = 0;
   tmp.pending_stream = nullptr;
   tmp.seg_delta = nullptr; tmp.seg_rope = nullptr; tmp.seg_rope_blocks = 0;
+  tmp.seg_gen = nullptr; tmp.seg_gen_value = 0; tmp.seg_counter = 0; tmp.maps = nullptr;
   return ba_reencode_launch(&tmp, k_src, src_off, n_src_rows, k_dst, cu, delta, n_blocks, n_rows,
                             g_noalloc_table[device], (cudaStream_t)stream);
 }

@@ -34,9 +34,6 @@ __device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w 
 // registers from one row to the next and is looked up again only when a row leaves the block.
 // The source rows are read once: streaming loads keep them from displacing the re-encoded keys,
 // which the attention launch that follows reads, in L2.
-#ifndef BA_RE_LOAD
-#define BA_RE_LOAD(p) __ldcs(p)
-#endif
 struct ba_reencode_state {
   int vec_x, vec_y, m0;              // the thread's vector column(s) and first rotary pair
   int c, c_begin, c_end;             // block of the last row and its row range
@@ -102,8 +99,8 @@ __device__ __forceinline__ void ba_reencode_rows(const ba_reencode_job &job, ba_
         live[i] = false;
       } else {
         const uint4 *p = src + sr * row_vecs;
-        x[i] = BA_RE_LOAD(p + vec_x);
-        if (kLayout == BA_ROPE_HALF) y[i] = BA_RE_LOAD(p + vec_y);
+        x[i] = __ldcs(p + vec_x);
+        if (kLayout == BA_ROPE_HALF) y[i] = __ldcs(p + vec_y);
       }
     }
   }
@@ -188,6 +185,10 @@ __device__ __forceinline__ void ba_reencode_background(const ba_reencode_job &jo
   const int total_rows = min(job.n_rows, __ldg(job.cu + job.n_blocks));
   const int n_chunks = (total_rows + rows_per_chunk - 1) / rows_per_chunk;
   const bool adjacent = job.layout == BA_ROPE_ADJACENT;
+  if (job.gen && __ldg(job.gen) != job.gen_expected) {     // the rotation table is not the one this job was given
+    if (lane == 0) ba_record_status(status, BA_ERR_INVALID_ARG);
+    return;
+  }
 
   // fetch: draw a chunk, resolve its rows, start the copies into stage `s`; returns false when the job is exhausted
   auto fetch = [&](int s) -> bool {

@@ -54,12 +54,12 @@ __device__ __forceinline__ int upper_bound(const int32_t *a, int n, int x) {
 
 __global__ void __launch_bounds__(kScanThreads)
 ba_segment_blocks_kernel(const int32_t *__restrict__ lens, const int32_t *__restrict__ seq_nblocks,
-                         int batch, int B, int T, int mode, int tile_tok, ba_segments seg,
+                         int batch, int B, int T, int mode, int tile_tok, int gen, ba_segments seg,
                          int32_t *status) {
   __shared__ int scan_smem[33];
   __shared__ int bad;
   const int tid = threadIdx.x;
-  if (tid == 0) { bad = 0; seg.totals[7] = 0; }
+  if (tid == 0) { bad = 0; seg.totals[7] = 0; seg.totals[6] = gen; }   // [6]: stamp of this call
   __syncthreads();
 
   // --- first block of every sequence
@@ -187,10 +187,10 @@ ba_segment_tokens_kernel(int B, int T, ba_segments seg) {
 }  // namespace
 
 ba_status ba_segment_launch(ba_ctx *ctx, const int32_t *d_block_lens, const int32_t *d_seq_nblocks,
-                            int32_t batch, int32_t n_blocks, int32_t n_tokens, int mode,
+                            int32_t batch, int32_t n_blocks, int32_t n_tokens, int mode, int32_t gen,
                             const ba_segments *seg, cudaStream_t stream) {
   ba_segment_blocks_kernel<<<1, kScanThreads, 0, stream>>>(
-      d_block_lens, d_seq_nblocks, batch, n_blocks, n_tokens, mode, seg->q_tile_tokens, *seg,
+      d_block_lens, d_seq_nblocks, batch, n_blocks, n_tokens, mode, seg->q_tile_tokens, gen, *seg,
       ctx->dev_status);
   BA_CUDA_TRY(cudaGetLastError());
   ba_segment_tokens_kernel<<<(n_tokens + 255) / 256, 256, 0, stream>>>(n_blocks, n_tokens, *seg);

@@ -53,34 +53,13 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
   return ok != 0;
 }
 
-// The same with a suspend-time hint: the thread may be parked by the hardware for up to `ns`
-// nanoseconds and resumes as soon as the phase completes.
-__device__ __forceinline__ bool mbar_try_wait_hint(uint64_t *bar, uint32_t parity, uint32_t ns) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}\n"
-      : "=r"(ok)
-      : "r"(smem_u32(bar)), "r"(parity), "r"(ns)
-      : "memory");
-  return ok != 0;
-}
-
 // Bounded wait.  Gives up after about one second (kWaitLimitNs on the global nanosecond timer)
 // or as soon as another thread of the CTA has raised *abort_flag (a shared-memory word); the
 // caller then leaves its role loop.  A wait that gives up raises the flag itself.  Legitimate
 // waits in these kernels last microseconds.
 constexpr unsigned long long kWaitLimitNs = 1000000000ull;
-#ifndef BA_FAST_POLLS
-#define BA_FAST_POLLS 64      // polls before the slow path (timer, abort flag, back-off)
-#endif
-#ifndef BA_WAIT_HINT_NS
-#define BA_WAIT_HINT_NS 0     // > 0: the slow path parks the thread with this suspend-time hint instead of sleeping
-#endif
-#ifndef BA_SLEEP_NS
-#define BA_SLEEP_NS 32        // back-off between polls on the slow path
-#endif
+constexpr int kFastPolls = 64;          // polls before the slow path (timer, abort flag, back-off)
+constexpr unsigned kSleepNs = 32;       // back-off between polls on the slow path
 __device__ __forceinline__ unsigned long long global_ns() {
   unsigned long long t;
   asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
@@ -88,21 +67,15 @@ __device__ __forceinline__ unsigned long long global_ns() {
 }
 __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag) {
 #pragma unroll 1
-  for (int it = 0; it < BA_FAST_POLLS; ++it)
+  for (int it = 0; it < kFastPolls; ++it)
     if (mbar_try_wait(bar, parity)) return true;
   const unsigned long long t0 = global_ns();
 #pragma unroll 1
   for (uint32_t it = 0;; ++it) {
-#if BA_WAIT_HINT_NS > 0
-    if (mbar_try_wait_hint(bar, parity, BA_WAIT_HINT_NS)) return true;
-#else
     if (mbar_try_wait(bar, parity)) return true;
-#endif
     if (*abort_flag) return false;
     if (global_ns() - t0 > kWaitLimitNs) break;
-#if BA_WAIT_HINT_NS == 0
-    if (BA_SLEEP_NS > 0) __nanosleep(it > 4096 ? 256 : BA_SLEEP_NS);
-#endif
+    __nanosleep(it > 4096 ? 256 : kSleepNs);
   }
   *abort_flag = 1;
   return false;
@@ -167,24 +140,6 @@ __device__ __forceinline__ void tmem_st_32x32b_x32(uint32_t taddr, const uint32_
         "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
         "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
         "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
-      : "memory");
-}
-
-__device__ __forceinline__ void tmem_ld_32x32b_x16(uint32_t taddr, uint32_t (&r)[16]) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-      : "r"(taddr)
-      : "memory");
-}
-__device__ __forceinline__ void tmem_st_32x32b_x16(uint32_t taddr, const uint32_t (&r)[16]) {
-  asm volatile(
-      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
-      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
-      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
-        "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
       : "memory");
 }
 

@@ -6,14 +6,15 @@ must not hit the device-wide synchronisation an allocation implies.  They cannot
 create a context (its workspace is allocated), so this entry point keeps its
 angle table in an array built into the library.  The test drives it through the
 C ABI twice in a row, with different prompts, and requires the same bytes the
-context-based ba_reencode_k produces: the second call must not see anything the
-first one left in the shared table.  It runs last so that a failure here cannot
+context-based ba_reencode_k produces (and a correct rounding of the fp64 oracle's
+rotation): the second call must not see anything the first one left in the shared table.  It runs last so that a failure here cannot
 hide results of the other tests.
 """
 import numpy as np
 import pytest
 import torch
 
+from oracle import block_attention as ob
 from paper_2409_15355_b200 import binding as B
 from paper_2409_15355_b200 import runtime as R
 from paper_2409_15355_b200 import workloads as W
@@ -40,6 +41,15 @@ def _both(w, layout):
     assert c.device_status() == B.BA_OK and int(status.item()) == 0
     assert torch.equal(got, want)
     assert not torch.equal(got, src[:Tc]) or w.pool_lens is not None
+    # and against the oracle directly: every key a correct rounding of the fp64 rotation
+    t = ob.segment_tables(w.block_lens, w.seq_nblocks)
+    src64 = W.bf16_bits_to_f64(x["k_cache"] if w.pool_lens is None else x["k_pool"])
+    ref = ob.reencode_blocks(src64, None if w.pool_lens is None else x["src_off"], t["cache_cu"], t["cache_delta"],
+                             w.rope_theta, ob.ROPE_HALF if layout == B.BA_ROPE_HALF else ob.ROPE_ADJACENT)
+    g = W.bf16_bits_to_f64(R.device_to_bits(got))
+    assert (np.abs(g - ref) <= np.abs(ref) * 2.0 ** -8 * 1.01 + 1e-6).all()
+    r = W.bf16_bits_to_f64(W.f32_to_bf16_bits(ref.astype(np.float32)))
+    assert (g == r).mean() >= 0.995
     c.close()
     return seg.n_cached_blocks
 
