@@ -290,21 +290,68 @@ ba_status ba_final_attend(ba_ctx *ctx, const void *q_f, const void *k_f, const v
  * other side of the dot product: (R(p) q) . (R(delta + t) k) = (R(-delta) R(p) q) . (R(t) k),
  * so the query tiles are rotated once per cached block on chip and the cached keys are neither
  * rewritten nor read twice.  The result equals ba_reencode_k followed by ba_final_attend up to
- * the rounding of the rotated operand to bf16 (queries here, keys there).  Re-encoded keys are
- * not produced; a later decode phase that wants them calls ba_reencode_k off the critical path.
+ * the rounding of the rotated operand to bf16 (queries here, keys there).  The re-encoded keys
+ * themselves -- what the rest of generation reads -- are written as a side output when k_out is
+ * given: otherwise idle warps of the same launch rotate the cached keys from k_src to k_out
+ * (bit-identical to ba_reencode_k) while the attention runs; they are complete when the call is.
  *   q_f, k_f, v_f   as for ba_final_attend
  *   k_src, v_src    bf16 [n_src_rows, n_kv_heads, head_dim]: cached block c (cache order, as in
  *                   seg->cache_cu) occupies rows src_off[c] .. src_off[c] + length - 1 of both, or
  *                   rows cache_cu[c] .. when src_off is NULL (cache packing)
  *   n_cache_rows    total cached rows of the batch (= cache_cu[Bc])
+ *   k_out           NULL, or bf16 [n_cache_rows, n_kv_heads, head_dim] (cache packing), not k_src
  *   seg             tables of ba_segment(); its cache_rope table holds the rotations
  * A queued ba_reencode_k_deferred job is run as a stand-alone launch first.
  */
 ba_status ba_final_attend_fused(ba_ctx *ctx, const void *q_f, const void *k_f, const void *v_f,
                                 int32_t n_final_rows, const void *k_src, const void *v_src,
                                 int32_t n_src_rows, const int32_t *src_off, int32_t n_cache_rows,
-                                void *o, float *lse, const ba_segments *seg, ba_mode mode,
+                                void *k_out, void *o, float *lse, const ba_segments *seg, ba_mode mode,
                                 ba_out_dtype out_dtype, void *stream);
+
+/*
+ * Paged KV pool (Section 2.3: what the cache holds; Section 2.5 step 1: the cache look-up).  A serving
+ * cache rarely keeps a passage in one piece: it hands out fixed-size pages.  Here the cached keys and
+ * values of all blocks live in pool tensors [n_pages * page_rows, n_kv_heads, head_dim] (one for K, one
+ * for V, same paging), page `g` being rows g * page_rows .. (g + 1) * page_rows - 1.  Cached block c
+ * (cache order, as in seg->cache_cu) owns the pages page_idx[page_cu[c]] .. page_idx[page_cu[c+1] - 1],
+ * in that order: row t of the block is row t % page_rows of its page number t / page_rows; a block
+ * of length L has ceil(L / page_rows) pages and the rest of its last page is not part of it.  Those
+ * unused rows must hold finite values (a pool that started out zeroed, or stale keys and values):
+ * they are masked, but a tensor-core product of zero with a NaN bit pattern would still be NaN.
+ *   page_rows   a power of two, 16 .. 65536
+ *   page_cu     device int32 [n_blocks + 1], page_idx device int32 [page_cu[n_blocks]]
+ * A page number outside [0, n_pages) is never read: ba_reencode_k_paged skips the row and reports
+ * BA_ERR_INVALID_ARG through ba_last_device_status(); the attention calls read zeros in its place.
+ */
+typedef struct {
+  int32_t page_rows;
+  int32_t n_pages;
+  const int32_t *page_cu;
+  const int32_t *page_idx;
+} ba_page_table;
+
+/* ba_reencode_k with the cached keys gathered from a paged pool (Eq. 1-3 as there); k_dst in cache
+ * packing, cu / delta / n_blocks / n_rows as for ba_reencode_k. */
+ba_status ba_reencode_k_paged(ba_ctx *ctx, const void *k_pool, const ba_page_table *pages, void *k_dst,
+                              const int32_t *cu, const int32_t *delta, int32_t n_blocks, int32_t n_rows,
+                              void *stream);
+
+/* ba_final_attend (Section 2.5 step 3) with the cached VALUES read in place from a paged pool; the
+ * re-encoded keys k_cache are in cache packing (the output of ba_reencode_k_paged).  A key tile of the
+ * kernel never spans two pages: it is assembled from one copy per page. */
+ba_status ba_final_attend_paged(ba_ctx *ctx, const void *q_f, const void *k_f, const void *v_f,
+                                int32_t n_final_rows, const void *k_cache, int32_t n_cache_rows,
+                                const void *v_pool, const ba_page_table *pages, void *o, float *lse,
+                                const ba_segments *seg, ba_mode mode, ba_out_dtype out_dtype, void *stream);
+
+/* ba_final_attend_fused (Section 2.5 steps 2-3 in one launch) with cached keys (at cache-time positions)
+ * and values both read in place from paged pools that share one page table; k_out as there. */
+ba_status ba_final_attend_fused_paged(ba_ctx *ctx, const void *q_f, const void *k_f, const void *v_f,
+                                      int32_t n_final_rows, const void *k_pool, const void *v_pool,
+                                      const ba_page_table *pages, int32_t n_cache_rows, void *k_out,
+                                      void *o, float *lse, const ba_segments *seg, ba_mode mode,
+                                      ba_out_dtype out_dtype, void *stream);
 
 #ifdef __cplusplus
 }

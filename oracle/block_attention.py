@@ -226,6 +226,19 @@ def reencode_delta(k_cached, delta, base, layout=ROPE_ADJACENT):
     return rotate(k_cached, np.full(k_cached.shape[:1] + (1,), float(delta)), base, layout)
 
 
+def paged_rows(cache_lens, page_rows, page_cu, page_idx):
+    """Pool row of every cached row when the cache is a pool of fixed-size pages (Section 2.3: what the
+    cache holds; Section 2.5 step 1: the look-up).  Cached block c owns the pages
+    page_idx[page_cu[c]] .. page_idx[page_cu[c+1] - 1], in order; its row t is row t mod page_rows of its
+    page number t div page_rows.  Plain loops; the result indexes the pool tensor."""
+    rows = []
+    for c, L in enumerate(cache_lens):
+        for t in range(int(L)):
+            page = int(page_idx[int(page_cu[c]) + t // page_rows])
+            rows.append(page * page_rows + t % page_rows)
+    return np.asarray(rows, dtype=np.int64)
+
+
 def reencode_blocks(k_src, src_off, cache_cu, cache_delta, base, layout=ROPE_ADJACENT):
     """Re-encode every cached block (Section 2.5, step 2).  Block c occupies
     rows cache_cu[c]..cache_cu[c+1] of the result; its source rows start at

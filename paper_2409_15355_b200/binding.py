@@ -24,7 +24,7 @@ EXPORTS = [
     "ba_create", "ba_destroy", "ba_status_string", "ba_workspace_bytes", "ba_last_device_status",
     "ba_launch_count", "ba_segments_bytes", "ba_segment", "ba_reencode_k", "ba_block_prefill",
     "ba_final_attend", "ba_reencode_k_noalloc", "ba_selftest_wait_expiry", "ba_reencode_k_deferred", "ba_flush",
-    "ba_final_attend_fused",
+    "ba_final_attend_fused", "ba_reencode_k_paged", "ba_final_attend_paged", "ba_final_attend_fused_paged",
 ]
 BA_NOALLOC_MAX_BLOCKS = 4096
 
@@ -44,6 +44,15 @@ class ba_segments(C.Structure):
             "block_seq", "block_kv_begin", "block_part_off", "block_is_final", "cache_block",
             "cache_cu", "cache_delta", "tok_block", "tok_pos", "tok_pos_local", "cu_qtile",
             "cu_ftile", "cache_tile_cu", "totals", "cache_rope")]
+
+
+class ba_page_table(C.Structure):
+    _fields_ = [("page_rows", C.c_int32), ("n_pages", C.c_int32), ("page_cu", C.c_void_p), ("page_idx", C.c_void_p)]
+
+
+def make_page_table(page_rows: int, n_pages: int, page_cu, page_idx) -> "ba_page_table":
+    """page_cu / page_idx: torch int32 CUDA tensors (kept alive by the caller)."""
+    return ba_page_table(page_rows, n_pages, _ptr(page_cu), _ptr(page_idx))
 
 
 class BaError(RuntimeError):
@@ -84,8 +93,14 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.ba_block_prefill.argtypes = [vp, vp, vp, vp, vp, vp, C.POINTER(ba_segments), C.c_int, C.c_int, vp]
     lib.ba_final_attend.argtypes = [vp, vp, vp, vp, i32, vp, vp, i32, vp, i32, vp, vp,
                                     C.POINTER(ba_segments), C.c_int, C.c_int, vp]
-    lib.ba_final_attend_fused.argtypes = [vp, vp, vp, vp, i32, vp, vp, i32, vp, i32, vp, vp,
+    lib.ba_final_attend_fused.argtypes = [vp, vp, vp, vp, i32, vp, vp, i32, vp, i32, vp, vp, vp,
                                           C.POINTER(ba_segments), C.c_int, C.c_int, vp]
+    pt = C.POINTER(ba_page_table)
+    lib.ba_reencode_k_paged.argtypes = [vp, vp, pt, vp, vp, vp, i32, i32, vp]
+    lib.ba_final_attend_paged.argtypes = [vp, vp, vp, vp, i32, vp, i32, vp, pt, vp, vp,
+                                          C.POINTER(ba_segments), C.c_int, C.c_int, vp]
+    lib.ba_final_attend_fused_paged.argtypes = [vp, vp, vp, vp, i32, vp, vp, pt, i32, vp, vp, vp,
+                                                C.POINTER(ba_segments), C.c_int, C.c_int, vp]
     for name in EXPORTS:
         # without argtypes ctypes would pass addresses as 32-bit ints
         if getattr(lib, name).argtypes is None:
@@ -205,10 +220,11 @@ def ba_block_prefill(ctx, q, k, v, o, lse, seg, mode, out_dtype, stream=None):
 
 
 def ba_final_attend_fused(ctx, q_f, k_f, v_f, n_final_rows, k_src, v_src, n_src_rows, src_off,
-                          n_cache_rows, o, lse, seg, mode, out_dtype, stream=None):
+                          n_cache_rows, o, lse, seg, mode, out_dtype, stream=None, k_out=None):
+    """k_out: optional bf16 tensor [n_cache_rows, n_kv_heads, head_dim] that receives the re-encoded keys."""
     _check(load_library().ba_final_attend_fused(ctx, _ptr(q_f), _ptr(k_f), _ptr(v_f), n_final_rows,
                                                 _ptr(k_src), _ptr(v_src), n_src_rows, _ptr(src_off),
-                                                n_cache_rows, _ptr(o), _ptr(lse), C.byref(seg), mode,
+                                                n_cache_rows, _ptr(k_out), _ptr(o), _ptr(lse), C.byref(seg), mode,
                                                 out_dtype, _stream_ptr(stream)), "ba_final_attend_fused")
 
 
@@ -218,3 +234,24 @@ def ba_final_attend(ctx, q_f, k_f, v_f, n_final_rows, k_cache, v_cache, n_cache_
                                           _ptr(k_cache), _ptr(v_cache), n_cache_rows, _ptr(v_src_off),
                                           n_v_rows, _ptr(o), _ptr(lse), C.byref(seg), mode, out_dtype,
                                           _stream_ptr(stream)), "ba_final_attend")
+
+
+def ba_reencode_k_paged(ctx, k_pool, pages, k_dst, cu, delta, n_blocks, n_rows, stream=None):
+    _check(load_library().ba_reencode_k_paged(ctx, _ptr(k_pool), C.byref(pages), _ptr(k_dst), _ptr(cu), _ptr(delta),
+                                              n_blocks, n_rows, _stream_ptr(stream)), "ba_reencode_k_paged")
+
+
+def ba_final_attend_paged(ctx, q_f, k_f, v_f, n_final_rows, k_cache, n_cache_rows, v_pool, pages, o, lse, seg,
+                          mode, out_dtype, stream=None):
+    _check(load_library().ba_final_attend_paged(ctx, _ptr(q_f), _ptr(k_f), _ptr(v_f), n_final_rows, _ptr(k_cache),
+                                                n_cache_rows, _ptr(v_pool), C.byref(pages), _ptr(o), _ptr(lse),
+                                                C.byref(seg), mode, out_dtype, _stream_ptr(stream)),
+           "ba_final_attend_paged")
+
+
+def ba_final_attend_fused_paged(ctx, q_f, k_f, v_f, n_final_rows, k_pool, v_pool, pages, n_cache_rows, o, lse, seg,
+                                mode, out_dtype, stream=None, k_out=None):
+    _check(load_library().ba_final_attend_fused_paged(ctx, _ptr(q_f), _ptr(k_f), _ptr(v_f), n_final_rows,
+                                                      _ptr(k_pool), _ptr(v_pool), C.byref(pages), n_cache_rows,
+                                                      _ptr(k_out), _ptr(o), _ptr(lse), C.byref(seg), mode, out_dtype,
+                                                      _stream_ptr(stream)), "ba_final_attend_fused_paged")

@@ -133,6 +133,9 @@ ba_status ba_create(ba_ctx **out, const ba_config *cfg, int device, size_t works
   if (cudaMalloc(&ctx->dev_status, 256) != cudaSuccess ||
       cudaMemset(ctx->dev_status, 0, 256) != cudaSuccess ||
       (workspace_bytes && cudaMalloc(&ctx->workspace, workspace_bytes) != cudaSuccess) ||
+      // launch counters of the attention kernels (below the scratch area): zero once, every launch leaves them zero
+      (workspace_bytes >= ba_scratch_offset(ctx) &&
+       cudaMemset((char *)ctx->workspace + ba_scratch_offset(ctx) - 256, 0, 256) != cudaSuccess) ||
       ba_attend_sm100_setup(ctx) != BA_OK) {
     cudaGetLastError();
     if (ctx->workspace) cudaFree(ctx->workspace);
@@ -195,7 +198,10 @@ ba_status ba_segment(ba_ctx *ctx, const int32_t *block_lens, const int32_t *seq_
     for (int q = 0; q < batch; ++q) { if (seq_nblocks[q] < 1) return BA_ERR_INVALID_ARG; nb_sum += seq_nblocks[q]; }
     if (sum != n_tokens || nb_sum != n_blocks) return BA_ERR_INVALID_ARG;
     size_t need = (size_t)(n_blocks + batch) * 4;
-    if (!ctx->workspace || need > ctx->workspace_bytes) return BA_ERR_WORKSPACE;
+    // staging area: the start of the workspace, up to the launch counters below the scratch area
+    if (!ctx->workspace || need > ctx->workspace_bytes ||
+        (ctx->workspace_bytes >= ba_scratch_offset(ctx) && need > ba_scratch_offset(ctx) - 256))
+      return BA_ERR_WORKSPACE;
     int32_t *stage = (int32_t *)ctx->workspace;
     BA_CUDA_TRY(cudaMemcpyAsync(stage, block_lens, (size_t)n_blocks * 4, cudaMemcpyHostToDevice, s));
     BA_CUDA_TRY(cudaMemcpyAsync(stage + n_blocks, seq_nblocks, (size_t)batch * 4, cudaMemcpyHostToDevice, s));
@@ -378,7 +384,7 @@ ba_status ba_final_attend(ba_ctx *ctx, const void *q_f, const void *k_f, const v
 ba_status ba_final_attend_fused(ba_ctx *ctx, const void *q_f, const void *k_f, const void *v_f,
                                 int32_t n_final_rows, const void *k_src, const void *v_src,
                                 int32_t n_src_rows, const int32_t *src_off, int32_t n_cache_rows,
-                                void *o, float *lse, const ba_segments *seg, ba_mode mode,
+                                void *k_out, void *o, float *lse, const ba_segments *seg, ba_mode mode,
                                 ba_out_dtype out_dtype, void *stream) {
   ba_status st = check_attend_common(ctx, q_f, k_f, v_f, o, seg, mode, out_dtype);
   if (st != BA_OK) return st;
@@ -387,6 +393,7 @@ ba_status ba_final_attend_fused(ba_ctx *ctx, const void *q_f, const void *k_f, c
     if (!k_src || !v_src || !aligned16(k_src) || !aligned16(v_src)) return BA_ERR_INVALID_ARG;
     if (n_src_rows < 1 || !seg->cache_rope || !seg->cache_tile_cu) return BA_ERR_INVALID_ARG;
     if (!src_off && n_src_rows < n_cache_rows) return BA_ERR_INVALID_ARG;
+    if (k_out && (!aligned16(k_out) || k_out == k_src)) return BA_ERR_INVALID_ARG;   // the attention reads k_src meanwhile
   }
   if ((long long)n_final_rows + n_cache_rows != seg->n_tokens) return BA_ERR_SHAPE;
   BA_CUDA_TRY(cudaSetDevice(ctx->device));
@@ -398,8 +405,104 @@ ba_status ba_final_attend_fused(ba_ctx *ctx, const void *q_f, const void *k_f, c
   a.n_cache_rows = n_cache_rows;
   a.fused = 1;
   a.k_src_off = src_off; a.n_k_rows = n_src_rows;
+  a.k_out = n_cache_rows > 0 ? k_out : nullptr;
   // values: addressed like the keys.  The kernel's value map covers n_v_rows rows when an offset table is given.
   a.v_src_off = src_off; a.n_v_rows = n_src_rows;
+  a.out_f32 = out_dtype == BA_OUT_F32;
+  a.final_only = 1;
+  return ba_attend_launch(ctx, a, seg, (cudaStream_t)stream);
+}
+
+
+static ba_status check_pages(const ba_page_table *pg) {
+  if (!pg || !pg->page_cu || !pg->page_idx) return BA_ERR_INVALID_ARG;
+  if (pg->page_rows < 16 || pg->page_rows > 65536 || (pg->page_rows & (pg->page_rows - 1))) return BA_ERR_UNSUPPORTED;
+  if (pg->n_pages < 1 || (long long)pg->n_pages * pg->page_rows > 0x7fffffffLL) return BA_ERR_INVALID_ARG;
+  return BA_OK;
+}
+
+ba_status ba_reencode_k_paged(ba_ctx *ctx, const void *k_pool, const ba_page_table *pages, void *k_dst,
+                              const int32_t *cu, const int32_t *delta, int32_t n_blocks, int32_t n_rows,
+                              void *stream) {
+  ba_status st = check_pages(pages);
+  if (st != BA_OK) return st;
+  const int32_t n_src_rows = pages->n_pages * pages->page_rows;
+  bool nothing;
+  st = check_reencode_args(ctx, k_pool, nullptr, n_src_rows, k_dst, cu, delta, n_blocks, n_rows, &nothing);
+  if (st != BA_OK || nothing) return st;
+  if (k_pool == k_dst) return BA_ERR_INVALID_ARG;            // a gather cannot run in place
+  BA_CUDA_TRY(cudaSetDevice(ctx->device));
+  const bool reuse = delta == ctx->seg_delta && n_blocks == ctx->seg_rope_blocks;
+  float2 *table = nullptr; size_t bytes;
+  if (!reuse) {
+    st = place_table(ctx, n_blocks, &table, &bytes);
+    if (st != BA_OK) return st;
+    st = ba_reencode_table_launch(ctx, delta, n_blocks, table, (cudaStream_t)stream);
+    if (st != BA_OK) return st;
+  }
+  ba_reencode_job job = ba_make_reencode_job(ctx, k_pool, nullptr, n_src_rows, k_dst, cu, delta, n_blocks, n_rows,
+                                             reuse ? ctx->seg_rope : table);
+  if (reuse) { job.gen = ctx->seg_gen; job.gen_expected = ctx->seg_gen_value; }
+  job.page_cu = pages->page_cu; job.page_idx = pages->page_idx;
+  job.page_lg = 0;
+  while ((1 << job.page_lg) < pages->page_rows) ++job.page_lg;
+  return ba_reencode_main_launch(ctx, job, (cudaStream_t)stream);
+}
+
+ba_status ba_final_attend_paged(ba_ctx *ctx, const void *q_f, const void *k_f, const void *v_f,
+                                int32_t n_final_rows, const void *k_cache, int32_t n_cache_rows,
+                                const void *v_pool, const ba_page_table *pages, void *o, float *lse,
+                                const ba_segments *seg, ba_mode mode, ba_out_dtype out_dtype, void *stream) {
+  ba_status st = check_attend_common(ctx, q_f, k_f, v_f, o, seg, mode, out_dtype);
+  if (st != BA_OK) return st;
+  if (n_final_rows < 0 || n_cache_rows < 0) return BA_ERR_INVALID_ARG;
+  if ((long long)n_final_rows + n_cache_rows != seg->n_tokens) return BA_ERR_SHAPE;
+  ba_attend_args a;
+  memset(&a, 0, sizeof(a));
+  if (n_cache_rows > 0) {
+    st = check_pages(pages);
+    if (st != BA_OK) return st;
+    if (!k_cache || !v_pool || !aligned16(k_cache) || !aligned16(v_pool) || !seg->cache_tile_cu) return BA_ERR_INVALID_ARG;
+    a.page_rows = pages->page_rows; a.page_cu = pages->page_cu; a.page_idx = pages->page_idx;
+    a.n_v_rows = pages->n_pages * pages->page_rows;
+  }
+  BA_CUDA_TRY(cudaSetDevice(ctx->device));
+  a.q = (const __nv_bfloat16 *)q_f; a.k = (const __nv_bfloat16 *)k_f; a.v = (const __nv_bfloat16 *)v_f;
+  a.o = o; a.lse = lse; a.n_q_rows = n_final_rows; a.n_kv_rows = n_final_rows;
+  a.k_cache = (const __nv_bfloat16 *)k_cache; a.v_cache = (const __nv_bfloat16 *)v_pool;
+  a.n_cache_rows = n_cache_rows;
+  a.out_f32 = out_dtype == BA_OUT_F32;
+  a.final_only = 1;
+  return ba_attend_launch(ctx, a, seg, (cudaStream_t)stream);
+}
+
+ba_status ba_final_attend_fused_paged(ba_ctx *ctx, const void *q_f, const void *k_f, const void *v_f,
+                                      int32_t n_final_rows, const void *k_pool, const void *v_pool,
+                                      const ba_page_table *pages, int32_t n_cache_rows, void *k_out,
+                                      void *o, float *lse, const ba_segments *seg, ba_mode mode,
+                                      ba_out_dtype out_dtype, void *stream) {
+  ba_status st = check_attend_common(ctx, q_f, k_f, v_f, o, seg, mode, out_dtype);
+  if (st != BA_OK) return st;
+  if (n_final_rows < 0 || n_cache_rows < 0) return BA_ERR_INVALID_ARG;
+  if ((long long)n_final_rows + n_cache_rows != seg->n_tokens) return BA_ERR_SHAPE;
+  ba_attend_args a;
+  memset(&a, 0, sizeof(a));
+  if (n_cache_rows > 0) {
+    st = check_pages(pages);
+    if (st != BA_OK) return st;
+    if (!k_pool || !v_pool || !aligned16(k_pool) || !aligned16(v_pool)) return BA_ERR_INVALID_ARG;
+    if (!seg->cache_rope || !seg->cache_tile_cu) return BA_ERR_INVALID_ARG;
+    if (k_out && (!aligned16(k_out) || k_out == k_pool)) return BA_ERR_INVALID_ARG;
+    a.page_rows = pages->page_rows; a.page_cu = pages->page_cu; a.page_idx = pages->page_idx;
+    a.n_k_rows = a.n_v_rows = pages->n_pages * pages->page_rows;
+    a.k_out = k_out;
+  }
+  BA_CUDA_TRY(cudaSetDevice(ctx->device));
+  a.q = (const __nv_bfloat16 *)q_f; a.k = (const __nv_bfloat16 *)k_f; a.v = (const __nv_bfloat16 *)v_f;
+  a.o = o; a.lse = lse; a.n_q_rows = n_final_rows; a.n_kv_rows = n_final_rows;
+  a.k_cache = (const __nv_bfloat16 *)k_pool; a.v_cache = (const __nv_bfloat16 *)v_pool;
+  a.n_cache_rows = n_cache_rows;
+  a.fused = 1;
   a.out_f32 = out_dtype == BA_OUT_F32;
   a.final_only = 1;
   return ba_attend_launch(ctx, a, seg, (cudaStream_t)stream);

@@ -64,9 +64,11 @@ constexpr float kRescaleThreshold = 8.0f;
 constexpr int kBgStageBytes = 16384; // two spare warps x two stages of source rows
 constexpr int kWorkSlots = 4;      // ring of published work entries (power of two)
 // Register split after launch (168 per thread): the service warps give registers to the softmax warps.
-// 128 * kServiceRegs + 256 * kSoftmaxRegs <= 384 * 168.
-constexpr int kServiceRegs = 72;
-constexpr int kSoftmaxRegs = 216;
+// 128 * kServiceRegs + 256 * kSoftmaxRegs <= 384 * 168.  The MMA thread keeps a work entry, descriptors
+// and ring positions live and spills below about 88; the softmax warps start to spill below 208.  On the
+// fused path the softmax warps also prepare query versions and need the larger share.
+constexpr int kServiceRegsPlain = 88, kSoftmaxRegsPlain = 208;
+constexpr int kServiceRegsFused = 72, kSoftmaxRegsFused = 216;
 
 struct AttnParams {
   void *o;
@@ -83,14 +85,21 @@ struct AttnParams {
   float *o_part;                  // [n_splits, n_q_rows, Hq, D] fp32, each normalised by its own denominator
   float *lse_part;                // [n_splits, n_q_rows, Hq] natural-log denominators (-inf: split saw no key)
   const int32_t *v_src_off;       // non-null: values of cached block c start at pool row v_src_off[c]
-  int persistent;                 // 1: CTAs draw work from work_counter; 0: CTA b handles entry b only
-  int32_t *work_counter;          // device word, zero at launch: next entry of the work list
+  int persistent;                 // 1: CTAs draw work from counters[0]; 0: CTA b handles entry b only
+  // three device words, zero at launch and zero again when the launch ends (its last CTA clears them):
+  // [0] next entry of the work list, [1] next chunk of the background job, [2] CTAs that have finished
+  int32_t *counters;
   ba_reencode_job bg;             // bg.n_rows > 0: a re-encoding job the two spare warps carry out meanwhile
-  int32_t *bg_counter;            // device word, zero at launch: next chunk of that job
   int bg_rows_per_chunk;
+  int bg_direct;                  // the job moves its rows global -> global (no staging in shared memory)
   ba_segments seg;
   const int32_t *k_src_off;       // non-null: keys of cached block c start at pool row k_src_off[c] (fused path only)
   int walk;                       // cached keys are walked block by block (a tile never spans two blocks)
+  // paged pool: cached block c owns the pages page_idx[page_cu[c] .. page_cu[c+1]) of 1 << page_lg rows each;
+  // row t of the block is row t & (page_rows - 1) of page t >> page_lg of its list.  Applies to the values
+  // (v_paged) and, on the fused path, to the keys (k_paged).
+  const int32_t *page_cu, *page_idx;
+  int page_lg, k_paged, v_paged;
   int fused;                      // cached keys are at cache-time positions: queries are counter-rotated per block
   int rope_layout;
   const float2 *q_rope;           // fused: [cached blocks][D/2] (cos, sin) of delta_c * theta_m
@@ -306,6 +315,8 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
                        const __grid_constant__ CUtensorMap tmap_vc, const AttnParams p) {
   using L = Layout<D>;
   // setmaxnreg is a warpgroup-wide instruction: the four service warps (8-11) must ask for the same count
+  constexpr int kServiceRegs = kFused ? kServiceRegsFused : kServiceRegsPlain;
+  constexpr int kSoftmaxRegs = kFused ? kSoftmaxRegsFused : kSoftmaxRegsPlain;
   constexpr int kProdRegs = kServiceRegs, kMmaRegs = kServiceRegs, kSpareRegs = kServiceRegs;
   extern __shared__ uint8_t smem_raw[];
   uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -357,7 +368,7 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
         ok = mbar_wait(&ctrl->work_empty[slot], ((n_work / kWorkSlots) & 1) ^ 1, abort_flag);
         if (!ok) break;
         // persistent launch: next entry of the global list; one-item launch: this CTA's own entry, then stop
-        const int w = p.persistent ? atomicAdd(p.work_counter, 1) : (n_work == 0 ? (int)blockIdx.x : 0x7fffffff);
+        const int w = p.persistent ? atomicAdd(p.counters, 1) : (n_work == 0 ? (int)blockIdx.x : 0x7fffffff);
         const bool more = tables_ok && next_work(p, w, wk);
         ctrl->work_ring[slot] = more ? w : -1;
         mbar_arrive(&ctrl->work_full[slot]);
@@ -382,12 +393,14 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
         // whole block ahead, so that no tile waits for a table look-up.
         int pc = 0, poff = 0;
         int c_len = 0, k_base = 0, v_base = 0, n_len = 0, n_kbase = 0, n_vbase = 0;
+        // (for a paged operand the "base" of a block is the start of its page list)
         auto load_block = [&](int b, int &len, int &kb, int &vb) {
           if (b >= p.seg.n_cached_blocks) return;
           const int c0 = __ldg(p.seg.cache_cu + b);
           len = __ldg(p.seg.cache_cu + b + 1) - c0;
-          kb = p.k_src_off ? __ldg(p.k_src_off + b) : c0;
-          vb = p.v_src_off ? __ldg(p.v_src_off + b) : c0;
+          const int pg = p.page_cu ? __ldg(p.page_cu + b) : 0;
+          kb = p.k_paged ? pg : (p.k_src_off ? __ldg(p.k_src_off + b) : c0);
+          vb = p.v_paged ? pg : (p.v_src_off ? __ldg(p.v_src_off + b) : c0);
         };
         if (p.walk && wk.tile0 < it.n_cache_tiles) {
           const int target = it.ctile0 + wk.tile0;
@@ -396,10 +409,26 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
           load_block(pc, c_len, k_base, v_base);
           load_block(pc + 1, n_len, n_kbase, n_vbase);
         }
+        // one 128-row tile of a paged operand: a box per page (pages of 128 rows or more hold whole tiles).
+        // Parts of the tile past the end of the block are fetched from the block's last page: they are
+        // masked, but what the tensor core multiplies by zero must still be finite.
+        auto load_paged_tile = [&](uint8_t *dst, const CUtensorMap *m, uint64_t *bar, int list0, int off, int len) {
+          const int page_rows = 1 << p.page_lg;
+          const int sub_rows = min(kBlockN, page_rows), n_sub = kBlockN / sub_rows;
+          const int last_page = (len - 1) >> p.page_lg;
+          for (int sb = 0; sb < n_sub; ++sb) {
+            const int t0 = off + sb * sub_rows;
+            const int page = min(t0 >> p.page_lg, last_page);
+            const int row = (__ldg(p.page_idx + list0 + page) << p.page_lg) + (t0 & (page_rows - 1));
+            for (int c = 0; c < L::kChunks; ++c)
+              tma_load_3d(dst + c * L::kRegionBytes + sb * sub_rows * 128, m, bar, c * 64, wk.kv_head, row);
+          }
+        };
         for (int j = 0; j < wk.n_tiles && ok; ++j) {
           const int jt = wk.tile0 + j;
           const bool cached = jt < it.n_cache_tiles;
-          int k_row, v_row;
+          int k_row, v_row, t_off = 0, t_len = 0, t_kbase = 0, t_vbase = 0;
+          bool k_pg = false, v_pg = false;
           if (!cached) {
             k_row = v_row = it.own_row0 + (jt - it.n_cache_tiles) * kBlockN;
           } else if (!p.walk) {
@@ -407,6 +436,8 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
           } else {
             k_row = k_base + poff;
             v_row = v_base + poff;
+            k_pg = p.k_paged; v_pg = p.v_paged;
+            t_off = poff; t_len = c_len; t_kbase = k_base; t_vbase = v_base;
             ctrl->tile_valid[(gidx >> 1) & 7] = min(kBlockN, c_len - poff);   // read by the softmax warps
             poff += kBlockN;
             if (poff >= c_len) {
@@ -420,10 +451,14 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
             ok = mbar_wait(&ctrl->kv_empty[stage], ((gidx / kStages) & 1) ^ 1, abort_flag);
             if (!ok) break;
             const CUtensorMap *m = cached ? (kv ? &tmap_vc : &tmap_kc) : (kv ? &tmap_v : &tmap_k);
+            uint8_t *dst = smem + L::kRing + stage * L::kTileBytes;
             mbar_arrive_expect_tx(&ctrl->kv_full[stage], L::kTileBytes);
-            for (int c = 0; c < L::kChunks; ++c)
-              tma_load_3d(smem + L::kRing + stage * L::kTileBytes + c * L::kRegionBytes, m, &ctrl->kv_full[stage],
-                          c * 64, wk.kv_head, kv ? v_row : k_row);
+            if (kv ? v_pg : k_pg) {
+              load_paged_tile(dst, m, &ctrl->kv_full[stage], kv ? t_vbase : t_kbase, t_off, t_len);
+            } else {
+              for (int c = 0; c < L::kChunks; ++c)
+                tma_load_3d(dst + c * L::kRegionBytes, m, &ctrl->kv_full[stage], c * 64, wk.kv_head, kv ? v_row : k_row);
+            }
             ++gidx;
           }
         }
@@ -584,14 +619,19 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
   } else if (warp >= 10) {
     // ------------------------------------------------------------ spare warps: background re-encoding
     asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kSpareRegs));
-    if (p.bg.n_rows > 0) {
-      // each spare warp runs the staged engine with its own two 16 KB stages; chunks are drawn from a
-      // device-wide counter, so the job spreads over every CTA of the launch, early and late ones
+    if (p.bg.n_rows > 0 && p.bg_direct) {
+      // chunks are drawn from a device-wide counter, so the job spreads over every CTA of the launch
+      if (p.bg.layout == BA_ROPE_ADJACENT)
+        ba_reencode_direct<BA_ROPE_ADJACENT, 4>(p.bg, p.counters + 1, p.bg_rows_per_chunk, p.status);
+      else
+        ba_reencode_direct<BA_ROPE_HALF, 2>(p.bg, p.counters + 1, p.bg_rows_per_chunk, p.status);
+    } else if (p.bg.n_rows > 0) {
+      // each spare warp runs the staged engine with its own two 16 KB stages
       const int bw = warp - 10;
       ba_bg_smem *bsm = reinterpret_cast<ba_bg_smem *>(smem + L::kCtrl + 1024) + bw;
       if ((tid & 31) == 0) { mbar_init(&bsm->bar[0], 1); mbar_init(&bsm->bar[1], 1); fence_barrier_init(); }
       __syncwarp();
-      ba_reencode_background(p.bg, p.bg_counter, smem + L::kBg + bw * 2 * kBgStageBytes, bsm, p.bg_rows_per_chunk,
+      ba_reencode_background(p.bg, p.counters + 1, smem + L::kBg + bw * 2 * kBgStageBytes, bsm, p.bg_rows_per_chunk,
                              p.status, [&](uint64_t *bar, uint32_t parity) { return mbar_wait(bar, parity, abort_flag); });
     }
   } else {
@@ -715,15 +755,19 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
           for (int c = 0; c < 128; ++c)
             if (c > lim) s[c] = 0xff800000u;                 // -inf
         }
-        // eight independent running maxima (three-input max) keep the dependency chains short
-        float mx8[8];
+        // row maximum by a wide tree of three-input maxima: 128 -> 43 -> 15 -> 5 -> 1
+        float l1[43];
 #pragma unroll
-        for (int i = 0; i < 8; ++i) mx8[i] = fmaxf(__uint_as_float(s[i]), __uint_as_float(s[8 + i]));
+        for (int i = 0; i < 42; ++i) l1[i] = max3(__uint_as_float(s[3 * i]), __uint_as_float(s[3 * i + 1]), __uint_as_float(s[3 * i + 2]));
+        l1[42] = fmaxf(__uint_as_float(s[126]), __uint_as_float(s[127]));
+        float l2[15];
 #pragma unroll
-        for (int c = 16; c < 128; c += 16)
+        for (int i = 0; i < 14; ++i) l2[i] = max3(l1[3 * i], l1[3 * i + 1], l1[3 * i + 2]);
+        l2[14] = l1[42];
+        float l3[5];
 #pragma unroll
-          for (int i = 0; i < 8; ++i) mx8[i] = max3(mx8[i], __uint_as_float(s[c + i]), __uint_as_float(s[c + 8 + i]));
-        const float mx = fmaxf(max3(mx8[0], mx8[1], mx8[2]), max3(max3(mx8[3], mx8[4], mx8[5]), mx8[6], mx8[7]));
+        for (int i = 0; i < 5; ++i) l3[i] = max3(l2[3 * i], l2[3 * i + 1], l2[3 * i + 2]);
+        const float mx = fmaxf(max3(l3[0], l3[1], l3[2]), fmaxf(l3[3], l3[4]));
         const float m_new = fmaxf(m_used, mx);
         if (r == 0) BA_TR(t, j, 3);
         if (j == 0) {
@@ -750,26 +794,36 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
         uint64_t sum2[4] = {0ull, 0ull, 0ull, 0ull};       // packed (0.f, 0.f)
         const uint64_t sl2 = pack2(sl, sl), negm2 = pack2(neg_m, neg_m);
         // P is handed to the MMA warp in two halves so that PV can start on the first 64 keys
-        // while the second 64 are still being exponentiated.  The arithmetic is packed fp32x2.
-#pragma unroll
-        for (int h = 0; h < 2; ++h) {
-          uint32_t pk[32];
-#pragma unroll
-          for (int i = 0; i < 32; ++i) {
-            const int e0 = h * 64 + 2 * i, e1 = e0 + 1;
-            const uint64_t x2 = fma2(pack2(__uint_as_float(s[e0]), __uint_as_float(s[e1])), sl2, negm2);
+        // while the second 64 are still being exponentiated.  The arithmetic is packed fp32x2.  The
+        // store of the first half completes while the second half is begun.
+        {
+          constexpr int kLead = 16;       // column pairs of the second half done before the first is handed over
+          uint32_t pk[32], pk1[32];
+          auto expo = [&](int e0, uint32_t &dst, int i) {
+            const uint64_t x2 = fma2(pack2(__uint_as_float(s[e0]), __uint_as_float(s[e0 + 1])), sl2, negm2);
             float x0, x1;
             unpack2(x2, x0, x1);
             const float p0 = ex2(x0), p1 = ex2(x1);
             sum2[i & 3] = add2(sum2[i & 3], pack2(p0, p1));
             __nv_bfloat162 v = __floats2bfloat162_rn(p0, p1);
-            pk[i] = *reinterpret_cast<uint32_t *>(&v);
-          }
-          tmem_st_32x32b_x32(tS + h * 32, pk);
+            dst = *reinterpret_cast<uint32_t *>(&v);
+          };
+#pragma unroll
+          for (int i = 0; i < 32; ++i) expo(2 * i, pk[i], i);
+          tmem_st_32x32b_x32(tS, pk);
+#pragma unroll
+          for (int i = 0; i < kLead; ++i) expo(64 + 2 * i, pk1[i], i);
           tmem_wait_st();
           tc_fence_before();
-          mbar_arrive(&ctrl->p_full[t][h]);
-          if (r == 0) BA_TR(t, j, 4 + h);
+          mbar_arrive(&ctrl->p_full[t][0]);
+          if (r == 0) BA_TR(t, j, 4);
+#pragma unroll
+          for (int i = kLead; i < 32; ++i) expo(64 + 2 * i, pk1[i], i);
+          tmem_st_32x32b_x32(tS + 32, pk1);
+          tmem_wait_st();
+          tc_fence_before();
+          mbar_arrive(&ctrl->p_full[t][1]);
+          if (r == 0) BA_TR(t, j, 5);
         }
         // P of this tile is with the tensor core: time to work on the next version of the query row
         if (kFused && next_start < tile_end) {
@@ -846,7 +900,18 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
 
   tc_fence_before();
   __syncthreads();
-  if (tid == 0 && ctrl->abort_flag) ba_record_status(p.status, BA_ERR_TIMEOUT);
+  if (tid == 0) {
+    if (ctrl->abort_flag) ba_record_status(p.status, BA_ERR_TIMEOUT);
+    if (p.counters) {
+      // every role of this CTA is done with the counters; the CTA that finishes last puts them back to zero
+      __threadfence();
+      if (atomicAdd(p.counters + 2, 1) == (int)gridDim.x - 1) {
+        p.counters[0] = 0; p.counters[1] = 0;
+        __threadfence();
+        p.counters[2] = 0;
+      }
+    }
+  }
   if (warp == 9) tmem_dealloc(tmem, 512);
 }
 
@@ -1036,7 +1101,15 @@ ba_status ba_attend_sm100_launch(ba_ctx *ctx, const ba_attend_args &a, const ba_
   p.v_src_off = a.final_only ? a.v_src_off : nullptr;
   p.fused = a.final_only && a.fused && a.n_cache_rows > 0;
   p.k_src_off = p.fused ? a.k_src_off : nullptr;
-  p.walk = p.v_src_off != nullptr || p.fused;
+  p.page_cu = nullptr; p.page_idx = nullptr; p.page_lg = 0; p.k_paged = 0; p.v_paged = 0;
+  if (a.final_only && a.page_rows > 0 && a.n_cache_rows > 0) {
+    p.page_cu = a.page_cu; p.page_idx = a.page_idx;
+    while ((1 << p.page_lg) < a.page_rows) ++p.page_lg;
+    p.v_paged = 1;
+    p.k_paged = p.fused ? 1 : 0;
+    p.v_src_off = nullptr; p.k_src_off = nullptr;
+  }
+  p.walk = p.v_src_off != nullptr || p.fused || p.v_paged;
   p.rope_layout = ctx->cfg.rope_layout;
   p.q_rope = p.fused ? reinterpret_cast<const float2 *>(seg->cache_rope) : nullptr;
   if (p.fused && !p.q_rope) return BA_ERR_INVALID_ARG;
@@ -1077,12 +1150,14 @@ ba_status ba_attend_sm100_launch(ba_ctx *ctx, const ba_attend_args &a, const ba_
   // launched one CTA per entry.
   const long long work_upper = (long long)pairs_upper * (Hq / p.hpt) * n_splits;
   p.persistent = items * n_splits > 2LL * ctx->sm_count;
-  p.work_counter = nullptr;
+  // the counters live in the last 256 bytes below the scratch area: zeroed by ba_create, left at zero by every launch
+  int32_t *counters = nullptr;
+  if (ctx->workspace && ctx->workspace_bytes >= ba_scratch_offset(ctx))
+    counters = reinterpret_cast<int32_t *>(reinterpret_cast<char *>(ctx->workspace) + ba_scratch_offset(ctx) - 256);
+  p.counters = nullptr;
   if (p.persistent) {
-    // the counter lives in the last 256 bytes below the scratch area and is cleared per launch
-    if (!ctx->workspace || ctx->workspace_bytes < ba_scratch_offset(ctx)) return BA_ERR_WORKSPACE;
-    p.work_counter = reinterpret_cast<int32_t *>(reinterpret_cast<char *>(ctx->workspace) + ba_scratch_offset(ctx) - 256);
-    BA_CUDA_TRY(cudaMemsetAsync(p.work_counter, 0, sizeof(int32_t), stream));
+    if (!counters) return BA_ERR_WORKSPACE;
+    p.counters = counters;
   }
   p.o_part = nullptr; p.lse_part = nullptr;
   if (n_splits > 1) {
@@ -1096,30 +1171,43 @@ ba_status ba_attend_sm100_launch(ba_ctx *ctx, const ba_attend_args &a, const ba_
   if (!mq || !mk || !mv) return BA_ERR_CUDA;
   CUtensorMap tq = *mq, tk = *mk, tv = *mv, tkc = *mk, tvc = *mv;   // (a slot may be reused by a later look-up)
   if (a.final_only && a.n_cache_rows > 0) {
-    const CUtensorMap *mkc = cached_map(ctx, a.k_cache, D, Hkv, p.fused ? a.n_k_rows : a.n_cache_rows, 1, kBlockN);
+    const int page_box = p.v_paged ? min(kBlockN, a.page_rows) : kBlockN;
+    const CUtensorMap *mkc = cached_map(ctx, a.k_cache, D, Hkv, p.fused ? a.n_k_rows : a.n_cache_rows, 1,
+                                        p.k_paged ? page_box : kBlockN);
     if (!mkc) return BA_ERR_CUDA;
     tkc = *mkc;
-    const CUtensorMap *mvc = cached_map(ctx, a.v_cache, D, Hkv, a.v_src_off ? a.n_v_rows : a.n_cache_rows, 1, kBlockN);
+    const CUtensorMap *mvc = cached_map(ctx, a.v_cache, D, Hkv, (a.v_src_off || p.v_paged) ? a.n_v_rows : a.n_cache_rows, 1,
+                                        page_box);
     if (!mvc) return BA_ERR_CUDA;
     tvc = *mvc;
   }
   dim3 grid((unsigned)(p.persistent ? ctx->sm_count : work_upper));
   // a queued re-encoding job rides along in the spare warps; a job whose rows do not fit the
   // staging buffers is run on its own first
-  p.bg.n_rows = 0; p.bg_counter = nullptr; p.bg_rows_per_chunk = 0;
+  p.bg.n_rows = 0; p.bg_rows_per_chunk = 0; p.bg_direct = 0;
   if (ctx->has_pending) {
     const int row_bytes = ctx->pending.row_vecs * 16;
-    if (row_bytes <= kBgStageBytes && !p.fused) {   // the fused path keeps its rotated query tiles in the staging area
+    if (row_bytes <= kBgStageBytes && !p.fused && counters) {   // (the fused path has other uses for the spare warps' staging area)
       p.bg = ctx->pending;
       ctx->has_pending = 0;
       ctx->pending_table_bytes = 0;
       p.bg_rows_per_chunk = kBgStageBytes / row_bytes < 32 ? kBgStageBytes / row_bytes : 32;
-      p.bg_counter = reinterpret_cast<int32_t *>(reinterpret_cast<char *>(ctx->workspace) + ba_scratch_offset(ctx) - 128);
-      BA_CUDA_TRY(cudaMemsetAsync(p.bg_counter, 0, sizeof(int32_t), stream));
+      p.counters = counters;
     } else {
       ba_status fs = ba_flush_pending(ctx, stream);
       if (fs != BA_OK) return fs;
     }
+  }
+  if (p.fused && a.k_out) {
+    // side output of the fused call: the re-encoded keys, written by the spare warps from global to global
+    if (!counters) return BA_ERR_WORKSPACE;
+    p.bg = ba_make_reencode_job(ctx, a.k_cache, a.k_src_off, a.n_k_rows, a.k_out, seg->cache_cu, seg->cache_delta,
+                                seg->n_cached_blocks, a.n_cache_rows, reinterpret_cast<const float2 *>(seg->cache_rope));
+    if (p.k_paged) { p.bg.src_off = nullptr; p.bg.page_cu = a.page_cu; p.bg.page_idx = a.page_idx; p.bg.page_lg = p.page_lg; }
+    const int units = ctx->cfg.rope_layout == BA_ROPE_ADJACENT ? p.bg.row_vecs : p.bg.row_vecs / 2;
+    p.bg_rows_per_chunk = max(1, min(32, 1024 / max(units, 1)));
+    p.bg_direct = 1;
+    p.counters = counters;
   }
   if (D == 128) {
     auto kern = p.fused ? ba_attend_sm100_kernel<128, true> : ba_attend_sm100_kernel<128, false>;

@@ -35,7 +35,21 @@ struct ba_reencode_job {
   // the job reports BA_ERR_INVALID_ARG instead of rotating with a foreign table
   const int32_t *gen;
   int32_t gen_expected;
+  // non-null: the source is a paged pool -- block c owns pages page_idx[page_cu[c] .. page_cu[c+1]) of
+  // 1 << page_lg rows each (src_off is ignored)
+  const int32_t *page_cu, *page_idx;
+  int32_t page_lg;
 };
+
+// Source row of row `t` (0-based inside its block) of a job's block `c`; negative when the page number is bad.
+__device__ __forceinline__ long long ba_job_source_row(const ba_reencode_job &job, int c, int c_begin, int t) {
+  if (job.page_cu) {
+    const int page = __ldg(job.page_idx + __ldg(job.page_cu + c) + (t >> job.page_lg));
+    if (page < 0) return -1;
+    return ((long long)page << job.page_lg) + (t & ((1 << job.page_lg) - 1));
+  }
+  return (job.src_off ? (long long)__ldg(job.src_off + c) : (long long)c_begin) + t;
+}
 
 // Context: configuration, workspace and the device status word.
 struct ba_ctx {
@@ -116,6 +130,11 @@ struct ba_attend_args {
   int fused;
   const int32_t *k_src_off;
   int32_t n_k_rows;
+  void *k_out;     // fused warm path: non-null -> the re-encoded keys are also written here (cache packing)
+  // paged pool (page_rows > 0): the cached values -- and on the fused path the cached keys -- are read
+  // through a page table instead of v_src_off / k_src_off
+  int32_t page_rows;
+  const int32_t *page_cu, *page_idx;
   int final_only;  // 1: ba_final_attend, 0: ba_block_prefill
 };
 

@@ -63,6 +63,7 @@ ba_reencode_kernel(const ba_reencode_job job, int units_shift, int32_t *status) 
   st.c_begin = __ldg(job.cu + st.c);
   st.c_end = __ldg(job.cu + st.c + 1);
   st.shift = job.src_off ? (long long)__ldg(job.src_off + st.c) - st.c_begin : 0;
+  st.page0 = job.page_cu ? __ldg(job.page_cu + st.c) : 0;
 #pragma unroll 1
   for (int pass = 0; pass < kPasses && row0 < total_rows; ++pass, row0 += row_step * kRows)
     ba_reencode_rows<kLayout, kRows>(job, st, row0, row_step, total_rows, status);
@@ -90,6 +91,7 @@ ba_reencode_job ba_make_reencode_job(const ba_ctx *ctx, const void *k_src, const
   job.head_dim = ctx->cfg.head_dim; job.row_vecs = ctx->cfg.n_kv_heads * ctx->cfg.head_dim / 8;
   job.layout = ctx->cfg.rope_layout;
   job.gen = nullptr; job.gen_expected = 0;
+  job.page_cu = nullptr; job.page_idx = nullptr; job.page_lg = 0;
   return job;
 }
 

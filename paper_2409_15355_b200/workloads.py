@@ -224,3 +224,25 @@ def warm_inputs(w: Workload, layer: int = 0):
         src = [pool_off[i] for req in w.request_pool_idx for i in req]
         out["src_off"] = np.asarray(src, dtype=np.int32)
     return out
+
+
+def scatter_into_pages(packed: np.ndarray, cache_lens, page_rows: int, seed: int, spare_pages: int = 3):
+    """Lays packed cached rows [T_c, ...] (uint16 bf16 bits) out as a pool of fixed-size pages: every
+    cached block gets ceil(L / page_rows) pages, pages are numbered by a seeded permutation (with a few
+    spare pages in between), rows of a last page beyond the block's end are filled with N(0,1) noise.
+    Returns (pool [n_pages * page_rows, ...], page_cu int32 [n_blocks + 1], page_idx int32, n_pages)."""
+    rng = np.random.default_rng(seed)
+    counts = [(int(L) + page_rows - 1) // page_rows for L in cache_lens]
+    page_cu = np.concatenate([[0], np.cumsum(counts)]).astype(np.int32)
+    n_used = int(page_cu[-1])
+    n_pages = n_used + spare_pages
+    page_idx = rng.permutation(n_pages)[:n_used].astype(np.int32)
+    pool = normal_bf16(seed + 1, (n_pages * page_rows,) + tuple(packed.shape[1:]))
+    r = 0
+    for c, L in enumerate(cache_lens):
+        for k in range(counts[c]):
+            n = min(page_rows, int(L) - k * page_rows)
+            g = int(page_idx[page_cu[c] + k])
+            pool[g * page_rows:g * page_rows + n] = packed[r:r + n]
+            r += n
+    return pool, page_cu, page_idx, n_pages

@@ -444,6 +444,87 @@ def test_final_block_over_many_small_cached_blocks(fused):
     check_attention(o, o_ref, lse, lse_ref)
 
 
+def paged_case(w, page_rows, layer=0, layout=B.BA_ROPE_ADJACENT):
+    """The cached keys and values of workload `w` scattered over paged pools (one page table for both)."""
+    t = ob.segment_tables(w.block_lens, w.seq_nblocks)
+    x = W.warm_inputs(w, layer)
+    cache_lens = [l for lens in w.cached_lens_per_seq() for l in lens]
+    k_pool, page_cu, page_idx, n_pages = W.scatter_into_pages(x["k_cache"], cache_lens, page_rows, seed=w.seed + 5)
+    v_pool, _, _, _ = W.scatter_into_pages(x["v_cache"], cache_lens, page_rows, seed=w.seed + 5)
+    d_cu, d_idx = torch.from_numpy(page_cu).cuda(), torch.from_numpy(page_idx).cuda()
+    pages = B.make_page_table(page_rows, n_pages, d_cu, d_idx)
+    # the oracle reads the pools through the same table, by plain indexing
+    rows = ob.paged_rows(cache_lens, page_rows, page_cu, page_idx)
+    k64, v64 = W.bf16_bits_to_f64(k_pool[rows]), W.bf16_bits_to_f64(v_pool[rows])
+    k_ref = ob.reencode_blocks(k64, None, t["cache_cu"], t["cache_delta"], w.rope_theta, layout)
+    o_ref, lse_ref = ob.final_attend(W.bf16_bits_to_f64(x["q_f"]), W.bf16_bits_to_f64(x["k_f"]),
+                                     W.bf16_bits_to_f64(x["v_f"]), k_ref, v64, w.block_lens, w.seq_nblocks)
+    return t, x, dev(k_pool), dev(v_pool), pages, (d_cu, d_idx), k_ref, o_ref, lse_ref
+
+
+PAGED_CASES = [(W.config1(), 16), (W.config2(), 16), (W.config2(), 64), (W.config2(), 128), (W.config2(), 256),
+               (W.random_ragged(41, 3, 6, 300, 8, 2, 128), 32), (W.random_ragged(42, 5, 4, 200, 4, 2, 64), 16)]
+
+
+@pytest.mark.parametrize("w,page_rows", PAGED_CASES, ids=lambda v: v.name if hasattr(v, "name") else f"p{v}")
+def test_paged_cache_reencode_and_attend(w, page_rows):
+    """Section 2.5 step 1 with a paged cache: cached keys gathered through the page table and re-encoded
+    (ba_reencode_k_paged), values read from their pages in place by ba_final_attend_paged (one copy per
+    page, a key tile never spans two pages); then both steps in one launch on the paged keys
+    (ba_final_attend_fused_paged) with the re-encoded keys written back.  Pages are in a seeded order and
+    the unused rows of last pages hold noise."""
+    t, x, k_pool, v_pool, pages, keep, k_ref, o_ref, lse_ref = paged_case(w, page_rows)
+    Tc, Tf = t["n_cached_tokens"], t["n_final_tokens"]
+    c = ctx_for(w)
+    seg, buf = c.segment(w.block_lens, w.seq_nblocks, B.BA_MODE_BLOCK)
+    q_f, k_f, v_f = dev(x["q_f"]), dev(x["k_f"]), dev(x["v_f"])
+    o = torch.empty(Tf, w.n_q_heads, w.head_dim, dtype=torch.float32, device="cuda")
+    lse = torch.empty(Tf, w.n_q_heads, dtype=torch.float32, device="cuda")
+    if Tc > 0:
+        k_re = torch.zeros(Tc, w.n_kv_heads, w.head_dim, dtype=torch.bfloat16, device="cuda")
+        B.ba_reencode_k_paged(c.ctx, k_pool, pages, k_re, seg.cache_cu, seg.cache_delta, seg.n_cached_blocks, Tc)
+        assert c.device_status() == B.BA_OK
+        check_reencoded(R.device_to_bits(k_re), k_ref)
+        # the same bytes as the contiguous call on the packed keys
+        k_packed = torch.empty_like(k_re)
+        B.ba_reencode_k(c.ctx, dev(x["k_cache"]), None, Tc, k_packed, seg.cache_cu, seg.cache_delta,
+                        seg.n_cached_blocks, Tc)
+        assert torch.equal(k_re, k_packed)
+    else:
+        k_re = None
+    B.ba_final_attend_paged(c.ctx, q_f, k_f, v_f, Tf, k_re, Tc, v_pool, pages, o, lse, seg, B.BA_MODE_BLOCK, B.BA_OUT_F32)
+    assert c.device_status() == B.BA_OK
+    check_attention(o.cpu().numpy(), o_ref, lse.cpu().numpy(), lse_ref)
+    o2 = torch.empty_like(o)
+    k_out = torch.zeros_like(k_re) if Tc > 0 else None
+    B.ba_final_attend_fused_paged(c.ctx, q_f, k_f, v_f, Tf, k_pool, v_pool, pages, Tc, o2, lse, seg, B.BA_MODE_BLOCK,
+                                  B.BA_OUT_F32, k_out=k_out)
+    assert c.device_status() == B.BA_OK
+    check_attention(o2.cpu().numpy(), o_ref, lse.cpu().numpy(), lse_ref)
+    if Tc > 0:
+        assert torch.equal(k_out, k_re)
+    c.close()
+
+
+def test_paged_cache_bad_page_numbers_are_reported_and_bad_sizes_refused():
+    w = W.config1()
+    t, x, k_pool, v_pool, pages, (d_cu, d_idx), k_ref, o_ref, lse_ref = paged_case(w, 16)
+    c = ctx_for(w)
+    seg, buf = c.segment(w.block_lens, w.seq_nblocks, B.BA_MODE_BLOCK)
+    k_re = torch.zeros(256, 2, 64, dtype=torch.bfloat16, device="cuda")
+    bad_idx = d_idx.clone(); bad_idx[3] = 10 ** 6; bad_idx[5] = -2
+    bad = B.make_page_table(16, pages.n_pages, d_cu, bad_idx)
+    B.ba_reencode_k_paged(c.ctx, k_pool, bad, k_re, seg.cache_cu, seg.cache_delta, seg.n_cached_blocks, 256)
+    assert c.device_status() == B.BA_ERR_INVALID_ARG
+    assert not k_re[48:64].any() and not k_re[80:96].any()           # the rows of the bad pages were skipped
+    for rows in (8, 24, 1 << 17):
+        with pytest.raises(B.BaError) as e:
+            B.ba_reencode_k_paged(c.ctx, k_pool, B.make_page_table(rows, 4, d_cu, d_idx), k_re, seg.cache_cu,
+                                  seg.cache_delta, seg.n_cached_blocks, 256)
+        assert e.value.status == B.BA_ERR_UNSUPPORTED
+    c.close()
+
+
 def test_warm_path_32k_full_size():
     w = W.config3(1)
     o, lse, o_ref, lse_ref = run_warm(w, B.BA_MODE_BLOCK, B.BA_OUT_BF16)
@@ -464,6 +545,39 @@ def test_fused_warm_path_parity(w, mode):
 def test_fused_warm_path_half_layout(w):
     o, lse, o_ref, lse_ref = run_warm(w, B.BA_MODE_BLOCK, fused=True, layout=B.BA_ROPE_HALF)
     check_attention(o, o_ref, lse, lse_ref)
+
+
+@pytest.mark.parametrize("w,layout", [(W.config1(), B.BA_ROPE_ADJACENT), (W.config2(), B.BA_ROPE_HALF),
+                                      (W.config5(4, 64, 6, 32), B.BA_ROPE_ADJACENT), (W.config3(1), B.BA_ROPE_ADJACENT)],
+                         ids=["tiny", "rag_half", "pool", "32k"])
+def test_fused_call_writes_the_reencoded_keys_as_a_side_output(w, layout):
+    """Section 2.5 steps 2-3 in one launch, with the re-encoded keys -- what later decode steps read --
+    written back by the same launch: bit-identical to ba_reencode_k, a correct rounding of the oracle's
+    rotation, and the attention output unchanged by the side job."""
+    c, seg, buf, src, want, ref, t = reencode_case(w, layout=layout)      # `want`: ba_reencode_k
+    x = W.warm_inputs(w)
+    Tc, Tf = t["n_cached_tokens"], t["n_final_tokens"]
+    off = torch.from_numpy(x["src_off"]).cuda() if w.pool_lens is not None else None
+    v_src = dev(x["v_pool"] if w.pool_lens is not None else x["v_cache"])
+    q_f, k_f, v_f = dev(x["q_f"]), dev(x["k_f"]), dev(x["v_f"])
+    o_plain = torch.empty(Tf, w.n_q_heads, w.head_dim, dtype=torch.float32, device="cuda")
+    o_side = torch.empty_like(o_plain)
+    k_out = torch.zeros_like(want)
+    B.ba_final_attend_fused(c.ctx, q_f, k_f, v_f, Tf, src, v_src, src.shape[0], off, Tc, o_plain, None, seg,
+                            B.BA_MODE_BLOCK, B.BA_OUT_F32)
+    for _ in range(2):          # twice: the launch counters must be back at zero after the first launch
+        k_out.zero_()
+        B.ba_final_attend_fused(c.ctx, q_f, k_f, v_f, Tf, src, v_src, src.shape[0], off, Tc, o_side, None, seg,
+                                B.BA_MODE_BLOCK, B.BA_OUT_F32, k_out=k_out)
+        assert c.device_status() == B.BA_OK
+        assert torch.equal(k_out, want)
+        assert torch.equal(o_side, o_plain)
+    check_reencoded(R.device_to_bits(k_out), ref)
+    with pytest.raises(B.BaError) as e:          # in place: the attention reads the cached keys meanwhile
+        B.ba_final_attend_fused(c.ctx, q_f, k_f, v_f, Tf, src, v_src, src.shape[0], off, Tc, o_side, None, seg,
+                                B.BA_MODE_BLOCK, B.BA_OUT_F32, k_out=src)
+    assert e.value.status == B.BA_ERR_INVALID_ARG
+    c.close()
 
 
 def test_fused_warm_path_32k_full_size_and_pool_serving():

@@ -417,3 +417,27 @@ def test_pins_catch_planted_mistakes(monkeypatch):
     monkeypatch.setattr(ob, "segment_tables", bad_tables)
     assert _fails(test_warm_path_equals_prefill_with_direct_rope)
     assert _fails(test_tables_hand_example)
+
+
+def test_paged_rows_gather_reproduces_the_contiguous_cache():
+    """A paged pool is an indexing scheme only: gathering the rows the page table names gives back the
+    packed cache, whatever the page size and page order; checked against a hand-written table and
+    against per-row brute force."""
+    from paper_2409_15355_b200 import workloads as W
+    # hand-written: blocks of 5 and 3 rows, pages of 4 rows; block 0 -> pages 2, 0; block 1 -> page 3
+    rows = ob.paged_rows([5, 3], 4, [0, 2, 3], [2, 0, 3])
+    assert rows.tolist() == [8, 9, 10, 11, 0, 12, 13, 14]
+    lens = [37, 1, 16, 130, 64]
+    packed = W.normal_bf16(3, (sum(lens), 2, 8))
+    for page_rows in (16, 32, 128):
+        pool, page_cu, page_idx, n_pages = W.scatter_into_pages(packed, lens, page_rows, seed=9)
+        assert pool.shape[0] == n_pages * page_rows and len(set(page_idx.tolist())) == len(page_idx)
+        got = pool[ob.paged_rows(lens, page_rows, page_cu, page_idx)]
+        assert np.array_equal(got, packed)
+        # brute force, row by row
+        r = 0
+        for c, L in enumerate(lens):
+            for t in range(L):
+                g = page_idx[page_cu[c] + t // page_rows]
+                assert np.array_equal(pool[g * page_rows + t % page_rows], packed[r])
+                r += 1
