@@ -281,7 +281,7 @@ def run_ours(args):
     att_events = []
     re_events = []
 
-    def step_overlap(inputs, record=False):
+    def step_overlap(inputs, record=False, ready=None, done=None):
         seg = B.ba_segment(ctx.ctx, lens, nb, 1, len(lens), w.n_tokens, B.BA_MODE_BLOCK, tbuf)
         ev_seg = torch.cuda.Event(); ev_seg.record(stream)
         re_stream.wait_event(ev_seg)          # tables ready; the previous step no longer reads k_re
@@ -290,16 +290,20 @@ def run_ours(args):
             x = inputs[l]
             if l >= 2:
                 re_stream.wait_event(ev_att[l - 2])     # stay one layer ahead of the attention, not more
+            if ready is not None:
+                re_stream.wait_event(ready[l])          # this layer's inputs have arrived from the host
             B.ba_reencode_k(ctx.ctx, x["k_cache"], None, Tc, k_re[l], seg.cache_cu, seg.cache_delta,
                             seg.n_cached_blocks, Tc, stream=re_stream)
             e = torch.cuda.Event(); e.record(re_stream); ev_re.append(e)
             if l >= 1:
                 issue_attend(inputs, l - 1, seg, ev_re, ev_att, record)
         issue_attend(inputs, L - 1, seg, ev_re, ev_att, record)
+        if done is not None:
+            done.extend(ev_att)
 
     def issue_attend(inputs, l, seg, ev_re, ev_att, record):
         x = inputs[l]
-        stream.wait_event(ev_re[l])
+        stream.wait_event(ev_re[l])                     # (the re-encode stream waited for the layer's inputs)
         if record:
             e0 = torch.cuda.Event(enable_timing=True); e0.record(stream)
         B.ba_final_attend(ctx.ctx, x["q_f"], x["k_f"], x["v_f"], Tf, k_re[l], x["v_cache"], Tc, None, 0,
@@ -309,9 +313,11 @@ def run_ours(args):
         if record:
             att_events.append((e0, e1))
 
-    def step(inputs, record=False):
+    def step(inputs, record=False, ready=None, done=None):
         if args.overlap:
-            return step_overlap(inputs, record)
+            return step_overlap(inputs, record, ready, done)
+        if ready is not None:
+            stream.wait_event(ready[-1])                # single-stream order: all inputs first
         seg = B.ba_segment(ctx.ctx, lens, nb, 1, len(lens), w.n_tokens, B.BA_MODE_BLOCK, tbuf)
         # Layer l+1 is re-encoded before layer l attends (the cached keys of all layers are known up
         # front); with --deferred that re-encoding is queued and runs inside layer l's attention launch.
@@ -338,6 +344,8 @@ def run_ours(args):
             if record:
                 e1 = torch.cuda.Event(enable_timing=True); e1.record(stream)
                 att_events.append((e0, e1))
+            if done is not None:
+                e = torch.cuda.Event(); e.record(stream); done.append(e)
 
     def barrier():
         if world > 1:
@@ -387,13 +395,24 @@ def run_ours(args):
     d2h = sum(t.numel() * 2 for t in o_host)
     stage = [{k: torch.empty_like(d_in[l][k]) for k in names} for l in range(L)]
 
+    # copies run on streams of their own: layer l+1 arrives while layer l is worked on, results leave as
+    # soon as their layer is done (PCIe is full duplex); everything is inside the timed region
+    h2d_stream, d2h_stream = torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)
+
     def e2e_step():
-        for l in range(L):
-            for k in names:
-                stage[l][k].copy_(host[l][k], non_blocking=True)
-        step(stage)
-        for l in range(L):
-            o_host[l].copy_(o[l], non_blocking=True)
+        h2d_stream.wait_stream(stream)                  # the previous step has consumed the staging buffers
+        ready, done = [], []
+        with torch.cuda.stream(h2d_stream):
+            for l in range(L):
+                for k in names:
+                    stage[l][k].copy_(host[l][k], non_blocking=True)
+                e = torch.cuda.Event(); e.record(h2d_stream); ready.append(e)
+        step(stage, ready=ready, done=done)
+        with torch.cuda.stream(d2h_stream):
+            for l in range(L):
+                d2h_stream.wait_event(done[l])
+                o_host[l].copy_(o[l], non_blocking=True)
+        stream.wait_stream(d2h_stream)                  # the step ends when its last result is on the host
 
     e2e_step()
     barrier()
@@ -586,12 +605,15 @@ def main():
     ap.add_argument("--layers", type=int, default=32, help="layers per step (32 = the metric's workload)")
     ap.add_argument("--no-prefill", action="store_true", help="skip the secondary cold-prefill measurement")
     ap.add_argument("--no-fused", action="store_true", help="skip the secondary fused-warm-path measurement")
-    ap.add_argument("--overlap", action="store_true",
-                    help="re-encode layer l+1 on a second stream while layer l attends")
+    ap.add_argument("--no-overlap", dest="overlap", action="store_false",
+                    help="issue re-encode and attend of every layer on one stream (default: layer l+1 is "
+                         "re-encoded on a second stream while layer l attends)")
     ap.add_argument("--deferred", action="store_true",
                     help="queue each layer's re-encoding so that it runs in the background of the previous layer's "
                          "attention launch (ba_reencode_k_deferred) instead of as a stand-alone launch")
     args = ap.parse_args()
+    if args.deferred:
+        args.overlap = False
     if args.impl == "reference":
         return run_reference(args)
     return run_ours(args)

@@ -18,6 +18,8 @@ What is computed, and where the paper defines it:
 * RoPE re-encoding    -- Section 2.3, Eq. 1 (rotation to position i), Eq. 2
                          (inverse rotation, back to position zero), Eq. 3
                          (rotation to the new position).
+* backward pass       -- Section 2.4 (block fine-tune): gradients of that attention
+                         under the same mask, by the softmax Jacobian.
 * attention           -- plain softmax(Q K^T / sqrt(d)) V under that mask, with
                          grouped-query heads (query head h reads KV head
                          floor(h / G)).  The paper keeps the model's attention
@@ -350,6 +352,64 @@ def final_attend(q_f, k_f, v_f, k_cache_reencoded, v_cache, block_lens, seq_nblo
                                               k_all, v_all, m, scale)
         b0 += nb
     return o, lse
+
+
+# ---------------------------------------------------------------------------
+# Backward pass under the same mask (Section 2.4: block fine-tuning trains the model with
+# the Block-attention mask in place of the lower-triangular one, so gradients flow through
+# exactly the masked softmax attention defined above)
+# ---------------------------------------------------------------------------
+def attention_rows_backward(q_rows, k, v, mask, d_o, scale=None):
+    """Gradients of  L = sum(d_o * O)  for the rows computed by attention_rows.
+
+    With P the row-wise softmax of the masked scaled scores S (P = 0 where the mask forbids)
+    and O = P V:   dV = P^T dO;   dP = dO V^T;   dS = P * (dP - rowsum(P * dP))   (the softmax
+    Jacobian applied to dP);   dQ = scale * dS K;   dK = scale * dS^T Q.  Query head h reads KV
+    head floor(h / G), so dK and dV collect the contributions of the G heads of their group.
+    Returns dq [n, Hq, d] and dk, dv [T, Hkv, d] (the contributions of these rows only)."""
+    q_rows = np.asarray(q_rows, dtype=np.float64)
+    k = np.asarray(k, dtype=np.float64)
+    v = np.asarray(v, dtype=np.float64)
+    d_o = np.asarray(d_o, dtype=np.float64)
+    n, Hq, d = q_rows.shape
+    Hkv = k.shape[1]
+    G = Hq // Hkv
+    if scale is None:
+        scale = 1.0 / np.sqrt(np.float64(d))
+    dq = np.zeros_like(q_rows)
+    dk = np.zeros_like(k)
+    dv = np.zeros_like(v)
+    neg = np.where(mask, 0.0, -np.inf)
+    for h in range(Hq):
+        g = h // G
+        s = (q_rows[:, h, :] @ k[:, g, :].T) * scale + neg
+        p = np.exp(s - s.max(axis=1, keepdims=True))
+        p /= p.sum(axis=1, keepdims=True)
+        dv[:, g, :] += p.T @ d_o[:, h, :]
+        dp = d_o[:, h, :] @ v[:, g, :].T
+        ds = p * (dp - (p * dp).sum(axis=1, keepdims=True))
+        dq[:, h, :] = (ds @ k[:, g, :]) * scale
+        dk[:, g, :] += (ds.T @ q_rows[:, h, :]) * scale
+    return dq, dk, dv
+
+
+def block_prefill_backward(q, k, v, d_o, block_lens, seq_nblocks, mode, scale=None):
+    """dQ, dK, dV of block_prefill over the whole packed batch, sequence by sequence (keys of other
+    sequences are masked for every row, so they receive no gradient)."""
+    qf, kf, vf, gf = (np.asarray(x, dtype=np.float64) for x in (q, k, v, d_o))
+    dq, dk, dv = np.zeros_like(qf), np.zeros_like(kf), np.zeros_like(vf)
+    b0, row0 = 0, 0
+    for nb in seq_nblocks:
+        lens = [int(x) for x in block_lens[b0:b0 + nb]]
+        n = sum(lens)
+        rows = np.arange(n)
+        m = mask_rows(lens, [nb], mode, rows)
+        sl = slice(row0, row0 + n)
+        a, b, c = attention_rows_backward(qf[sl], kf[sl], vf[sl], m, gf[sl], scale)
+        dq[sl], dk[sl], dv[sl] = a, b, c
+        b0 += nb
+        row0 += n
+    return dq, dk, dv
 
 
 def allowed_pairs(block_lens, seq_nblocks, mode):

@@ -256,6 +256,34 @@ def test_prefill_parity(w, mode):
     check_attention(o, o_ref, lse, lse_ref)
 
 
+@pytest.mark.parametrize("mode", [B.BA_MODE_BLOCK, B.BA_MODE_FULL])
+def test_prefill_running_maximum_that_keeps_growing(mode):
+    """Keys whose magnitude grows along the sequence: the row maximum of the logits keeps rising from key
+    tile to key tile and inside tiles, by far more than the factor the kernel lets its reference maximum
+    lag behind, so every rescaling path of the online softmax runs many times."""
+    w = W.Workload("growing_logits", 8, 2, 128, 1e4, [700, 300, 45], [2, 1], seed=55)
+    qb, kb, vb = W.prefill_inputs(w)
+    ramp = (1.0 + 60.0 * np.arange(w.n_tokens) / w.n_tokens).astype(np.float32)
+    kb = W.f32_to_bf16_bits(W.bf16_bits_to_f32(kb) * ramp[:, None, None])
+    c = ctx_for(w)
+    seg, buf = c.segment(w.block_lens, w.seq_nblocks, mode)
+    o = torch.empty(w.n_tokens, w.n_q_heads, w.head_dim, device="cuda", dtype=torch.float32)
+    lse = torch.empty(w.n_tokens, w.n_q_heads, dtype=torch.float32, device="cuda")
+    B.ba_block_prefill(c.ctx, dev(qb), dev(kb), dev(vb), o, lse, seg, mode, B.BA_OUT_F32)
+    assert c.device_status() == B.BA_OK
+    o_ref, lse_ref = ob.block_prefill(W.bf16_bits_to_f64(qb), W.bf16_bits_to_f64(kb), W.bf16_bits_to_f64(vb),
+                                      w.block_lens, w.seq_nblocks, mode)
+    # logits reach the hundreds: the log-sum-exp is compared relative to its size, the outputs (convex
+    # combinations of N(0,1) values) under the usual bounds
+    og = o.cpu().numpy()
+    assert np.isfinite(og).all()
+    d = np.abs(og - o_ref)
+    assert d.max() <= 2e-2 and d.mean() <= 1e-3, (d.max(), d.mean())
+    assert np.linalg.norm(og - o_ref) / np.linalg.norm(o_ref) <= 5e-3
+    assert (np.abs(lse.cpu().numpy() - lse_ref) <= 2e-3 + 1e-5 * np.abs(lse_ref)).all()
+    c.close()
+
+
 def test_prefill_bf16_output():
     o, lse, o_ref, lse_ref = run_prefill(W.config2(), B.BA_MODE_BLOCK, B.BA_OUT_BF16)
     check_attention(o, o_ref, lse, lse_ref, bf16_store=True)

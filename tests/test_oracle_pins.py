@@ -441,3 +441,102 @@ def test_paged_rows_gather_reproduces_the_contiguous_cache():
                 g = page_idx[page_cu[c] + t // page_rows]
                 assert np.array_equal(pool[g * page_rows + t % page_rows], packed[r])
                 r += 1
+
+
+# --------------------------------------------------------------------------- backward pass
+def _tiny_backward_case(seed=0, lens=(3, 2, 2), nbs=(2, 1), Hq=4, Hkv=2, d=4):
+    rng = np.random.default_rng(seed)
+    T = sum(lens)
+    q, g = rng.standard_normal((T, Hq, d)), rng.standard_normal((T, Hq, d))
+    k, v = rng.standard_normal((T, Hkv, d)), rng.standard_normal((T, Hkv, d))
+    return list(lens), list(nbs), q, k, v, g
+
+
+@pytest.mark.parametrize("mode", [ob.MODE_BLOCK, ob.MODE_FULL])
+def test_backward_matches_central_finite_differences(mode):
+    """dQ, dK, dV against (L(x + e) - L(x - e)) / 2e of L = sum(dO * O), element by element, on a tiny
+    two-sequence layout with grouped heads: a dropped term, a wrong sign, a missing scale or a wrong
+    head-to-group map each change some entry by far more than the 1e-6 allowed."""
+    lens, nbs, q, k, v, g = _tiny_backward_case()
+    dq, dk, dv = ob.block_prefill_backward(q, k, v, g, lens, nbs, mode)
+    loss = lambda q_, k_, v_: float((ob.block_prefill(q_, k_, v_, lens, nbs, mode)[0] * g).sum())
+    eps = 1e-6
+    for name, x, dx in (("q", q, dq), ("k", k, dk), ("v", v, dv)):
+        num = np.zeros_like(x)
+        for idx in np.ndindex(*x.shape):
+            xp, xm = x.copy(), x.copy()
+            xp[idx] += eps; xm[idx] -= eps
+            args_p = {"q": (xp, k, v), "k": (q, xp, v), "v": (q, k, xp)}[name]
+            args_m = {"q": (xm, k, v), "k": (q, xm, v), "v": (q, k, xm)}[name]
+            num[idx] = (loss(*args_p) - loss(*args_m)) / (2 * eps)
+        assert np.abs(num - dx).max() <= 1e-6, (name, np.abs(num - dx).max())
+
+
+def test_backward_single_block_matches_library_autograd():
+    """One block is ordinary causal attention: gradients equal those torch's autograd gives for its
+    scaled-dot-product attention in fp64 (grouped heads expanded for the library call)."""
+    import torch
+    rng = np.random.default_rng(5)
+    L, Hq, Hkv, d = 9, 4, 2, 8
+    q, g = rng.standard_normal((L, Hq, d)), rng.standard_normal((L, Hq, d))
+    k, v = rng.standard_normal((L, Hkv, d)), rng.standard_normal((L, Hkv, d))
+    for mode in (ob.MODE_BLOCK, ob.MODE_FULL):
+        dq, dk, dv = ob.block_prefill_backward(q, k, v, g, [L], [1], mode)
+        tq = torch.tensor(q.transpose(1, 0, 2), requires_grad=True)
+        tk = torch.tensor(k.transpose(1, 0, 2), requires_grad=True)
+        tv = torch.tensor(v.transpose(1, 0, 2), requires_grad=True)
+        o = torch.nn.functional.scaled_dot_product_attention(tq, tk.repeat_interleave(Hq // Hkv, 0),
+                                                             tv.repeat_interleave(Hq // Hkv, 0), is_causal=True)
+        (o * torch.tensor(g.transpose(1, 0, 2))).sum().backward()
+        assert np.abs(tq.grad.numpy().transpose(1, 0, 2) - dq).max() <= 1e-10
+        assert np.abs(tk.grad.numpy().transpose(1, 0, 2) - dk).max() <= 1e-10
+        assert np.abs(tv.grad.numpy().transpose(1, 0, 2) - dv).max() <= 1e-10
+
+
+def test_backward_of_a_nonfinal_block_stays_inside_it():
+    """Rows of a non-final block see only their own block, so a loss on those rows alone gives no
+    gradient to keys and values outside the block (nor to other queries) and equals the gradient of
+    attention over that block taken alone; in full mode the same loss does reach the earlier blocks."""
+    lens, nbs, q, k, v, g = _tiny_backward_case(seed=3, lens=(4, 3, 5), nbs=(3,), Hq=2, Hkv=1, d=4)
+    gm = np.zeros_like(g); gm[4:7] = g[4:7]                       # block 1 (rows 4..6), non-final
+    dq, dk, dv = ob.block_prefill_backward(q, k, v, gm, lens, nbs, ob.MODE_BLOCK)
+    outside = np.r_[0:4, 7:12]
+    assert not dq[outside].any() and not dk[outside].any() and not dv[outside].any()
+    aq, ak, av = ob.block_prefill_backward(q[4:7], k[4:7], v[4:7], g[4:7], [3], [1], ob.MODE_BLOCK)
+    assert np.abs(dq[4:7] - aq).max() <= 1e-14 and np.abs(dk[4:7] - ak).max() <= 1e-14 and np.abs(dv[4:7] - av).max() <= 1e-14
+    fq, fk, fv = ob.block_prefill_backward(q, k, v, gm, lens, nbs, ob.MODE_FULL)
+    assert fk[0:4].any() and fv[0:4].any()
+    # a loss on the final block reaches every earlier block in both modes
+    gf = np.zeros_like(g); gf[7:] = g[7:]
+    _, dk2, dv2 = ob.block_prefill_backward(q, k, v, gf, lens, nbs, ob.MODE_BLOCK)
+    assert dk2[0:4].any() and dv2[4:7].any()
+
+
+def test_backward_pins_catch_planted_mistakes(monkeypatch):
+    good = ob.attention_rows_backward
+
+    def no_jacobian_term(q_rows, k, v, mask, d_o, scale=None):     # dS = P * dP: the row term of the softmax Jacobian dropped
+        n, Hq, d = q_rows.shape
+        G = Hq // k.shape[1]
+        sc = 1.0 / np.sqrt(d) if scale is None else scale
+        dq, dk, dv = np.zeros_like(q_rows), np.zeros_like(k), np.zeros_like(v)
+        for h in range(Hq):
+            g = h // G
+            s = (q_rows[:, h] @ k[:, g].T) * sc + np.where(mask, 0.0, -np.inf)
+            p = np.exp(s - s.max(axis=1, keepdims=True)); p /= p.sum(axis=1, keepdims=True)
+            dv[:, g] += p.T @ d_o[:, h]
+            ds = p * (d_o[:, h] @ v[:, g].T)
+            dq[:, h] = (ds @ k[:, g]) * sc
+            dk[:, g] += (ds.T @ q_rows[:, h]) * sc
+        return dq, dk, dv
+    monkeypatch.setattr(ob, "attention_rows_backward", no_jacobian_term)
+    assert _fails(test_backward_matches_central_finite_differences, ob.MODE_BLOCK)
+    monkeypatch.setattr(ob, "attention_rows_backward", lambda q, k, v, m, g, scale=None: good(q, k, v, m, g, 1.0))
+    assert _fails(test_backward_matches_central_finite_differences, ob.MODE_BLOCK)
+    assert _fails(test_backward_single_block_matches_library_autograd)
+
+    def swapped_groups(q_rows, k, v, mask, d_o, scale=None):
+        dq, dk, dv = good(q_rows, k, v, mask, d_o, scale)
+        return dq, dk[:, ::-1], dv
+    monkeypatch.setattr(ob, "attention_rows_backward", swapped_groups)
+    assert _fails(test_backward_matches_central_finite_differences, ob.MODE_FULL)
