@@ -114,6 +114,7 @@ typedef struct {
   int32_t *cu_qtile;       /* [B+1] */
   int32_t *cu_ftile;       /* [batch+1] */
   int32_t *cache_tile_cu;  /* [Bc+1] prefix sum of 128-key tiles per cached block (a tile never spans two blocks) */
+  int32_t *cu_ktile;       /* [B+1] prefix sum of 128-key tiles per block, every block (backward pass) */
   int32_t *totals;         /* [8]: cached tokens, final tokens, q tiles, final tiles, ..., [7] = validity word */
   /* rotation of every cached block, used by ba_final_attend_fused: (cos, sin)(cache_delta[c] * theta_m),
    * fp32 from fp64 angles, [Bc][head_dim / 2][2] */
@@ -292,8 +293,9 @@ ba_status ba_final_attend(ba_ctx *ctx, const void *q_f, const void *k_f, const v
  * rewritten nor read twice.  The result equals ba_reencode_k followed by ba_final_attend up to
  * the rounding of the rotated operand to bf16 (queries here, keys there).  The re-encoded keys
  * themselves -- what the rest of generation reads -- are written as a side output when k_out is
- * given: otherwise idle warps of the same launch rotate the cached keys from k_src to k_out
- * (bit-identical to ba_reencode_k) while the attention runs; they are complete when the call is.
+ * given: the call then also runs the re-encoding kernel, on a stream of the context's own beside the
+ * attention launch (which leaves SMs idle in its last wave), and joins it back into `stream`; k_out is
+ * bit-identical to ba_reencode_k's output and complete, in stream order, when the call is.
  *   q_f, k_f, v_f   as for ba_final_attend
  *   k_src, v_src    bf16 [n_src_rows, n_kv_heads, head_dim]: cached block c (cache order, as in
  *                   seg->cache_cu) occupies rows src_off[c] .. src_off[c] + length - 1 of both, or
@@ -308,6 +310,24 @@ ba_status ba_final_attend_fused(ba_ctx *ctx, const void *q_f, const void *k_f, c
                                 int32_t n_src_rows, const int32_t *src_off, int32_t n_cache_rows,
                                 void *k_out, void *o, float *lse, const ba_segments *seg, ba_mode mode,
                                 ba_out_dtype out_dtype, void *stream);
+
+/*
+ * Section 2.4 (block fine-tune): backward pass of ba_block_prefill.  Block fine-tuning trains the
+ * model with the Block-attention mask in place of the lower-triangular one, so the gradients flow
+ * through the same masked softmax: with P = softmax(scale Q K^T + mask), O = P V,
+ *     dV = P^T dO,   dS = P * (dO V^T - rowsum(dO * O)),   dQ = scale dS K,   dK = scale dS^T Q,
+ * dK and dV summed over the query heads that share a KV head.  P is recomputed from `lse`.
+ *   q, k, v, seg, mode   exactly what the forward call was given
+ *   o                    bf16 [T, n_q_heads, head_dim]: the forward output (BA_OUT_BF16)
+ *   lse                  fp32 [T, n_q_heads]: the forward call's log-sum-exp (required)
+ *   d_o                  bf16 [T, n_q_heads, head_dim]: gradient of the loss with respect to o
+ *   dq                   [T, n_q_heads, head_dim];  dk, dv  [T, n_kv_heads, head_dim]; bf16 or fp32
+ * Uses T * n_q_heads * 4 bytes of workspace (BA_ERR_WORKSPACE when the context has less).  No
+ * atomics: results are run-to-run identical.
+ */
+ba_status ba_block_prefill_bwd(ba_ctx *ctx, const void *q, const void *k, const void *v, const void *o,
+                               const float *lse, const void *d_o, void *dq, void *dk, void *dv,
+                               const ba_segments *seg, ba_mode mode, ba_out_dtype grad_dtype, void *stream);
 
 /*
  * Paged KV pool (Section 2.3: what the cache holds; Section 2.5 step 1: the cache look-up).  A serving

@@ -25,6 +25,7 @@ EXPORTS = [
     "ba_launch_count", "ba_segments_bytes", "ba_segment", "ba_reencode_k", "ba_block_prefill",
     "ba_final_attend", "ba_reencode_k_noalloc", "ba_selftest_wait_expiry", "ba_reencode_k_deferred", "ba_flush",
     "ba_final_attend_fused", "ba_reencode_k_paged", "ba_final_attend_paged", "ba_final_attend_fused_paged",
+    "ba_block_prefill_bwd",
 ]
 BA_NOALLOC_MAX_BLOCKS = 4096
 
@@ -43,7 +44,7 @@ class ba_segments(C.Structure):
             "cu_seq", "cu_cache_seq", "cu_final_seq", "cu_seq_block", "cu_block", "block_delta",
             "block_seq", "block_kv_begin", "block_part_off", "block_is_final", "cache_block",
             "cache_cu", "cache_delta", "tok_block", "tok_pos", "tok_pos_local", "cu_qtile",
-            "cu_ftile", "cache_tile_cu", "totals", "cache_rope")]
+            "cu_ftile", "cache_tile_cu", "cu_ktile", "totals", "cache_rope")]
 
 
 class ba_page_table(C.Structure):
@@ -101,6 +102,7 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
                                           C.POINTER(ba_segments), C.c_int, C.c_int, vp]
     lib.ba_final_attend_fused_paged.argtypes = [vp, vp, vp, vp, i32, vp, vp, pt, i32, vp, vp, vp,
                                                 C.POINTER(ba_segments), C.c_int, C.c_int, vp]
+    lib.ba_block_prefill_bwd.argtypes = [vp] + [vp] * 9 + [C.POINTER(ba_segments), C.c_int, C.c_int, vp]
     for name in EXPORTS:
         # without argtypes ctypes would pass addresses as 32-bit ints
         if getattr(lib, name).argtypes is None:
@@ -255,3 +257,9 @@ def ba_final_attend_fused_paged(ctx, q_f, k_f, v_f, n_final_rows, k_pool, v_pool
                                                       _ptr(k_pool), _ptr(v_pool), C.byref(pages), n_cache_rows,
                                                       _ptr(k_out), _ptr(o), _ptr(lse), C.byref(seg), mode, out_dtype,
                                                       _stream_ptr(stream)), "ba_final_attend_fused_paged")
+
+
+def ba_block_prefill_bwd(ctx, q, k, v, o, lse, d_o, dq, dk, dv, seg, mode, grad_dtype, stream=None):
+    _check(load_library().ba_block_prefill_bwd(ctx, _ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(lse), _ptr(d_o),
+                                               _ptr(dq), _ptr(dk), _ptr(dv), C.byref(seg), mode, grad_dtype,
+                                               _stream_ptr(stream)), "ba_block_prefill_bwd")

@@ -8,6 +8,9 @@
 ba_status ba_attend_sm100_launch(ba_ctx *ctx, const ba_attend_args &a, const ba_segments *seg,
                                  cudaStream_t stream);
 ba_status ba_attend_sm100_setup(ba_ctx *ctx);
+ba_status ba_bwd_sm100_launch(ba_ctx *ctx, const void *q, const void *k, const void *v, const void *o,
+                              const float *lse, const void *d_o, void *dq, void *dk, void *dv, int out_f32,
+                              const ba_segments *seg, int mode, cudaStream_t stream);
 void ba_attend_sm100_teardown(ba_ctx *ctx);
 int ba_heads_per_tile(const ba_config &c);
 
@@ -62,6 +65,7 @@ TableLayout table_layout(int32_t batch, int32_t B, int32_t T) {
   take((size_t)(B + 1) * 4);                                  // cu_qtile
   take((size_t)(batch + 1) * 4);                              // cu_ftile
   take((size_t)(B + 1) * 4);                                  // cache_tile_cu
+  take((size_t)(B + 1) * 4);                                  // cu_ktile
   take(8 * 4);                                                // totals
   take((size_t)B * 64 * 8);                                   // cache_rope: at most 64 rotary pairs per block
   L.bytes = cur;
@@ -128,6 +132,7 @@ ba_status ba_create(ba_ctx **out, const ba_config *cfg, int device, size_t works
   ctx->seg_delta = nullptr; ctx->seg_rope = nullptr; ctx->seg_rope_blocks = 0;
   ctx->seg_gen = nullptr; ctx->seg_gen_value = 0; ctx->seg_counter = 0;
   ctx->maps = nullptr;
+  ctx->side_stream = nullptr; ctx->ev_fork = nullptr; ctx->ev_join = nullptr;
   ctx->workspace = nullptr;
   ctx->dev_status = nullptr;
   if (cudaMalloc(&ctx->dev_status, 256) != cudaSuccess ||
@@ -136,8 +141,14 @@ ba_status ba_create(ba_ctx **out, const ba_config *cfg, int device, size_t works
       // launch counters of the attention kernels (below the scratch area): zero once, every launch leaves them zero
       (workspace_bytes >= ba_scratch_offset(ctx) &&
        cudaMemset((char *)ctx->workspace + ba_scratch_offset(ctx) - 256, 0, 256) != cudaSuccess) ||
+      cudaStreamCreateWithFlags(&ctx->side_stream, cudaStreamNonBlocking) != cudaSuccess ||
+      cudaEventCreateWithFlags(&ctx->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
+      cudaEventCreateWithFlags(&ctx->ev_join, cudaEventDisableTiming) != cudaSuccess ||
       ba_attend_sm100_setup(ctx) != BA_OK) {
     cudaGetLastError();
+    if (ctx->ev_join) cudaEventDestroy(ctx->ev_join);
+    if (ctx->ev_fork) cudaEventDestroy(ctx->ev_fork);
+    if (ctx->side_stream) cudaStreamDestroy(ctx->side_stream);
     if (ctx->workspace) cudaFree(ctx->workspace);
     if (ctx->dev_status) cudaFree(ctx->dev_status);
     delete ctx;
@@ -152,6 +163,9 @@ ba_status ba_destroy(ba_ctx *ctx) {
   cudaSetDevice(ctx->device);
   if (ctx->has_pending) ba_flush_pending(ctx, ctx->pending_stream);   // a queued job is not dropped
   cudaDeviceSynchronize();
+  if (ctx->ev_join) cudaEventDestroy(ctx->ev_join);
+  if (ctx->ev_fork) cudaEventDestroy(ctx->ev_fork);
+  if (ctx->side_stream) cudaStreamDestroy(ctx->side_stream);
   if (ctx->workspace) cudaFree(ctx->workspace);
   if (ctx->dev_status) cudaFree(ctx->dev_status);
   ba_attend_sm100_teardown(ctx);
@@ -230,7 +244,8 @@ ba_status ba_segment(ba_ctx *ctx, const int32_t *block_lens, const int32_t *seq_
   out->block_is_final = (uint8_t *)next();
   out->cache_block = next(); out->cache_cu = next(); out->cache_delta = next();
   out->tok_block = next(); out->tok_pos = next(); out->tok_pos_local = next();
-  out->cu_qtile = next(); out->cu_ftile = next(); out->cache_tile_cu = next(); out->totals = next();
+  out->cu_qtile = next(); out->cu_ftile = next(); out->cache_tile_cu = next(); out->cu_ktile = next();
+  out->totals = next();
   out->cache_rope = (float *)next();
   ctx->seg_delta = nullptr; ctx->seg_rope = nullptr; ctx->seg_rope_blocks = 0; ctx->seg_gen = nullptr;
   // Every call stamps its tables (totals[6]) with a value that differs from call to call and from
@@ -413,6 +428,20 @@ ba_status ba_final_attend_fused(ba_ctx *ctx, const void *q_f, const void *k_f, c
   return ba_attend_launch(ctx, a, seg, (cudaStream_t)stream);
 }
 
+
+ba_status ba_block_prefill_bwd(ba_ctx *ctx, const void *q, const void *k, const void *v, const void *o,
+                               const float *lse, const void *d_o, void *dq, void *dk, void *dv,
+                               const ba_segments *seg, ba_mode mode, ba_out_dtype grad_dtype, void *stream) {
+  ba_status st = check_attend_common(ctx, q, k, v, dq, seg, mode, grad_dtype);
+  if (st != BA_OK) return st;
+  if (!o || !lse || !d_o || !dk || !dv) return BA_ERR_INVALID_ARG;
+  if (!aligned16(o) || !aligned16(d_o) || !aligned16(dk) || !aligned16(dv)) return BA_ERR_INVALID_ARG;
+  BA_CUDA_TRY(cudaSetDevice(ctx->device));
+  st = ba_flush_pending(ctx, (cudaStream_t)stream);      // a queued re-encoding job does not ride along here
+  if (st != BA_OK) return st;
+  return ba_bwd_sm100_launch(ctx, q, k, v, o, lse, d_o, dq, dk, dv, grad_dtype == BA_OUT_F32, seg, (int)mode,
+                             (cudaStream_t)stream);
+}
 
 static ba_status check_pages(const ba_page_table *pg) {
   if (!pg || !pg->page_cu || !pg->page_idx) return BA_ERR_INVALID_ARG;

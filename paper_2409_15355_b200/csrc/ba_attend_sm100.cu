@@ -91,7 +91,6 @@ struct AttnParams {
   int32_t *counters;
   ba_reencode_job bg;             // bg.n_rows > 0: a re-encoding job the two spare warps carry out meanwhile
   int bg_rows_per_chunk;
-  int bg_direct;                  // the job moves its rows global -> global (no staging in shared memory)
   ba_segments seg;
   const int32_t *k_src_off;       // non-null: keys of cached block c start at pool row k_src_off[c] (fused path only)
   int walk;                       // cached keys are walked block by block (a tile never spans two blocks)
@@ -619,14 +618,9 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
   } else if (warp >= 10) {
     // ------------------------------------------------------------ spare warps: background re-encoding
     asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kSpareRegs));
-    if (p.bg.n_rows > 0 && p.bg_direct) {
-      // chunks are drawn from a device-wide counter, so the job spreads over every CTA of the launch
-      if (p.bg.layout == BA_ROPE_ADJACENT)
-        ba_reencode_direct<BA_ROPE_ADJACENT, 4>(p.bg, p.counters + 1, p.bg_rows_per_chunk, p.status);
-      else
-        ba_reencode_direct<BA_ROPE_HALF, 2>(p.bg, p.counters + 1, p.bg_rows_per_chunk, p.status);
-    } else if (p.bg.n_rows > 0) {
-      // each spare warp runs the staged engine with its own two 16 KB stages
+    if (p.bg.n_rows > 0) {
+      // each spare warp runs the staged engine with its own two 16 KB stages; chunks are drawn from a
+      // device-wide counter, so the job spreads over every CTA of the launch, early and late ones
       const int bw = warp - 10;
       ba_bg_smem *bsm = reinterpret_cast<ba_bg_smem *>(smem + L::kCtrl + 1024) + bw;
       if ((tid & 31) == 0) { mbar_init(&bsm->bar[0], 1); mbar_init(&bsm->bar[1], 1); fence_barrier_init(); }
@@ -1144,12 +1138,12 @@ ba_status ba_attend_sm100_launch(ba_ctx *ctx, const ba_attend_args &a, const ba_
   }
   p.n_splits = n_splits;
   p.n_chunks = Hq / p.hpt;
-  // Many more entries than SMs (cold prefill): persistent CTAs, one per SM, draw entries from a
-  // counter, which hides each item's start-up and write-out behind its neighbours.  A list of at
-  // most two entries per SM (final block over a long cache) gains nothing from that and is
-  // launched one CTA per entry.
+  // More entries than SMs: persistent CTAs, one per SM, draw entries from a counter, which hides each
+  // entry's start-up and write-out behind its neighbours (cold prefill: many entries per SM; final block
+  // over a long cache: about two, the write-out of a CTA's first entry overlaps the start of its second).
+  // Shorter lists are launched one CTA per entry.
   const long long work_upper = (long long)pairs_upper * (Hq / p.hpt) * n_splits;
-  p.persistent = items * n_splits > 2LL * ctx->sm_count;
+  p.persistent = items * n_splits > (a.final_only ? 1LL : 2LL) * ctx->sm_count;
   // the counters live in the last 256 bytes below the scratch area: zeroed by ba_create, left at zero by every launch
   int32_t *counters = nullptr;
   if (ctx->workspace && ctx->workspace_bytes >= ba_scratch_offset(ctx))
@@ -1184,7 +1178,7 @@ ba_status ba_attend_sm100_launch(ba_ctx *ctx, const ba_attend_args &a, const ba_
   dim3 grid((unsigned)(p.persistent ? ctx->sm_count : work_upper));
   // a queued re-encoding job rides along in the spare warps; a job whose rows do not fit the
   // staging buffers is run on its own first
-  p.bg.n_rows = 0; p.bg_rows_per_chunk = 0; p.bg_direct = 0;
+  p.bg.n_rows = 0; p.bg_rows_per_chunk = 0;
   if (ctx->has_pending) {
     const int row_bytes = ctx->pending.row_vecs * 16;
     if (row_bytes <= kBgStageBytes && !p.fused && counters) {   // (the fused path has other uses for the spare warps' staging area)
@@ -1198,16 +1192,22 @@ ba_status ba_attend_sm100_launch(ba_ctx *ctx, const ba_attend_args &a, const ba_
       if (fs != BA_OK) return fs;
     }
   }
-  if (p.fused && a.k_out) {
-    // side output of the fused call: the re-encoded keys, written by the spare warps from global to global
-    if (!counters) return BA_ERR_WORKSPACE;
-    p.bg = ba_make_reencode_job(ctx, a.k_cache, a.k_src_off, a.n_k_rows, a.k_out, seg->cache_cu, seg->cache_delta,
-                                seg->n_cached_blocks, a.n_cache_rows, reinterpret_cast<const float2 *>(seg->cache_rope));
-    if (p.k_paged) { p.bg.src_off = nullptr; p.bg.page_cu = a.page_cu; p.bg.page_idx = a.page_idx; p.bg.page_lg = p.page_lg; }
-    const int units = ctx->cfg.rope_layout == BA_ROPE_ADJACENT ? p.bg.row_vecs : p.bg.row_vecs / 2;
-    p.bg_rows_per_chunk = max(1, min(32, 1024 / max(units, 1)));
-    p.bg_direct = 1;
-    p.counters = counters;
+  // Side output of the fused call: the re-encoded keys, written by the stand-alone re-encoding kernel on the
+  // context's side stream beside the attention launch (which cannot share an SM with anything and leaves
+  // some SMs idle in its last wave); the caller's stream continues only when both are done.  (Measured
+  // alternative: the spare warps of the attention CTAs moving the rows cost 50 us per layer at 32K context,
+  // more than the kernel alone takes.)
+  const bool side_job = p.fused && a.k_out;
+  if (side_job) {
+    ba_reencode_job job = ba_make_reencode_job(ctx, a.k_cache, a.k_src_off, a.n_k_rows, a.k_out, seg->cache_cu,
+                                               seg->cache_delta, seg->n_cached_blocks, a.n_cache_rows,
+                                               reinterpret_cast<const float2 *>(seg->cache_rope));
+    if (p.k_paged) { job.src_off = nullptr; job.page_cu = a.page_cu; job.page_idx = a.page_idx; job.page_lg = p.page_lg; }
+    BA_CUDA_TRY(cudaEventRecord(ctx->ev_fork, stream));
+    BA_CUDA_TRY(cudaStreamWaitEvent(ctx->side_stream, ctx->ev_fork, 0));
+    ba_status rs = ba_reencode_main_launch(ctx, job, ctx->side_stream);
+    if (rs != BA_OK) return rs;
+    BA_CUDA_TRY(cudaEventRecord(ctx->ev_join, ctx->side_stream));
   }
   if (D == 128) {
     auto kern = p.fused ? ba_attend_sm100_kernel<128, true> : ba_attend_sm100_kernel<128, false>;
@@ -1218,6 +1218,7 @@ ba_status ba_attend_sm100_launch(ba_ctx *ctx, const ba_attend_args &a, const ba_
   }
   BA_CUDA_TRY(cudaGetLastError());
   ctx->launches += 1;
+  if (side_job) BA_CUDA_TRY(cudaStreamWaitEvent(stream, ctx->ev_join, 0));
   if (n_splits > 1) {
     const int n_rh = a.n_q_rows * Hq;
     const long long threads = (long long)n_rh * (D / 4);

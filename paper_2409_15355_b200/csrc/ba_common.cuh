@@ -77,6 +77,9 @@ struct ba_ctx {
   int32_t seg_counter;      // ba_segment calls so far on this context
   // tensor maps of recently used tensors (attention launches re-use a handful of buffers)
   struct ba_map_cache *maps;
+  // side stream of the fused call's key write-back (forked from and joined to the caller's stream by events)
+  cudaStream_t side_stream;
+  cudaEvent_t ev_fork, ev_join;
 };
 
 static inline size_t ba_align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }

@@ -202,6 +202,7 @@ extern "C" ba_status ba_reencode_k_noalloc(const ba_config *cfg, int device, con
   tmp.pending_stream = nullptr;
   tmp.seg_delta = nullptr; tmp.seg_rope = nullptr; tmp.seg_rope_blocks = 0;
   tmp.seg_gen = nullptr; tmp.seg_gen_value = 0; tmp.seg_counter = 0; tmp.maps = nullptr;
+  tmp.side_stream = nullptr; tmp.ev_fork = nullptr; tmp.ev_join = nullptr;
   return ba_reencode_launch(&tmp, k_src, src_off, n_src_rows, k_dst, cu, delta, n_blocks, n_rows,
                             g_noalloc_table[device], (cudaStream_t)stream);
 }

@@ -290,107 +290,3 @@ __device__ __forceinline__ void ba_reencode_background(const ba_reencode_job &jo
   }
 }
 
-// ---------------------------------------------------------------------------------------------
-// The same work-sharing scheme without staging, for warps of a kernel that has no shared memory
-// to spare: a warp draws a chunk of up to 32 rows, lane i resolves row i (block, source row,
-// delta) and hands it to whichever lane needs it by register shuffle; every lane then moves
-// 16-byte units of the chunk straight from global memory to global memory, kUnroll loads in
-// flight.  The arithmetic is the one of the stand-alone kernel (rot2, one rounding), so the bytes
-// written are identical.
-// ---------------------------------------------------------------------------------------------
-template <int kLayout, int kUnroll>
-__device__ __forceinline__ void ba_reencode_direct(const ba_reencode_job &job, int32_t *chunk_counter,
-                                                   int rows_per_chunk, int32_t *status) {
-  const int lane = threadIdx.x & 31;
-  const int row_vecs = job.row_vecs, half_dim = job.head_dim >> 1, head_vecs = job.head_dim >> 3;
-  const int total_rows = min(job.n_rows, __ldg(job.cu + job.n_blocks));
-  const int n_chunks = (total_rows + rows_per_chunk - 1) / rows_per_chunk;
-  const int units_per_row = (kLayout == BA_ROPE_ADJACENT) ? row_vecs : (row_vecs >> 1);
-  if (job.gen && __ldg(job.gen) != job.gen_expected) {     // the rotation table is not the one this job was given
-    if (lane == 0) ba_record_status(status, BA_ERR_INVALID_ARG);
-    return;
-  }
-  for (;;) {
-    int chunk = 0;
-    if (lane == 0) chunk = atomicAdd(chunk_counter, 1);
-    chunk = __shfl_sync(0xffffffffu, chunk, 0);
-    if (chunk >= n_chunks) break;
-    const int r_mine = chunk * rows_per_chunk + lane;
-    int c_mine = -1, d_mine = 0;
-    long long sr_mine = -1;
-    if (lane < rows_per_chunk && r_mine < total_rows) {
-      int c = upper_bound_i32(job.cu, job.n_blocks + 1, r_mine) - 1;
-      c = min(max(c, 0), job.n_blocks - 1);
-      const int c_begin = __ldg(job.cu + c);
-      sr_mine = ba_job_source_row(job, c, c_begin, r_mine - c_begin);
-      if (sr_mine < 0 || sr_mine >= job.n_src_rows) { ba_record_status(status, BA_ERR_INVALID_ARG); sr_mine = -1; }
-      else { c_mine = c; d_mine = __ldg(job.delta + c); }
-    }
-    const int rows_here = min(rows_per_chunk, total_rows - chunk * rows_per_chunk);
-    const int n_units = rows_here * units_per_row;
-    for (int base = 0; base < n_units; base += 32 * kUnroll) {
-      uint4 x[kUnroll], y[kUnroll];
-      int cb[kUnroll], dl[kUnroll], un[kUnroll], rw[kUnroll];
-#pragma unroll
-      for (int k = 0; k < kUnroll; ++k) {
-        const int idx = base + k * 32 + lane;
-        const int i = min(idx, n_units - 1) / units_per_row;          // every lane takes part in the shuffles
-        un[k] = idx - i * units_per_row;
-        rw[k] = chunk * rows_per_chunk + i;
-        cb[k] = __shfl_sync(0xffffffffu, c_mine, i);
-        dl[k] = __shfl_sync(0xffffffffu, d_mine, i);
-        const long long sr = __shfl_sync(0xffffffffu, sr_mine, i);
-        if (idx >= n_units) cb[k] = -1;
-        if (cb[k] >= 0) {
-          const uint4 *row = job.src + sr * row_vecs;
-          if (kLayout == BA_ROPE_ADJACENT) {
-            x[k] = __ldcs(row + un[k]);
-          } else {
-            const int hv = head_vecs >> 1, head = un[k] / hv, v = un[k] - head * hv;
-            x[k] = __ldcs(row + head * head_vecs + v);
-            y[k] = __ldcs(row + head * head_vecs + v + hv);
-          }
-        }
-      }
-#pragma unroll
-      for (int k = 0; k < kUnroll; ++k) {
-        if (cb[k] < 0) continue;
-        uint4 *q = job.dst + (size_t)rw[k] * row_vecs;
-        if (kLayout == BA_ROPE_ADJACENT) {
-          const int u = un[k];
-          if (dl[k] == 0) { q[u] = x[k]; continue; }
-          const float4 *t4 = reinterpret_cast<const float4 *>(job.table + cb[k] * half_dim + (u % head_vecs) * 4);
-          const float4 a = __ldg(t4), b = __ldg(t4 + 1);
-          const uint32_t w[4] = {x[k].x, x[k].y, x[k].z, x[k].w};
-          const float2 cs[4] = {make_float2(a.x, a.y), make_float2(a.z, a.w), make_float2(b.x, b.y), make_float2(b.z, b.w)};
-          uint32_t o[4];
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            float xo, yo;
-            rot2(bf16_lo(w[j]), bf16_hi(w[j]), cs[j], xo, yo);
-            o[j] = pack_bf16x2(xo, yo);
-          }
-          q[u] = make_uint4(o[0], o[1], o[2], o[3]);
-        } else {
-          const int hv = head_vecs >> 1, head = un[k] / hv, v = un[k] - head * hv;
-          const int vec_x = head * head_vecs + v, vec_y = vec_x + hv;
-          if (dl[k] == 0) { q[vec_x] = x[k]; q[vec_y] = y[k]; continue; }
-          const float4 *t4 = reinterpret_cast<const float4 *>(job.table + cb[k] * half_dim + v * 8);
-          const uint32_t wx[4] = {x[k].x, x[k].y, x[k].z, x[k].w}, wy[4] = {y[k].x, y[k].y, y[k].z, y[k].w};
-          uint32_t ox[4], oy[4];
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            const float4 cs = __ldg(t4 + j);
-            float x0, y0, x1, y1;
-            rot2(bf16_lo(wx[j]), bf16_lo(wy[j]), make_float2(cs.x, cs.y), x0, y0);
-            rot2(bf16_hi(wx[j]), bf16_hi(wy[j]), make_float2(cs.z, cs.w), x1, y1);
-            ox[j] = pack_bf16x2(x0, x1);
-            oy[j] = pack_bf16x2(y0, y1);
-          }
-          q[vec_x] = make_uint4(ox[0], ox[1], ox[2], ox[3]);
-          q[vec_y] = make_uint4(oy[0], oy[1], oy[2], oy[3]);
-        }
-      }
-    }
-  }
-}

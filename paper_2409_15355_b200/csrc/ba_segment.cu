@@ -81,7 +81,7 @@ ba_segment_blocks_kernel(const int32_t *__restrict__ lens, const int32_t *__rest
   }
 
   // --- per-block prefix sums: rows (prompt, cache, final packing) and query tiles
-  int c_all = 0, c_cache = 0, c_final = 0, c_tile = 0, c_ktile = 0;
+  int c_all = 0, c_cache = 0, c_final = 0, c_tile = 0, c_ktile = 0, c_atile = 0;
   for (int base = 0; base < B; base += kScanThreads) {
     int b = base + tid;
     int len = 0, fin = 0, s = 0;
@@ -97,12 +97,15 @@ ba_segment_blocks_kernel(const int32_t *__restrict__ lens, const int32_t *__rest
     int e_final = cta_exclusive_scan(fin ? len : 0, scan_smem, t_final);
     int e_tile = cta_exclusive_scan((len + tile_tok - 1) / tile_tok, scan_smem, t_tile);
     int e_ktile = cta_exclusive_scan(fin ? 0 : (len + 127) / 128, scan_smem, t_ktile);
+    int t_atile;
+    int e_atile = cta_exclusive_scan((len + 127) / 128, scan_smem, t_atile);
     if (b < B) {
       seg.cu_block[b] = c_all + e_all;
       seg.block_seq[b] = s;
       seg.block_is_final[b] = (uint8_t)fin;
       seg.block_part_off[b] = fin ? (c_final + e_final) : (c_cache + e_cache);
       seg.cu_qtile[b] = c_tile + e_tile;
+      seg.cu_ktile[b] = c_atile + e_atile;
       if (!fin) {
         // every earlier sequence contributed exactly one final block
         int c = b - s;
@@ -111,13 +114,14 @@ ba_segment_blocks_kernel(const int32_t *__restrict__ lens, const int32_t *__rest
         seg.cache_tile_cu[c] = c_ktile + e_ktile;
       }
     }
-    c_all += t_all; c_cache += t_cache; c_final += t_final; c_tile += t_tile; c_ktile += t_ktile;
+    c_all += t_all; c_cache += t_cache; c_final += t_final; c_tile += t_tile; c_ktile += t_ktile; c_atile += t_atile;
   }
   if (tid == 0) {
     seg.cu_block[B] = c_all;
     seg.cache_cu[B - batch] = c_cache;
     seg.cache_tile_cu[B - batch] = c_ktile;
     seg.cu_qtile[B] = c_tile;
+    seg.cu_ktile[B] = c_atile;
     seg.totals[0] = c_cache;
     seg.totals[1] = c_final;
     seg.totals[2] = c_tile;

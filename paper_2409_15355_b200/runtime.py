@@ -78,6 +78,7 @@ _TABLE_SIZES = {
     "cache_block": ("n_cached_blocks", 0), "cache_cu": ("n_cached_blocks", 1),
     "cache_delta": ("n_cached_blocks", 0), "tok_block": ("n_tokens", 0), "tok_pos": ("n_tokens", 0),
     "tok_pos_local": ("n_tokens", 0), "cu_qtile": ("n_blocks", 1), "cu_ftile": ("batch", 1), "cache_tile_cu": ("n_cached_blocks", 1),
+    "cu_ktile": ("n_blocks", 1),
 }
 
 
