@@ -448,8 +448,27 @@ def run_ours(args):
                    "ms": ms4, "algorithmic_flops": fl4, "tflops": fl4 / ms4 / 1e9, "allowed_pairs_per_head": pairs4,
                    "inputs": "seeded N(0,1) bf16 (workloads.prefill_inputs)"}
         assert ctx4.device_status() == B.BA_OK
+        # the backward pass of the same launch (block fine-tuning): forward with log-sum-exp, then gradients
+        lse4 = torch.empty(w4.n_tokens, w4.n_q_heads, dtype=torch.float32, device=dev)
+        B.ba_block_prefill(ctx4.ctx, q4, k4, v4, o4, lse4, seg4, B.BA_MODE_BLOCK, B.BA_OUT_BF16)
+        g4 = R.bits_to_tensor(W.normal_bf16(4004077, tuple(q4.shape))).to(dev)
+        dq4, dk4, dv4 = torch.empty_like(q4), torch.empty_like(k4), torch.empty_like(v4)
+        for _ in range(2):
+            B.ba_block_prefill_bwd(ctx4.ctx, q4, k4, v4, o4, lse4, g4, dq4, dk4, dv4, seg4, B.BA_MODE_BLOCK, B.BA_OUT_BF16)
+        torch.cuda.synchronize()
+        ev0.record(stream)
+        for _ in range(5):
+            B.ba_block_prefill_bwd(ctx4.ctx, q4, k4, v4, o4, lse4, g4, dq4, dk4, dv4, seg4, B.BA_MODE_BLOCK, B.BA_OUT_BF16)
+        ev1.record(stream)
+        torch.cuda.synchronize()
+        msb = ev0.elapsed_time(ev1) / 5
+        prefill["backward"] = {"workload": "gradients of the same launch (ba_block_prefill_bwd, bf16 gradients)", "ms": msb,
+                               "algorithmic_flops": 2.5 * fl4, "tflops": 2.5 * fl4 / msb / 1e9,
+                               "note": "five products per allowed pair (S, dP, dV, dK, dQ); the two kernels execute "
+                                       "seven (S and dP are formed in both)"}
+        assert ctx4.device_status() == B.BA_OK
         ctx4.close()
-        del q4, k4, v4, o4
+        del q4, k4, v4, o4, g4, dq4, dk4, dv4, lse4
         # the 32K prompt of the metric's workload encoded cold, under the full causal mask and under the
         # Block-attention mask (same tensors, one launch each): the paper's FLOPs / latency comparison
         T3 = w.n_tokens

@@ -234,6 +234,16 @@ __device__ __forceinline__ bool next_work(const AttnParams &p, int w, Work &wk) 
   return true;
 }
 
+// The last own key tile of an item covers the diagonal of the causal range.  When every row of the item
+// ends in the tile's first 64 keys (true for every other item: items are 64-token aligned, key tiles 128),
+// its second half is masked for all of them: the products and the exponentials of that half are skipped.
+__device__ __forceinline__ bool last_tile_is_half(const Work &wk) {
+  const Item &it = wk.it;
+  if (wk.tile0 + wk.n_tiles != it.n_tiles || it.n_tiles == it.n_cache_tiles) return false;   // the entry does not end the item
+  const int last_key0 = it.own_row0 + (it.n_tiles - it.n_cache_tiles - 1) * kBlockN;
+  return it.q_row0 + it.q_rows - 1 - last_key0 < kBlockN / 2;
+}
+
 // Block-by-block walk of the cached keys: index (cache order) of the block that holds key tile
 // `target` (counted over the whole batch); the sequence's blocks follow cb0.
 __device__ __forceinline__ int find_cache_block(const AttnParams &p, const Item &it, int target) {
@@ -476,6 +486,7 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
       const uint32_t tS[2] = {tmem, tmem + 128};
       const uint32_t tO[2] = {tmem + 256, tmem + 384};
       constexpr uint32_t idesc_qk = make_idesc_bf16(128, kBlockN, 0);
+      constexpr uint32_t idesc_qk_half = make_idesc_bf16(128, kBlockN / 2, 0);   // keys 0..63 of the tile only
       constexpr uint32_t idesc_pv = make_idesc_bf16(128, D, 1);
       const uint32_t q_addr[2] = {smem_u32(smem + L::kQ0), smem_u32(smem + L::kQ1)};
       const uint32_t ring = smem_u32(smem + L::kRing);
@@ -485,12 +496,15 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
       const uint64_t q_desc[2] = {make_smem_desc(q_addr[0], 16, 1024), make_smem_desc(q_addr[1], 16, 1024)};
       const uint64_t k_desc0 = make_smem_desc(ring, 16, 1024);
       const uint64_t v_desc0 = make_smem_desc(ring, L::kRegionBytes, 1024);
-      auto issue_qk_with = [&](int t, int idx, uint64_t qd) {
+      bool half_last = false;              // the entry's last key tile is used in its first 64 keys only
+      int entry_tiles = 0;
+      auto issue_qk_with = [&](int t, int jrel, int idx, uint64_t qd) {
         const uint64_t kd = k_desc0 + (uint64_t)(((idx % kStages) * L::kTileBytes) >> 4);
+        const uint32_t idesc = (half_last && jrel + 1 == entry_tiles) ? idesc_qk_half : idesc_qk;
 #pragma unroll
         for (int k = 0; k < D / 16; ++k) {
           const uint64_t off = (uint64_t)(((k >> 2) * L::kRegionBytes + (k & 3) * 32) >> 4);
-          mma_ss(tS[t], qd + off, kd + off, idesc_qk, k > 0);
+          mma_ss(tS[t], qd + off, kd + off, idesc, k > 0);
         }
         mma_commit(&ctrl->s_full[t]);
       };
@@ -519,7 +533,7 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
       int cached_end = 0;                  // tiles [tile0, cached_end) of the entry are cached keys
       // S_t = Q_t K^T for tile `jrel` of the entry, whose keys sit at ring position idx
       auto issue_qk = [&](int t, int jrel, int idx) -> bool {
-        if (!kFused) { issue_qk_with(t, idx, q_desc[t]); return true; }
+        if (!kFused) { issue_qk_with(t, jrel, idx, q_desc[t]); return true; }
         const int jt = wk.tile0 + jrel;
         bool change = false;
         if (jt < cached_end) {
@@ -541,7 +555,7 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
           ++n_ver[t];
           tc_fence_after();
         }
-        issue_qk_with(t, idx, ((n_ver[t] - 1) & 1) ? qb_desc[t] : q_desc[t]);
+        issue_qk_with(t, jrel, idx, ((n_ver[t] - 1) & 1) ? qb_desc[t] : q_desc[t]);
         return true;
       };
       for (;;) {
@@ -554,6 +568,8 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
         mbar_arrive(&ctrl->work_empty[slot]);          // the entry has been decoded into registers
         const int n_tiles = wk.n_tiles, n_qt = wk.it.n_qt;
         if (n_tiles == 0) continue;
+        half_last = last_tile_is_half(wk);
+        entry_tiles = n_tiles;
         walk_end = -1; ver_end[0] = ver_end[1] = -1;
         cached_end = min(wk.tile0 + n_tiles, wk.it.n_cache_tiles);
         if (!kFused) {
@@ -593,7 +609,7 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
             ok = mbar_wait(&ctrl->p_full[t][1], p_uses[t] & 1, abort_flag);
             if (!ok) continue;
             tc_fence_after();
-            issue_pv(t, iv, j == 0, 1);
+            if (!(last && half_last)) issue_pv(t, iv, j == 0, 1);
             ++p_uses[t];
             BA_TR(2, j, t * 4 + 2);
             if (last) mma_commit(&ctrl->o_done[t]);
@@ -656,6 +672,7 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
       if ((tid & 31) == 0) mbar_arrive(&ctrl->work_empty[slot]);   // one arrival per softmax warp
       const Item &it = wk.it;
       const int n_tiles = wk.n_tiles, tile0 = wk.tile0, head0 = wk.head0;
+      const bool half_last = last_tile_is_half(wk);
       if (t < it.n_qt) {
       const int q_last = it.q_row0 + it.q_rows - 1;
       const int row_tok = it.q_row0 + t * p.tok + (r >> p.hpt_log2);
@@ -733,66 +750,73 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
         ++s_uses;
         tc_fence_after();
         if (r == 0) BA_TR(t, j, 1);
-        uint32_t s[128];
-#pragma unroll
-        for (int c = 0; c < 4; ++c) tmem_ld_32x32b_x32(tS + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[c * 32]));
-        tmem_wait_ld();
-        if (r == 0) BA_TR(t, j, 2);
         // visible columns of this tile for this row: 0 .. lim
         int lim;
         const int jt = tile0 + j;
         if (jt < it.n_cache_tiles) lim = p.walk ? ctrl->tile_valid[(tiles_before + j) & 7] - 1
                                                      : it.cache_len - jt * kBlockN - 1;
         else lim = tok_c - (it.own_row0 + (jt - it.n_cache_tiles) * kBlockN);
-        if (lim < kBlockN - 1) {
+        uint64_t sum2[4] = {0ull, 0ull, 0ull, 0ull};       // packed (0.f, 0.f)
+        // One tile of softmax for this row over kCols key columns: 128, or 64 for a half tile (only the first
+        // 64 keys were multiplied; nothing of the second half is loaded, exponentiated or handed over).
+        auto tile_softmax = [&](auto cols_tag) {
+          constexpr int kCols = decltype(cols_tag)::value;
+          uint32_t s[kCols];
 #pragma unroll
-          for (int c = 0; c < 128; ++c)
-            if (c > lim) s[c] = 0xff800000u;                 // -inf
-        }
-        // row maximum by a wide tree of three-input maxima: 128 -> 43 -> 15 -> 5 -> 1
-        float l1[43];
+          for (int c = 0; c < kCols / 32; ++c) tmem_ld_32x32b_x32(tS + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[c * 32]));
+          tmem_wait_ld();
+          if (r == 0) BA_TR(t, j, 2);
+          if (lim < kCols - 1) {
 #pragma unroll
-        for (int i = 0; i < 42; ++i) l1[i] = max3(__uint_as_float(s[3 * i]), __uint_as_float(s[3 * i + 1]), __uint_as_float(s[3 * i + 2]));
-        l1[42] = fmaxf(__uint_as_float(s[126]), __uint_as_float(s[127]));
-        float l2[15];
+            for (int c = 0; c < kCols; ++c)
+              if (c > lim) s[c] = 0xff800000u;               // -inf
+          }
+          // row maximum by a wide tree of three-input maxima (128 -> 43 -> 15 -> 5 -> 1)
+          constexpr int n1 = (kCols + 2) / 3, n2 = (n1 + 2) / 3, n3 = (n2 + 2) / 3;
+          float l1[n1], l2[n2], l3[n3];
+          auto mx_at = [](const float *a, int n, int i) {    // max of a[3i], a[3i+1], a[3i+2] where they exist
+            return (3 * i + 2 < n) ? max3(a[3 * i], a[3 * i + 1], a[3 * i + 2])
+                                   : (3 * i + 1 < n) ? fmaxf(a[3 * i], a[3 * i + 1]) : a[3 * i];
+          };
+          const float *sf = reinterpret_cast<const float *>(s);
 #pragma unroll
-        for (int i = 0; i < 14; ++i) l2[i] = max3(l1[3 * i], l1[3 * i + 1], l1[3 * i + 2]);
-        l2[14] = l1[42];
-        float l3[5];
+          for (int i = 0; i < n1; ++i) l1[i] = mx_at(sf, kCols, i);
 #pragma unroll
-        for (int i = 0; i < 5; ++i) l3[i] = max3(l2[3 * i], l2[3 * i + 1], l2[3 * i + 2]);
-        const float mx = fmaxf(max3(l3[0], l3[1], l3[2]), fmaxf(l3[3], l3[4]));
-        const float m_new = fmaxf(m_used, mx);
-        if (r == 0) BA_TR(t, j, 3);
-        if (j == 0) {
-          m_used = m_new;
-        } else {
-          const bool grow = (m_new - m_used) * sl > kRescaleThreshold;
-          if (__any_sync(0xffffffffu, grow)) {
-            // 1 when this row's maximum did not move (also when the row has seen no key yet)
-            const float alpha = (m_new == -INFINITY) ? 1.f : ex2((m_used - m_new) * sl);
+          for (int i = 0; i < n2; ++i) l2[i] = mx_at(l1, n1, i);
+#pragma unroll
+          for (int i = 0; i < n3; ++i) l3[i] = mx_at(l2, n2, i);
+          float mx = l3[0];
+#pragma unroll
+          for (int i = 1; i < n3; ++i) mx = fmaxf(mx, l3[i]);
+          const float m_new = fmaxf(m_used, mx);
+          if (r == 0) BA_TR(t, j, 3);
+          if (j == 0) {
             m_used = m_new;
-            l *= alpha;
+          } else {
+            const bool grow = (m_new - m_used) * sl > kRescaleThreshold;
+            if (__any_sync(0xffffffffu, grow)) {
+              // 1 when this row's maximum did not move (also when the row has seen no key yet)
+              const float alpha = (m_new == -INFINITY) ? 1.f : ex2((m_used - m_new) * sl);
+              m_used = m_new;
+              l *= alpha;
 #pragma unroll
-            for (int c = 0; c < D / 32; ++c) {
-              uint32_t o[32];
-              tmem_ld_32x32b_x32(tO + c * 32, o);
-              tmem_wait_ld();
+              for (int c = 0; c < D / 32; ++c) {
+                uint32_t o[32];
+                tmem_ld_32x32b_x32(tO + c * 32, o);
+                tmem_wait_ld();
 #pragma unroll
-              for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
-              tmem_st_32x32b_x32(tO + c * 32, o);
+                for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+                tmem_st_32x32b_x32(tO + c * 32, o);
+              }
             }
           }
-        }
-        const float neg_m = (m_used == -INFINITY) ? 0.f : -m_used * sl;   // no visible key so far: every p is 0
-        uint64_t sum2[4] = {0ull, 0ull, 0ull, 0ull};       // packed (0.f, 0.f)
-        const uint64_t sl2 = pack2(sl, sl), negm2 = pack2(neg_m, neg_m);
-        // P is handed to the MMA warp in two halves so that PV can start on the first 64 keys
-        // while the second 64 are still being exponentiated.  The arithmetic is packed fp32x2.  The
-        // store of the first half completes while the second half is begun.
-        {
-          constexpr int kLead = 16;       // column pairs of the second half done before the first is handed over
-          uint32_t pk[32], pk1[32];
+          const float neg_m = (m_used == -INFINITY) ? 0.f : -m_used * sl;   // no visible key so far: every p is 0
+          const uint64_t sl2 = pack2(sl, sl), negm2 = pack2(neg_m, neg_m);
+          // P is handed to the MMA warp in two halves so that PV can start on the first 64 keys
+          // while the second 64 are still being exponentiated.  The arithmetic is packed fp32x2.  The
+          // store of the first half completes while the second half is begun.
+          constexpr int kLead = kCols > 64 ? 16 : 0;       // column pairs of the second half done before the first is handed over
+          uint32_t pk[32], pk1[kCols > 64 ? 32 : 1];
           auto expo = [&](int e0, uint32_t &dst, int i) {
             const uint64_t x2 = fma2(pack2(__uint_as_float(s[e0]), __uint_as_float(s[e0 + 1])), sl2, negm2);
             float x0, x1;
@@ -811,14 +835,18 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
           tc_fence_before();
           mbar_arrive(&ctrl->p_full[t][0]);
           if (r == 0) BA_TR(t, j, 4);
+          if constexpr (kCols > 64) {
 #pragma unroll
-          for (int i = kLead; i < 32; ++i) expo(64 + 2 * i, pk1[i], i);
-          tmem_st_32x32b_x32(tS + 32, pk1);
-          tmem_wait_st();
-          tc_fence_before();
-          mbar_arrive(&ctrl->p_full[t][1]);
+            for (int i = kLead; i < 32; ++i) expo(64 + 2 * i, pk1[i], i);
+            tmem_st_32x32b_x32(tS + 32, *reinterpret_cast<uint32_t(*)[32]>(&pk1[0]));
+            tmem_wait_st();
+            tc_fence_before();
+          }
+          mbar_arrive(&ctrl->p_full[t][1]);               // (half tile: nothing to hand over, that product is skipped)
           if (r == 0) BA_TR(t, j, 5);
-        }
+        };
+        if (half_last && j + 1 == n_tiles) tile_softmax(std::integral_constant<int, kBlockN / 2>{});
+        else tile_softmax(std::integral_constant<int, kBlockN>{});
         // P of this tile is with the tensor core: time to work on the next version of the query row
         if (kFused && next_start < tile_end) {
           const bool due = tile0 + j + 1 == next_start;    // the next tile is the first to need it
