@@ -8,6 +8,7 @@
 ba_status ba_attend_sm100_launch(ba_ctx *ctx, const ba_attend_args &a, const ba_segments *seg,
                                  cudaStream_t stream);
 ba_status ba_attend_sm100_setup(ba_ctx *ctx);
+ba_status ba_bwd_sm100_setup(ba_ctx *ctx);
 ba_status ba_bwd_sm100_launch(ba_ctx *ctx, const void *q, const void *k, const void *v, const void *o,
                               const float *lse, const void *d_o, void *dq, void *dk, void *dv, int out_f32,
                               const ba_segments *seg, int mode, cudaStream_t stream);
@@ -144,8 +145,9 @@ ba_status ba_create(ba_ctx **out, const ba_config *cfg, int device, size_t works
       cudaStreamCreateWithFlags(&ctx->side_stream, cudaStreamNonBlocking) != cudaSuccess ||
       cudaEventCreateWithFlags(&ctx->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
       cudaEventCreateWithFlags(&ctx->ev_join, cudaEventDisableTiming) != cudaSuccess ||
-      ba_attend_sm100_setup(ctx) != BA_OK) {
+      ba_attend_sm100_setup(ctx) != BA_OK || ba_bwd_sm100_setup(ctx) != BA_OK) {
     cudaGetLastError();
+    ba_attend_sm100_teardown(ctx);
     if (ctx->ev_join) cudaEventDestroy(ctx->ev_join);
     if (ctx->ev_fork) cudaEventDestroy(ctx->ev_fork);
     if (ctx->side_stream) cudaStreamDestroy(ctx->side_stream);

@@ -1177,10 +1177,8 @@ ba_status ba_attend_sm100_launch(ba_ctx *ctx, const ba_attend_args &a, const ba_
   if (ctx->workspace && ctx->workspace_bytes >= ba_scratch_offset(ctx))
     counters = reinterpret_cast<int32_t *>(reinterpret_cast<char *>(ctx->workspace) + ba_scratch_offset(ctx) - 256);
   p.counters = nullptr;
-  if (p.persistent) {
-    if (!counters) return BA_ERR_WORKSPACE;
-    p.counters = counters;
-  }
+  if (p.persistent && !counters) p.persistent = 0;   // a context without workspace: one CTA per entry, however many
+  if (p.persistent) p.counters = counters;
   p.o_part = nullptr; p.lse_part = nullptr;
   if (n_splits > 1) {
     p.o_part = reinterpret_cast<float *>(reinterpret_cast<char *>(ctx->workspace) + ba_scratch_offset(ctx));

@@ -217,6 +217,14 @@ ba_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
           tma_load_3d(smem + L::kQ + c * L::kRegion, &tmap_q, &ctrl->q_full, c * 64, head0, row0);
           tma_load_3d(smem + L::kDO + c * L::kRegion, &tmap_do, &ctrl->q_full, c * 64, head0, row0);
         }
+        if (it + 1 < n_iter) {                           // the next iteration's tiles are asked into L2 meanwhile
+          const int tn = (it + 1) / n_chunks, cn = it + 1 - tn * n_chunks;
+          const int rown = tn < tiles1 ? r1_begin + tn * p.tok : r2_begin + (tn - tiles1) * p.tok;
+          for (int c = 0; c < L::kChunks; ++c) {
+            tma_prefetch_3d(&tmap_q, c * 64, g * p.G + cn * p.hpt, rown);
+            tma_prefetch_3d(&tmap_do, c * 64, g * p.G + cn * p.hpt, rown);
+          }
+        }
         ok = mbar_wait(&ctrl->q_full, it & 1, abort_flag);
         if (!ok) break;
         tc_fence_after();
@@ -360,6 +368,11 @@ ba_bwd_dq_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
           tma_load_3d(smem + L::kK + c * L::kRegion, &tmap_k, &ctrl->kv_full, c * 64, g, kr);
           tma_load_3d(smem + L::kV + c * L::kRegion, &tmap_v, &ctrl->kv_full, c * 64, g, kr);
         }
+        if (it + 1 < n_iter)
+          for (int c = 0; c < L::kChunks; ++c) {
+            tma_prefetch_3d(&tmap_k, c * 64, g, kr + kTile);
+            tma_prefetch_3d(&tmap_v, c * 64, g, kr + kTile);
+          }
         ok = mbar_wait(&ctrl->kv_full, it & 1, abort_flag);
         if (!ok) break;
         tc_fence_after();
@@ -469,8 +482,6 @@ ba_status launch_bwd(ba_ctx *ctx, const BwdParams &p, const CUtensorMap &tq, con
                      const CUtensorMap &tk, const CUtensorMap &tv, int n_ktiles_upper, int n_pairs_upper,
                      cudaStream_t stream) {
   const int smem = BwdLayout<D>::kBytes + 1024;
-  BA_CUDA_TRY(cudaFuncSetAttribute(ba_bwd_dkv_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-  BA_CUDA_TRY(cudaFuncSetAttribute(ba_bwd_dq_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
   ba_bwd_dkv_kernel<D><<<dim3((unsigned)n_ktiles_upper, (unsigned)p.Hkv), kBwdThreads, smem, stream>>>(tq, tdo, tk, tv, p);
   BA_CUDA_TRY(cudaGetLastError());
   ba_bwd_dq_kernel<D><<<dim3((unsigned)(2 * n_pairs_upper), (unsigned)(p.Hq / p.hpt)), kBwdThreads, smem, stream>>>(tq, tdo, tk, tv, p);
@@ -480,6 +491,15 @@ ba_status launch_bwd(ba_ctx *ctx, const BwdParams &p, const CUtensorMap &tq, con
 }
 
 }  // namespace
+
+// Per-context set-up (device current): the kernels' shared-memory limit is raised once.
+ba_status ba_bwd_sm100_setup(ba_ctx *) {
+  BA_CUDA_TRY(cudaFuncSetAttribute(ba_bwd_dkv_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdLayout<128>::kBytes + 1024));
+  BA_CUDA_TRY(cudaFuncSetAttribute(ba_bwd_dq_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdLayout<128>::kBytes + 1024));
+  BA_CUDA_TRY(cudaFuncSetAttribute(ba_bwd_dkv_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdLayout<64>::kBytes + 1024));
+  BA_CUDA_TRY(cudaFuncSetAttribute(ba_bwd_dq_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdLayout<64>::kBytes + 1024));
+  return BA_OK;
+}
 
 ba_status ba_bwd_sm100_launch(ba_ctx *ctx, const void *q, const void *k, const void *v, const void *o,
                               const float *lse, const void *d_o, void *dq, void *dk, void *dv, int out_f32,
