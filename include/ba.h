@@ -129,7 +129,9 @@ ba_status ba_create(ba_ctx **ctx, const ba_config *cfg, int device, size_t works
 ba_status ba_destroy(ba_ctx *ctx);
 const char *ba_status_string(ba_status s);
 
-/* Workspace ba_create() should be given so that calls of at most these sizes fit. */
+/* Workspace ba_create() should be given so that calls of at most these sizes fit: max_blocks cached
+ * blocks per re-encoding call, max_q_rows query rows per attention call (split-KV partial results are
+ * only used for short query sides) and per backward call (its dO . O buffer). */
 ba_status ba_workspace_bytes(const ba_config *cfg, int32_t max_blocks, int32_t max_q_rows, size_t *bytes);
 
 /* Synchronises the context's device and returns (then clears) the first

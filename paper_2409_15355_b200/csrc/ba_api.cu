@@ -100,7 +100,10 @@ ba_status ba_workspace_bytes(const ba_config *cfg, int32_t max_blocks, int32_t m
   size_t splits = split_rows * cfg->n_q_heads * (cfg->head_dim + 1) * sizeof(float) * 6;
   size_t stage = stage_bytes_for(max_blocks);
   if (stage < 64 * 1024) stage = 64 * 1024;
+  // the backward pass keeps dO . O (fp32 per row and query head) there
+  size_t bwd = (size_t)max_q_rows * cfg->n_q_heads * sizeof(float);
   size_t scratch = table > splits ? table : splits;
+  if (bwd > scratch) scratch = bwd;
   *bytes = stage + ba_align_up(scratch, 256) + 256;
   return BA_OK;
 }
