@@ -8,12 +8,16 @@
 // 128 x 128 tiles on the tensor cores (tcgen05.mma, accumulators in tensor memory), neither uses
 // atomics, so results are run-to-run identical:
 //   * ba_bwd_dkv_kernel: one CTA owns 128 keys of one block and one KV head and walks over every
-//     query tile that sees them (all heads of the group): S and dP by two products, P and dS by its
-//     128 row threads (written to shared memory as bf16), then dV += P^T dO and dK += dS^T Q.
+//     query tile that sees them (all heads of the group).  It forms the scores transposed, S^T = K Q^T
+//     and dP^T = V dO^T (keys on the tensor-memory lanes, query rows on the columns), so that its 128
+//     threads -- one per key -- write P^T and dS^T back to tensor memory as bf16, where they are the A
+//     operands of dV += P^T dO and dK += dS^T Q (nothing goes through shared memory, nothing is transposed).
 //   * ba_bwd_dq_kernel: one CTA owns one query tile (tokens x heads of one KV group, as in the
-//     forward kernel) and walks over the key tiles it sees: S, dP, dS as above, dQ += dS K.
-// The steps of a tile run one after the other (loads, two products, row work, two products): the
-// kernels are simple rather than pipelined.
+//     forward kernel) and walks over the key tiles it sees: S = Q K^T, dP = dO V^T (query rows on the
+//     lanes), dS written to tensor memory, dQ += dS K.
+// The tiles a CTA walks over (Q and dO there, K and V here) are double-buffered in shared memory, so the
+// loads of the next step run under the current one; within a step the two score products, the thread
+// work and the two (one) gradient products follow one another, because S and dP exist once in tensor memory.
 #include <math.h>
 
 #include "ba_common.cuh"
@@ -46,18 +50,30 @@ struct BwdLayout {
   static constexpr int kChunks = D / 64;
   static constexpr int kRegion = 128 * 128;              // 128 rows x 128 bytes
   static constexpr int kTileBytes = 128 * D * 2;
-  static constexpr int kQ = 0, kDO = kTileBytes, kK = 2 * kTileBytes, kV = 3 * kTileBytes;
-  static constexpr int kP = 4 * kTileBytes;               // [128 q rows x 128 keys] bf16
-  static constexpr int kDS = kP + 2 * kRegion;
-  static constexpr int kCtrl = kDS + 2 * kRegion;
+  // two tiles that stay for the whole CTA (K, V in the dK/dV kernel; Q, dO in the dQ kernel) and two
+  // buffers of two tiles each for the ones it walks over
+  static constexpr int kFix0 = 0, kFix1 = kTileBytes;
+  static constexpr int kWalk = 2 * kTileBytes;            // buffer b: tiles at kWalk + b * 2 * kTileBytes, + kTileBytes
+  static constexpr int kStats = 6 * kTileBytes;           // dK/dV kernel: per query row {lse * log2 e, dO . O, visible keys, -}, two buffers
+  static constexpr int kCtrl = kStats + 2 * 128 * 16;
   static constexpr int kBytes = kCtrl + 256;
 };
 
 struct BwdCtrl {
-  uint64_t kv_full, q_full, sd_full, rows_done, acc_done;
+  uint64_t fix_full, walk_full[2], sd_full, rows_done, acc_done;
   uint32_t tmem_base;
   int abort_flag;
 };
+
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+        "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+      : "memory");
+}
+__device__ __forceinline__ void named_barrier_128() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
 __device__ __forceinline__ int upper_bound_dev(const int32_t *a, int n, int x) {
   int lo = 0, hi = n;
@@ -68,20 +84,19 @@ __device__ __forceinline__ int upper_bound_dev(const int32_t *a, int n, int x) {
   return lo;
 }
 
-// One row of P and dS for a 128-key tile: reads the row of S and dP from tensor memory in chunks of 32
-// columns, p = exp2(s * scale_log2 - lse_log2) where the mask allows, ds = p (dp - delta) scale, and stores
-// both as bf16 in the 128-byte swizzled layout of a [128 rows x 128 keys] tile (two 64-key regions).
+// dQ kernel, one query row (= lane) against a 128-key tile: reads the row of S and dP from tensor memory in
+// chunks of 32 columns, p = exp2(s * scale_log2 - lse_log2) where the mask allows, ds = p (dp - delta) scale,
+// and writes dS back over the dP columns as bf16 (two per column), the A operand of dQ += dS K.
 // `n_ok`: columns 0 .. n_ok - 1 are visible to this row (0: none).
-__device__ __forceinline__ void bwd_row(uint32_t tS, uint32_t tDP, uint8_t *p_s, uint8_t *ds_s, int r, int n_ok,
-                                        float scale_log2, float lse_log2, float delta, float scale) {
-  const int rb = r * 128, sw = r & 7;
+__device__ __forceinline__ void bwd_row_ds(uint32_t tS, uint32_t tDP, int n_ok, float scale_log2, float lse_log2,
+                                           float delta, float scale) {
 #pragma unroll
   for (int c = 0; c < 4; ++c) {
     uint32_t s[32], dp[32];
     tmem_ld_32x32b_x32(tS + c * 32, s);
     tmem_ld_32x32b_x32(tDP + c * 32, dp);
     tmem_wait_ld();
-    uint32_t pw[16], dw[16];
+    uint32_t dw[16];
 #pragma unroll
     for (int i = 0; i < 16; ++i) {
       const int e0 = c * 32 + 2 * i;
@@ -91,19 +106,44 @@ __device__ __forceinline__ void bwd_row(uint32_t tS, uint32_t tDP, uint8_t *p_s,
       if (e0 + 1 >= n_ok) p1 = 0.f;
       const float d0 = p0 * (__uint_as_float(dp[2 * i]) - delta) * scale;
       const float d1 = p1 * (__uint_as_float(dp[2 * i + 1]) - delta) * scale;
+      __nv_bfloat162 dv = __floats2bfloat162_rn(d0, d1);
+      dw[i] = *reinterpret_cast<uint32_t *>(&dv);
+    }
+    tmem_st16(tDP + c * 16, dw);         // columns 16 c .. 16 c + 15: inside the part of dP already read
+  }
+  tmem_wait_st();
+}
+
+// dK/dV kernel, one key (= lane `j`) against the 128 query rows of a tile (= columns): S^T and dP^T come
+// from tensor memory in chunks of 32 columns; the per-row values (lse * log2 e, dO . O, number of keys of
+// this tile the row sees) are read from shared memory, the same address by every thread.  P^T goes back
+// over the S^T columns and dS^T over the dP^T columns as bf16.
+__device__ __forceinline__ void bwd_key_p_ds(uint32_t tST, uint32_t tDPT, int j, const float4 *stats,
+                                             float scale_log2, float scale) {
+#pragma unroll
+  for (int c = 0; c < 4; ++c) {
+    uint32_t s[32], dp[32];
+    tmem_ld_32x32b_x32(tST + c * 32, s);
+    tmem_ld_32x32b_x32(tDPT + c * 32, dp);
+    tmem_wait_ld();
+    uint32_t pw[16], dw[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      const float4 a = stats[c * 32 + 2 * i], b = stats[c * 32 + 2 * i + 1];
+      float p0 = ex2(fmaf(__uint_as_float(s[2 * i]), scale_log2, -a.x));
+      float p1 = ex2(fmaf(__uint_as_float(s[2 * i + 1]), scale_log2, -b.x));
+      if (j >= __float_as_int(a.z)) p0 = 0.f;
+      if (j >= __float_as_int(b.z)) p1 = 0.f;
+      const float d0 = p0 * (__uint_as_float(dp[2 * i]) - a.y) * scale;
+      const float d1 = p1 * (__uint_as_float(dp[2 * i + 1]) - b.y) * scale;
       __nv_bfloat162 pv = __floats2bfloat162_rn(p0, p1), dv = __floats2bfloat162_rn(d0, d1);
       pw[i] = *reinterpret_cast<uint32_t *>(&pv);
       dw[i] = *reinterpret_cast<uint32_t *>(&dv);
     }
-    // columns 32 c .. 32 c + 31 = four 16-byte chunks: chunk index 4 c + k of the row
-#pragma unroll
-    for (int k = 0; k < 4; ++k) {
-      const int ch = 4 * c + k;
-      const int off = (ch >> 3) * (128 * 128) + rb + (((ch & 7) ^ sw) << 4);
-      if (p_s) *reinterpret_cast<uint4 *>(p_s + off) = make_uint4(pw[4 * k], pw[4 * k + 1], pw[4 * k + 2], pw[4 * k + 3]);
-      *reinterpret_cast<uint4 *>(ds_s + off) = make_uint4(dw[4 * k], dw[4 * k + 1], dw[4 * k + 2], dw[4 * k + 3]);
-    }
+    tmem_st16(tST + c * 16, pw);
+    tmem_st16(tDPT + c * 16, dw);
   }
+  tmem_wait_st();
 }
 
 // Writes one accumulator row (D fp32 columns of tensor memory, lane = row) to global memory.
@@ -166,16 +206,24 @@ ba_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
   const int seq1 = __ldg(sg.cu_seq + sq + 1);
   const int fin0 = __ldg(sg.cu_block + __ldg(sg.cu_seq_block + sq + 1) - 1);    // first row of the final block
   const bool is_final = __ldg(sg.block_is_final + b) != 0;
-  int r1_begin = k0, r1_end = (p.mode == BA_MODE_FULL) ? seq1 : blk1;           // causal range
+  const int r1_begin = k0, r1_end = (p.mode == BA_MODE_FULL) ? seq1 : blk1;     // causal range
   int r2_begin = 0, r2_end = 0;                                                 // range that sees all the keys
   if (p.mode == BA_MODE_BLOCK && !is_final) { r2_begin = fin0; r2_end = seq1; }
   const int tiles1 = (r1_end - r1_begin + p.tok - 1) / p.tok, tiles2 = (r2_end - r2_begin + p.tok - 1) / p.tok;
   const int n_chunks = p.G / p.hpt;                                             // head chunks of this KV group
   const int n_iter = (tiles1 + tiles2) * n_chunks;
+  // iteration `it`: token tile it / n_chunks, head chunk it % n_chunks
+  auto iter_rows = [&](int it, int &row0, int &row_end, bool &causal, int &head0) {
+    const int ti = it / n_chunks, ch = it - ti * n_chunks;
+    causal = ti < tiles1;
+    row0 = causal ? r1_begin + ti * p.tok : r2_begin + (ti - tiles1) * p.tok;
+    row_end = causal ? r1_end : r2_end;
+    head0 = g * p.G + ch * p.hpt;
+  };
 
   if (tid == 0) {
-    mbar_init(&ctrl->kv_full, 1); mbar_init(&ctrl->q_full, 1); mbar_init(&ctrl->sd_full, 1);
-    mbar_init(&ctrl->rows_done, 128); mbar_init(&ctrl->acc_done, 1);
+    mbar_init(&ctrl->fix_full, 1); mbar_init(&ctrl->walk_full[0], 1); mbar_init(&ctrl->walk_full[1], 1);
+    mbar_init(&ctrl->sd_full, 1); mbar_init(&ctrl->rows_done, 128); mbar_init(&ctrl->acc_done, 1);
     ctrl->abort_flag = 0;
     fence_barrier_init();
   }
@@ -185,114 +233,109 @@ ba_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
   tc_fence_after();
   const uint32_t tmem = ctrl->tmem_base;
   volatile int *abort_flag = &ctrl->abort_flag;
-  const uint32_t tS = tmem, tDP = tmem + 128, tDV = tmem + 256, tDK = tmem + 384;
+  const uint32_t tST = tmem, tDPT = tmem + 128, tDV = tmem + 256, tDK = tmem + 384;
 
   if (warp == 4) {
     if (elect_one()) {
       constexpr uint32_t idesc_nt = make_idesc_bf16(128, kTile, 0);             // both operands K-major
-      constexpr uint32_t idesc_tn = make_idesc_bf16(128, D, 1) | (1u << 15);    // both operands MN-major
-      const uint64_t q_desc = make_smem_desc(smem_u32(smem + L::kQ), 16, 1024);
-      const uint64_t do_desc = make_smem_desc(smem_u32(smem + L::kDO), 16, 1024);
-      const uint64_t k_desc = make_smem_desc(smem_u32(smem + L::kK), 16, 1024);
-      const uint64_t v_desc = make_smem_desc(smem_u32(smem + L::kV), 16, 1024);
-      const uint64_t p_mn = make_smem_desc(smem_u32(smem + L::kP), L::kRegion, 1024);
-      const uint64_t ds_mn = make_smem_desc(smem_u32(smem + L::kDS), L::kRegion, 1024);
-      const uint64_t do_mn = make_smem_desc(smem_u32(smem + L::kDO), L::kRegion, 1024);
-      const uint64_t q_mn = make_smem_desc(smem_u32(smem + L::kQ), L::kRegion, 1024);
+      constexpr uint32_t idesc_tn = make_idesc_bf16(128, D, 1);                 // A from tensor memory, B MN-major
+      const uint64_t k_desc = make_smem_desc(smem_u32(smem + L::kFix0), 16, 1024);
+      const uint64_t v_desc = make_smem_desc(smem_u32(smem + L::kFix1), 16, 1024);
       bool ok = true;
-      mbar_arrive_expect_tx(&ctrl->kv_full, 2 * L::kTileBytes);
-      for (int c = 0; c < L::kChunks; ++c) {
-        tma_load_3d(smem + L::kK + c * L::kRegion, &tmap_k, &ctrl->kv_full, c * 64, g, k0);
-        tma_load_3d(smem + L::kV + c * L::kRegion, &tmap_v, &ctrl->kv_full, c * 64, g, k0);
-      }
-      ok = mbar_wait(&ctrl->kv_full, 0, abort_flag);
-      for (int it = 0; it < n_iter && ok; ++it) {
-        const int ti = it / n_chunks, ch = it - ti * n_chunks;
-        const int row0 = ti < tiles1 ? r1_begin + ti * p.tok : r2_begin + (ti - tiles1) * p.tok;
-        const int head0 = g * p.G + ch * p.hpt;
-        // the products of the previous iteration have read Q, dO, P and dS: the buffers may be refilled
-        if (it > 0) { ok = mbar_wait(&ctrl->acc_done, (it - 1) & 1, abort_flag); if (!ok) break; }
-        mbar_arrive_expect_tx(&ctrl->q_full, 2 * L::kTileBytes);
+      auto load_walk = [&](int it) {                     // Q and dO tiles of iteration `it` into buffer it & 1
+        int row0, row_end, head0; bool causal;
+        iter_rows(it, row0, row_end, causal, head0);
+        uint8_t *dst = smem + L::kWalk + (it & 1) * 2 * L::kTileBytes;
+        mbar_arrive_expect_tx(&ctrl->walk_full[it & 1], 2 * L::kTileBytes);
         for (int c = 0; c < L::kChunks; ++c) {
-          tma_load_3d(smem + L::kQ + c * L::kRegion, &tmap_q, &ctrl->q_full, c * 64, head0, row0);
-          tma_load_3d(smem + L::kDO + c * L::kRegion, &tmap_do, &ctrl->q_full, c * 64, head0, row0);
+          tma_load_3d(dst + c * L::kRegion, &tmap_q, &ctrl->walk_full[it & 1], c * 64, head0, row0);
+          tma_load_3d(dst + L::kTileBytes + c * L::kRegion, &tmap_do, &ctrl->walk_full[it & 1], c * 64, head0, row0);
         }
-        if (it + 1 < n_iter) {                           // the next iteration's tiles are asked into L2 meanwhile
-          const int tn = (it + 1) / n_chunks, cn = it + 1 - tn * n_chunks;
-          const int rown = tn < tiles1 ? r1_begin + tn * p.tok : r2_begin + (tn - tiles1) * p.tok;
-          for (int c = 0; c < L::kChunks; ++c) {
-            tma_prefetch_3d(&tmap_q, c * 64, g * p.G + cn * p.hpt, rown);
-            tma_prefetch_3d(&tmap_do, c * 64, g * p.G + cn * p.hpt, rown);
-          }
-        }
-        ok = mbar_wait(&ctrl->q_full, it & 1, abort_flag);
+      };
+      mbar_arrive_expect_tx(&ctrl->fix_full, 2 * L::kTileBytes);
+      for (int c = 0; c < L::kChunks; ++c) {
+        tma_load_3d(smem + L::kFix0 + c * L::kRegion, &tmap_k, &ctrl->fix_full, c * 64, g, k0);
+        tma_load_3d(smem + L::kFix1 + c * L::kRegion, &tmap_v, &ctrl->fix_full, c * 64, g, k0);
+      }
+      if (n_iter > 0) load_walk(0);
+      if (n_iter > 1) load_walk(1);
+      ok = mbar_wait(&ctrl->fix_full, 0, abort_flag);
+      for (int it = 0; it < n_iter && ok; ++it) {
+        const int bf = it & 1;
+        const uint32_t walk = smem_u32(smem + L::kWalk + bf * 2 * L::kTileBytes);
+        const uint64_t q_desc = make_smem_desc(walk, 16, 1024);
+        const uint64_t do_desc = make_smem_desc(walk + L::kTileBytes, 16, 1024);
+        const uint64_t q_mn = make_smem_desc(walk, L::kRegion, 1024);
+        const uint64_t do_mn = make_smem_desc(walk + L::kTileBytes, L::kRegion, 1024);
+        ok = mbar_wait(&ctrl->walk_full[bf], (it >> 1) & 1, abort_flag);
         if (!ok) break;
         tc_fence_after();
+        // S^T = K Q^T, dP^T = V dO^T (they follow the previous iteration's gradient products on the tensor
+        // pipe in issue order, so those have read P^T and dS^T before these overwrite the columns)
 #pragma unroll
         for (int k = 0; k < D / 16; ++k) {
           const uint64_t off = (uint64_t)(((k >> 2) * L::kRegion + (k & 3) * 32) >> 4);
-          mma_ss(tS, q_desc + off, k_desc + off, idesc_nt, k > 0);
+          mma_ss(tST, k_desc + off, q_desc + off, idesc_nt, k > 0);
         }
 #pragma unroll
         for (int k = 0; k < D / 16; ++k) {
           const uint64_t off = (uint64_t)(((k >> 2) * L::kRegion + (k & 3) * 32) >> 4);
-          mma_ss(tDP, do_desc + off, v_desc + off, idesc_nt, k > 0);
+          mma_ss(tDPT, v_desc + off, do_desc + off, idesc_nt, k > 0);
         }
         mma_commit(&ctrl->sd_full);
-        // the row threads turn S and dP into P and dS in shared memory
+        // the previous iteration's gradient products have read its Q and dO: that buffer takes iteration it + 1
+        if (it > 0) {
+          ok = mbar_wait(&ctrl->acc_done, (it - 1) & 1, abort_flag);
+          if (!ok) break;
+          if (it + 1 < n_iter) load_walk(it + 1);
+        }
+        // the key threads turn S^T and dP^T into P^T and dS^T (bf16, in place)
         ok = mbar_wait(&ctrl->rows_done, it & 1, abort_flag);
         if (!ok) break;
         tc_fence_after();
 #pragma unroll
-        for (int k = 0; k < kTile / 16; ++k) {           // contraction over the 128 query rows, 16 at a time
-          const uint64_t off = (uint64_t)((k * 2048) >> 4);
-          mma_ss(tDV, p_mn + off, do_mn + off, idesc_tn, (it > 0 || k > 0) ? 1u : 0u);
-        }
+        for (int k = 0; k < kTile / 16; ++k)             // contraction over the 128 query rows, 16 at a time
+          mma_ts(tDV, tST + k * 8, do_mn + (uint64_t)((k * 2048) >> 4), idesc_tn, (it > 0 || k > 0) ? 1u : 0u);
 #pragma unroll
-        for (int k = 0; k < kTile / 16; ++k) {
-          const uint64_t off = (uint64_t)((k * 2048) >> 4);
-          mma_ss(tDK, ds_mn + off, q_mn + off, idesc_tn, (it > 0 || k > 0) ? 1u : 0u);
-        }
+        for (int k = 0; k < kTile / 16; ++k)
+          mma_ts(tDK, tDPT + k * 8, q_mn + (uint64_t)((k * 2048) >> 4), idesc_tn, (it > 0 || k > 0) ? 1u : 0u);
         mma_commit(&ctrl->acc_done);
       }
     }
   } else {
-    const int r = tid;                                   // row of the query tile = tensor-memory lane
+    const int j = tid;                                   // key of the tile = tensor-memory lane
     const uint32_t lane_off = (uint32_t)(warp * 32) << 16;
+    float4 *stats = reinterpret_cast<float4 *>(smem + L::kStats);
     bool ok = true;
     for (int it = 0; it < n_iter; ++it) {
-      const int ti = it / n_chunks, ch = it - ti * n_chunks;
-      const bool causal = ti < tiles1;
-      const int row0 = causal ? r1_begin + ti * p.tok : r2_begin + (ti - tiles1) * p.tok;
-      const int row_end = causal ? r1_end : r2_end;
-      const int tok_i = row0 + (r >> p.hpt_log2);
-      const int head = g * p.G + ch * p.hpt + (r & (p.hpt - 1));
-      const bool row_ok = tok_i < row_end;
-      int n_ok = 0;                                      // visible key columns of this row
-      if (row_ok) n_ok = causal ? min(n_keys, tok_i - k0 + 1) : n_keys;
-      float lse2 = 0.f, dl = 0.f;
-      if (row_ok) {
-        lse2 = __ldg(p.lse + (size_t)tok_i * p.Hq + head) * 1.4426950408889634f;
-        dl = __ldg(p.delta + (size_t)tok_i * p.Hq + head);
+      // this thread also prepares what every key thread needs to know about query row `tid` of the tile
+      int row0, row_end, head0; bool causal;
+      iter_rows(it, row0, row_end, causal, head0);
+      const int tok_i = row0 + (tid >> p.hpt_log2);
+      const int head = head0 + (tid & (p.hpt - 1));
+      float4 st = make_float4(0.f, 0.f, __int_as_float(0), 0.f);
+      if (tok_i < row_end) {
+        st.x = __ldg(p.lse + (size_t)tok_i * p.Hq + head) * 1.4426950408889634f;
+        st.y = __ldg(p.delta + (size_t)tok_i * p.Hq + head);
+        st.z = __int_as_float(causal ? max(0, min(n_keys, tok_i - k0 + 1)) : n_keys);   // keys 0 .. z - 1 of the tile are visible
       }
+      stats[(it & 1) * 128 + tid] = st;
+      named_barrier_128();
       ok = mbar_wait(&ctrl->sd_full, it & 1, abort_flag);
       if (!ok) break;
       tc_fence_after();
-      bwd_row(tS + lane_off, tDP + lane_off, smem + L::kP, smem + L::kDS, r, n_ok, p.scale_log2, lse2, dl, p.scale);
+      bwd_key_p_ds(tST + lane_off, tDPT + lane_off, j, stats + (it & 1) * 128, p.scale_log2, p.scale);
       tc_fence_before();
-      fence_proxy_async();                               // the tensor core reads P and dS through the async proxy
       mbar_arrive(&ctrl->rows_done);
     }
     // accumulators: lane = key row of the tile
     if (ok && n_iter > 0) ok = mbar_wait(&ctrl->acc_done, (n_iter - 1) & 1, abort_flag);
-    if (ok) {
+    if (ok && n_iter > 0) {
       tc_fence_after();
-      const bool valid = r < n_keys;
-      const size_t off = ((size_t)(k0 + r) * p.Hkv + g) * D;
-      if (n_iter > 0) {
-        store_acc_row<D>(tDV + lane_off, p.dv, off, p.out_f32, valid);
-        store_acc_row<D>(tDK + lane_off, p.dk, off, p.out_f32, valid);
-      }
+      const bool valid = j < n_keys;
+      const size_t off = ((size_t)(k0 + j) * p.Hkv + g) * D;
+      store_acc_row<D>(tDV + lane_off, p.dv, off, p.out_f32, valid);
+      store_acc_row<D>(tDK + lane_off, p.dk, off, p.out_f32, valid);
     }
   }
   tc_fence_before();
@@ -330,8 +373,8 @@ ba_bwd_dq_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
   const int n_iter = (q_end - kv0 + kTile - 1) / kTile;   // key tiles kv0 + 128 j
 
   if (tid == 0) {
-    mbar_init(&ctrl->kv_full, 1); mbar_init(&ctrl->q_full, 1); mbar_init(&ctrl->sd_full, 1);
-    mbar_init(&ctrl->rows_done, 128); mbar_init(&ctrl->acc_done, 1);
+    mbar_init(&ctrl->fix_full, 1); mbar_init(&ctrl->walk_full[0], 1); mbar_init(&ctrl->walk_full[1], 1);
+    mbar_init(&ctrl->sd_full, 1); mbar_init(&ctrl->rows_done, 128); mbar_init(&ctrl->acc_done, 1);
     ctrl->abort_flag = 0;
     fence_barrier_init();
   }
@@ -346,34 +389,33 @@ ba_bwd_dq_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
   if (warp == 4) {
     if (elect_one()) {
       constexpr uint32_t idesc_nt = make_idesc_bf16(128, kTile, 0);
-      constexpr uint32_t idesc_nn = make_idesc_bf16(128, D, 1);                 // A K-major (dS), B MN-major (K)
-      const uint64_t q_desc = make_smem_desc(smem_u32(smem + L::kQ), 16, 1024);
-      const uint64_t do_desc = make_smem_desc(smem_u32(smem + L::kDO), 16, 1024);
-      const uint64_t k_desc = make_smem_desc(smem_u32(smem + L::kK), 16, 1024);
-      const uint64_t v_desc = make_smem_desc(smem_u32(smem + L::kV), 16, 1024);
-      const uint64_t ds_desc = make_smem_desc(smem_u32(smem + L::kDS), 16, 1024);
-      const uint64_t k_mn = make_smem_desc(smem_u32(smem + L::kK), L::kRegion, 1024);
+      constexpr uint32_t idesc_nn = make_idesc_bf16(128, D, 1);                 // A from tensor memory (dS), B MN-major (K)
+      const uint64_t q_desc = make_smem_desc(smem_u32(smem + L::kFix0), 16, 1024);
+      const uint64_t do_desc = make_smem_desc(smem_u32(smem + L::kFix1), 16, 1024);
       bool ok = true;
-      mbar_arrive_expect_tx(&ctrl->q_full, 2 * L::kTileBytes);
-      for (int c = 0; c < L::kChunks; ++c) {
-        tma_load_3d(smem + L::kQ + c * L::kRegion, &tmap_q, &ctrl->q_full, c * 64, head0, q0);
-        tma_load_3d(smem + L::kDO + c * L::kRegion, &tmap_do, &ctrl->q_full, c * 64, head0, q0);
-      }
-      ok = mbar_wait(&ctrl->q_full, 0, abort_flag);
-      for (int it = 0; it < n_iter && ok; ++it) {
-        const int kr = kv0 + it * kTile;
-        if (it > 0) { ok = mbar_wait(&ctrl->acc_done, (it - 1) & 1, abort_flag); if (!ok) break; }   // K, V, dS free again
-        mbar_arrive_expect_tx(&ctrl->kv_full, 2 * L::kTileBytes);
+      auto load_walk = [&](int it) {                     // K and V tiles of iteration `it` into buffer it & 1
+        uint8_t *dst = smem + L::kWalk + (it & 1) * 2 * L::kTileBytes;
+        mbar_arrive_expect_tx(&ctrl->walk_full[it & 1], 2 * L::kTileBytes);
         for (int c = 0; c < L::kChunks; ++c) {
-          tma_load_3d(smem + L::kK + c * L::kRegion, &tmap_k, &ctrl->kv_full, c * 64, g, kr);
-          tma_load_3d(smem + L::kV + c * L::kRegion, &tmap_v, &ctrl->kv_full, c * 64, g, kr);
+          tma_load_3d(dst + c * L::kRegion, &tmap_k, &ctrl->walk_full[it & 1], c * 64, g, kv0 + it * kTile);
+          tma_load_3d(dst + L::kTileBytes + c * L::kRegion, &tmap_v, &ctrl->walk_full[it & 1], c * 64, g, kv0 + it * kTile);
         }
-        if (it + 1 < n_iter)
-          for (int c = 0; c < L::kChunks; ++c) {
-            tma_prefetch_3d(&tmap_k, c * 64, g, kr + kTile);
-            tma_prefetch_3d(&tmap_v, c * 64, g, kr + kTile);
-          }
-        ok = mbar_wait(&ctrl->kv_full, it & 1, abort_flag);
+      };
+      mbar_arrive_expect_tx(&ctrl->fix_full, 2 * L::kTileBytes);
+      for (int c = 0; c < L::kChunks; ++c) {
+        tma_load_3d(smem + L::kFix0 + c * L::kRegion, &tmap_q, &ctrl->fix_full, c * 64, head0, q0);
+        tma_load_3d(smem + L::kFix1 + c * L::kRegion, &tmap_do, &ctrl->fix_full, c * 64, head0, q0);
+      }
+      if (n_iter > 0) load_walk(0);
+      if (n_iter > 1) load_walk(1);
+      ok = mbar_wait(&ctrl->fix_full, 0, abort_flag);
+      for (int it = 0; it < n_iter && ok; ++it) {
+        const int bf = it & 1;
+        const uint32_t walk = smem_u32(smem + L::kWalk + bf * 2 * L::kTileBytes);
+        const uint64_t k_desc = make_smem_desc(walk, 16, 1024);
+        const uint64_t v_desc = make_smem_desc(walk + L::kTileBytes, 16, 1024);
+        const uint64_t k_mn = make_smem_desc(walk, L::kRegion, 1024);
+        ok = mbar_wait(&ctrl->walk_full[bf], (it >> 1) & 1, abort_flag);
         if (!ok) break;
         tc_fence_after();
 #pragma unroll
@@ -387,15 +429,17 @@ ba_bwd_dq_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
           mma_ss(tDP, do_desc + off, v_desc + off, idesc_nt, k > 0);
         }
         mma_commit(&ctrl->sd_full);
+        if (it > 0) {                                    // the previous iteration's K tile has been read: refill its buffer
+          ok = mbar_wait(&ctrl->acc_done, (it - 1) & 1, abort_flag);
+          if (!ok) break;
+          if (it + 1 < n_iter) load_walk(it + 1);
+        }
         ok = mbar_wait(&ctrl->rows_done, it & 1, abort_flag);
         if (!ok) break;
         tc_fence_after();
 #pragma unroll
-        for (int k = 0; k < kTile / 16; ++k) {           // contraction over the 128 keys of the tile
-          const uint64_t a_off = (uint64_t)(((k >> 2) * L::kRegion + (k & 3) * 32) >> 4);
-          const uint64_t b_off = (uint64_t)((k * 2048) >> 4);
-          mma_ss(tDQ, ds_desc + a_off, k_mn + b_off, idesc_nn, (it > 0 || k > 0) ? 1u : 0u);
-        }
+        for (int k = 0; k < kTile / 16; ++k)             // contraction over the 128 keys of the tile
+          mma_ts(tDQ, tDP + k * 8, k_mn + (uint64_t)((k * 2048) >> 4), idesc_nn, (it > 0 || k > 0) ? 1u : 0u);
         mma_commit(&ctrl->acc_done);
       }
     }
@@ -417,9 +461,8 @@ ba_bwd_dq_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
       ok = mbar_wait(&ctrl->sd_full, it & 1, abort_flag);
       if (!ok) break;
       tc_fence_after();
-      bwd_row(tS + lane_off, tDP + lane_off, nullptr, smem + L::kDS, r, n_ok, p.scale_log2, lse2, dl, p.scale);
+      bwd_row_ds(tS + lane_off, tDP + lane_off, n_ok, p.scale_log2, lse2, dl, p.scale);
       tc_fence_before();
-      fence_proxy_async();
       mbar_arrive(&ctrl->rows_done);
     }
     if (ok && n_iter > 0) ok = mbar_wait(&ctrl->acc_done, (n_iter - 1) & 1, abort_flag);
