@@ -16,8 +16,10 @@
 //     forward kernel) and walks over the key tiles it sees: S = Q K^T, dP = dO V^T (query rows on the
 //     lanes), dS written to tensor memory, dQ += dS K.
 // The tiles a CTA walks over (Q and dO there, K and V here) are double-buffered in shared memory, so the
-// loads of the next step run under the current one; within a step the two score products, the thread
-// work and the two (one) gradient products follow one another, because S and dP exist once in tensor memory.
+// loads of the next tile run under the current one.  Both kernels work in steps of 64 columns of S and dP with
+// two buffers of each in tensor memory (2 x 2 x 64 columns beside the accumulators): while the threads turn
+// one step's scores into P and dS, the tensor core forms the next step's scores and multiplies the previous
+// step's P and dS.
 #include <math.h>
 
 #include "ba_common.cuh"
@@ -60,7 +62,9 @@ struct BwdLayout {
 };
 
 struct BwdCtrl {
-  uint64_t fix_full, walk_full[2], sd_full, rows_done, acc_done;
+  uint64_t fix_full, walk_full[2], walk_free[2];
+  uint64_t sd_full[2], rows_done[2];     // per buffer of S / dP in tensor memory
+  uint64_t fin;                          // every product of the CTA has completed
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -84,14 +88,18 @@ __device__ __forceinline__ int upper_bound_dev(const int32_t *a, int n, int x) {
   return lo;
 }
 
-// dQ kernel, one query row (= lane) against a 128-key tile: reads the row of S and dP from tensor memory in
-// chunks of 32 columns, p = exp2(s * scale_log2 - lse_log2) where the mask allows, ds = p (dp - delta) scale,
-// and writes dS back over the dP columns as bf16 (two per column), the A operand of dQ += dS K.
+// The kernels work in steps of 64 columns of S and dP: tensor memory then holds two buffers of each next to the
+// accumulators, so the threads turn one step's scores into P / dS while the tensor core forms the next step's
+// scores and multiplies the previous step's P / dS.
+//
+// dQ kernel, one query row (= lane) against 64 keys: reads the row of S and dP from tensor memory in two chunks
+// of 32 columns, p = exp2(s * scale_log2 - lse_log2) where the mask allows, ds = p (dp - delta) scale, and writes
+// dS back over the dP columns as bf16 (two per column), the A operand of dQ += dS K.
 // `n_ok`: columns 0 .. n_ok - 1 are visible to this row (0: none).
 __device__ __forceinline__ void bwd_row_ds(uint32_t tS, uint32_t tDP, int n_ok, float scale_log2, float lse_log2,
                                            float delta, float scale) {
 #pragma unroll
-  for (int c = 0; c < 4; ++c) {
+  for (int c = 0; c < 2; ++c) {
     uint32_t s[32], dp[32];
     tmem_ld_32x32b_x32(tS + c * 32, s);
     tmem_ld_32x32b_x32(tDP + c * 32, dp);
@@ -114,14 +122,14 @@ __device__ __forceinline__ void bwd_row_ds(uint32_t tS, uint32_t tDP, int n_ok, 
   tmem_wait_st();
 }
 
-// dK/dV kernel, one key (= lane `j`) against the 128 query rows of a tile (= columns): S^T and dP^T come
-// from tensor memory in chunks of 32 columns; the per-row values (lse * log2 e, dO . O, number of keys of
-// this tile the row sees) are read from shared memory, the same address by every thread.  P^T goes back
-// over the S^T columns and dS^T over the dP^T columns as bf16.
+// dK/dV kernel, one key (= lane `j`) against 64 query rows of a tile (= columns): S^T and dP^T come from tensor
+// memory in two chunks of 32 columns; the per-row values (lse * log2 e, dO . O, number of keys of this tile the
+// row sees) are read from shared memory, the same address by every thread.  P^T goes back over the S^T
+// columns and dS^T over the dP^T columns as bf16.
 __device__ __forceinline__ void bwd_key_p_ds(uint32_t tST, uint32_t tDPT, int j, const float4 *stats,
                                              float scale_log2, float scale) {
 #pragma unroll
-  for (int c = 0; c < 4; ++c) {
+  for (int c = 0; c < 2; ++c) {
     uint32_t s[32], dp[32];
     tmem_ld_32x32b_x32(tST + c * 32, s);
     tmem_ld_32x32b_x32(tDPT + c * 32, dp);
@@ -222,8 +230,11 @@ ba_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
   };
 
   if (tid == 0) {
-    mbar_init(&ctrl->fix_full, 1); mbar_init(&ctrl->walk_full[0], 1); mbar_init(&ctrl->walk_full[1], 1);
-    mbar_init(&ctrl->sd_full, 1); mbar_init(&ctrl->rows_done, 128); mbar_init(&ctrl->acc_done, 1);
+    mbar_init(&ctrl->fix_full, 1); mbar_init(&ctrl->fin, 1);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&ctrl->walk_full[i], 1); mbar_init(&ctrl->walk_free[i], 1);
+      mbar_init(&ctrl->sd_full[i], 1); mbar_init(&ctrl->rows_done[i], 128);
+    }
     ctrl->abort_flag = 0;
     fence_barrier_init();
   }
@@ -233,16 +244,18 @@ ba_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
   tc_fence_after();
   const uint32_t tmem = ctrl->tmem_base;
   volatile int *abort_flag = &ctrl->abort_flag;
+  // tensor memory: S^T buffers at columns 0 and 64, dP^T buffers at 128 and 192 (64 query rows each), dV, dK
   const uint32_t tST = tmem, tDPT = tmem + 128, tDV = tmem + 256, tDK = tmem + 384;
+  const int n_steps = 2 * n_iter;                        // step i: query rows 64 (i & 1) .. + 63 of tile i >> 1
 
   if (warp == 4) {
     if (elect_one()) {
-      constexpr uint32_t idesc_nt = make_idesc_bf16(128, kTile, 0);             // both operands K-major
+      constexpr uint32_t idesc_nt = make_idesc_bf16(128, 64, 0);                // both operands K-major, 64 query rows
       constexpr uint32_t idesc_tn = make_idesc_bf16(128, D, 1);                 // A from tensor memory, B MN-major
       const uint64_t k_desc = make_smem_desc(smem_u32(smem + L::kFix0), 16, 1024);
       const uint64_t v_desc = make_smem_desc(smem_u32(smem + L::kFix1), 16, 1024);
       bool ok = true;
-      auto load_walk = [&](int it) {                     // Q and dO tiles of iteration `it` into buffer it & 1
+      auto load_walk = [&](int it) {                     // Q and dO tiles of tile `it` into buffer it & 1
         int row0, row_end, head0; bool causal;
         iter_rows(it, row0, row_end, causal, head0);
         uint8_t *dst = smem + L::kWalk + (it & 1) * 2 * L::kTileBytes;
@@ -252,6 +265,49 @@ ba_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
           tma_load_3d(dst + L::kTileBytes + c * L::kRegion, &tmap_do, &ctrl->walk_full[it & 1], c * 64, head0, row0);
         }
       };
+      // S^T = K Q^T and dP^T = V dO^T for the 64 query rows of step i.  They follow the gradient products of step
+      // i - 2 (same buffers) on the tensor pipe in issue order, so those have read P^T and dS^T before.
+      auto issue_scores = [&](int i) -> bool {
+        const int it = i >> 1, h = i & 1;
+        if (h == 0) {
+          if (!mbar_wait(&ctrl->walk_full[it & 1], (it >> 1) & 1, abort_flag)) return false;
+          tc_fence_after();
+        }
+        const uint32_t walk = smem_u32(smem + L::kWalk + (it & 1) * 2 * L::kTileBytes) + h * 64 * 128;   // rows 64 h ..
+        const uint64_t q_desc = make_smem_desc(walk, 16, 1024);
+        const uint64_t do_desc = make_smem_desc(walk + L::kTileBytes, 16, 1024);
+#pragma unroll
+        for (int k = 0; k < D / 16; ++k) {
+          const uint64_t off = (uint64_t)(((k >> 2) * L::kRegion + (k & 3) * 32) >> 4);
+          mma_ss(tST + (i & 1) * 64, k_desc + off, q_desc + off, idesc_nt, k > 0);
+        }
+#pragma unroll
+        for (int k = 0; k < D / 16; ++k) {
+          const uint64_t off = (uint64_t)(((k >> 2) * L::kRegion + (k & 3) * 32) >> 4);
+          mma_ss(tDPT + (i & 1) * 64, v_desc + off, do_desc + off, idesc_nt, k > 0);
+        }
+        mma_commit(&ctrl->sd_full[i & 1]);
+        return true;
+      };
+      // dV += P^T dO, dK += dS^T Q over the 64 query rows of step i (16 at a time)
+      auto issue_grads = [&](int i) -> bool {
+        const int it = i >> 1, h = i & 1;
+        if (!mbar_wait(&ctrl->rows_done[i & 1], (i >> 1) & 1, abort_flag)) return false;
+        tc_fence_after();
+        const uint32_t walk = smem_u32(smem + L::kWalk + (it & 1) * 2 * L::kTileBytes);
+        const uint64_t q_mn = make_smem_desc(walk, L::kRegion, 1024);
+        const uint64_t do_mn = make_smem_desc(walk + L::kTileBytes, L::kRegion, 1024);
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+          mma_ts(tDV, tST + (i & 1) * 64 + k * 8, do_mn + (uint64_t)(((h * 64 + k * 16) * 128) >> 4), idesc_tn,
+                 (i > 0 || k > 0) ? 1u : 0u);
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+          mma_ts(tDK, tDPT + (i & 1) * 64 + k * 8, q_mn + (uint64_t)(((h * 64 + k * 16) * 128) >> 4), idesc_tn,
+                 (i > 0 || k > 0) ? 1u : 0u);
+        if (h == 1) mma_commit(&ctrl->walk_free[it & 1]);   // the tile's Q and dO have been read for the last time
+        return true;
+      };
       mbar_arrive_expect_tx(&ctrl->fix_full, 2 * L::kTileBytes);
       for (int c = 0; c < L::kChunks; ++c) {
         tma_load_3d(smem + L::kFix0 + c * L::kRegion, &tmap_k, &ctrl->fix_full, c * 64, g, k0);
@@ -260,76 +316,55 @@ ba_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
       if (n_iter > 0) load_walk(0);
       if (n_iter > 1) load_walk(1);
       ok = mbar_wait(&ctrl->fix_full, 0, abort_flag);
-      for (int it = 0; it < n_iter && ok; ++it) {
-        const int bf = it & 1;
-        const uint32_t walk = smem_u32(smem + L::kWalk + bf * 2 * L::kTileBytes);
-        const uint64_t q_desc = make_smem_desc(walk, 16, 1024);
-        const uint64_t do_desc = make_smem_desc(walk + L::kTileBytes, 16, 1024);
-        const uint64_t q_mn = make_smem_desc(walk, L::kRegion, 1024);
-        const uint64_t do_mn = make_smem_desc(walk + L::kTileBytes, L::kRegion, 1024);
-        ok = mbar_wait(&ctrl->walk_full[bf], (it >> 1) & 1, abort_flag);
-        if (!ok) break;
-        tc_fence_after();
-        // S^T = K Q^T, dP^T = V dO^T (they follow the previous iteration's gradient products on the tensor
-        // pipe in issue order, so those have read P^T and dS^T before these overwrite the columns)
-#pragma unroll
-        for (int k = 0; k < D / 16; ++k) {
-          const uint64_t off = (uint64_t)(((k >> 2) * L::kRegion + (k & 3) * 32) >> 4);
-          mma_ss(tST, k_desc + off, q_desc + off, idesc_nt, k > 0);
+      int reload = -1;                                   // tile whose buffer is refilled once its products have completed
+      for (int i = 0; i <= n_steps && ok; ++i) {
+        if (i < n_steps) ok = issue_scores(i);
+        if (ok && reload >= 0) {
+          if (reload + 2 < n_iter) {
+            ok = mbar_wait(&ctrl->walk_free[reload & 1], (reload >> 1) & 1, abort_flag);
+            if (ok) load_walk(reload + 2);
+          }
+          reload = -1;
         }
-#pragma unroll
-        for (int k = 0; k < D / 16; ++k) {
-          const uint64_t off = (uint64_t)(((k >> 2) * L::kRegion + (k & 3) * 32) >> 4);
-          mma_ss(tDPT, v_desc + off, do_desc + off, idesc_nt, k > 0);
+        if (ok && i > 0) {
+          ok = issue_grads(i - 1);
+          if ((i - 1) & 1) reload = (i - 1) >> 1;
         }
-        mma_commit(&ctrl->sd_full);
-        // the previous iteration's gradient products have read its Q and dO: that buffer takes iteration it + 1
-        if (it > 0) {
-          ok = mbar_wait(&ctrl->acc_done, (it - 1) & 1, abort_flag);
-          if (!ok) break;
-          if (it + 1 < n_iter) load_walk(it + 1);
-        }
-        // the key threads turn S^T and dP^T into P^T and dS^T (bf16, in place)
-        ok = mbar_wait(&ctrl->rows_done, it & 1, abort_flag);
-        if (!ok) break;
-        tc_fence_after();
-#pragma unroll
-        for (int k = 0; k < kTile / 16; ++k)             // contraction over the 128 query rows, 16 at a time
-          mma_ts(tDV, tST + k * 8, do_mn + (uint64_t)((k * 2048) >> 4), idesc_tn, (it > 0 || k > 0) ? 1u : 0u);
-#pragma unroll
-        for (int k = 0; k < kTile / 16; ++k)
-          mma_ts(tDK, tDPT + k * 8, q_mn + (uint64_t)((k * 2048) >> 4), idesc_tn, (it > 0 || k > 0) ? 1u : 0u);
-        mma_commit(&ctrl->acc_done);
       }
+      if (ok) mma_commit(&ctrl->fin);
     }
   } else {
     const int j = tid;                                   // key of the tile = tensor-memory lane
     const uint32_t lane_off = (uint32_t)(warp * 32) << 16;
     float4 *stats = reinterpret_cast<float4 *>(smem + L::kStats);
     bool ok = true;
-    for (int it = 0; it < n_iter; ++it) {
-      // this thread also prepares what every key thread needs to know about query row `tid` of the tile
-      int row0, row_end, head0; bool causal;
-      iter_rows(it, row0, row_end, causal, head0);
-      const int tok_i = row0 + (tid >> p.hpt_log2);
-      const int head = head0 + (tid & (p.hpt - 1));
-      float4 st = make_float4(0.f, 0.f, __int_as_float(0), 0.f);
-      if (tok_i < row_end) {
-        st.x = __ldg(p.lse + (size_t)tok_i * p.Hq + head) * 1.4426950408889634f;
-        st.y = __ldg(p.delta + (size_t)tok_i * p.Hq + head);
-        st.z = __int_as_float(causal ? max(0, min(n_keys, tok_i - k0 + 1)) : n_keys);   // keys 0 .. z - 1 of the tile are visible
+    for (int i = 0; i < n_steps; ++i) {
+      const int it = i >> 1, h = i & 1;
+      if (h == 0) {
+        // this thread also prepares what every key thread needs to know about query row `tid` of the tile
+        int row0, row_end, head0; bool causal;
+        iter_rows(it, row0, row_end, causal, head0);
+        const int tok_i = row0 + (tid >> p.hpt_log2);
+        const int head = head0 + (tid & (p.hpt - 1));
+        float4 st = make_float4(0.f, 0.f, __int_as_float(0), 0.f);
+        if (tok_i < row_end) {
+          st.x = __ldg(p.lse + (size_t)tok_i * p.Hq + head) * 1.4426950408889634f;
+          st.y = __ldg(p.delta + (size_t)tok_i * p.Hq + head);
+          st.z = __int_as_float(causal ? max(0, min(n_keys, tok_i - k0 + 1)) : n_keys);   // keys 0 .. z - 1 of the tile are visible
+        }
+        stats[(it & 1) * 128 + tid] = st;
+        named_barrier_128();
       }
-      stats[(it & 1) * 128 + tid] = st;
-      named_barrier_128();
-      ok = mbar_wait(&ctrl->sd_full, it & 1, abort_flag);
+      ok = mbar_wait(&ctrl->sd_full[i & 1], (i >> 1) & 1, abort_flag);
       if (!ok) break;
       tc_fence_after();
-      bwd_key_p_ds(tST + lane_off, tDPT + lane_off, j, stats + (it & 1) * 128, p.scale_log2, p.scale);
+      bwd_key_p_ds(tST + (i & 1) * 64 + lane_off, tDPT + (i & 1) * 64 + lane_off, j, stats + (it & 1) * 128 + h * 64,
+                   p.scale_log2, p.scale);
       tc_fence_before();
-      mbar_arrive(&ctrl->rows_done);
+      mbar_arrive(&ctrl->rows_done[i & 1]);
     }
     // accumulators: lane = key row of the tile
-    if (ok && n_iter > 0) ok = mbar_wait(&ctrl->acc_done, (n_iter - 1) & 1, abort_flag);
+    if (ok && n_iter > 0) ok = mbar_wait(&ctrl->fin, 0, abort_flag);
     if (ok && n_iter > 0) {
       tc_fence_after();
       const bool valid = j < n_keys;
@@ -371,10 +406,14 @@ ba_bwd_dq_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
   const int kv0 = __ldg(sg.block_kv_begin + b);           // row i sees keys kv0 .. i
   const int head0 = blockIdx.y * p.hpt, g = head0 / p.G;
   const int n_iter = (q_end - kv0 + kTile - 1) / kTile;   // key tiles kv0 + 128 j
+  const int n_steps = (q_end - kv0 + 63) / 64;            // step i: keys kv0 + 64 i .. + 63 (half of tile i >> 1)
 
   if (tid == 0) {
-    mbar_init(&ctrl->fix_full, 1); mbar_init(&ctrl->walk_full[0], 1); mbar_init(&ctrl->walk_full[1], 1);
-    mbar_init(&ctrl->sd_full, 1); mbar_init(&ctrl->rows_done, 128); mbar_init(&ctrl->acc_done, 1);
+    mbar_init(&ctrl->fix_full, 1); mbar_init(&ctrl->fin, 1);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&ctrl->walk_full[i], 1); mbar_init(&ctrl->walk_free[i], 1);
+      mbar_init(&ctrl->sd_full[i], 1); mbar_init(&ctrl->rows_done[i], 128);
+    }
     ctrl->abort_flag = 0;
     fence_barrier_init();
   }
@@ -384,22 +423,57 @@ ba_bwd_dq_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
   tc_fence_after();
   const uint32_t tmem = ctrl->tmem_base;
   volatile int *abort_flag = &ctrl->abort_flag;
+  // tensor memory: S buffers at columns 0 and 64, dP buffers at 128 and 192 (64 keys each), dQ
   const uint32_t tS = tmem, tDP = tmem + 128, tDQ = tmem + 256;
 
   if (warp == 4) {
     if (elect_one()) {
-      constexpr uint32_t idesc_nt = make_idesc_bf16(128, kTile, 0);
+      constexpr uint32_t idesc_nt = make_idesc_bf16(128, 64, 0);
       constexpr uint32_t idesc_nn = make_idesc_bf16(128, D, 1);                 // A from tensor memory (dS), B MN-major (K)
       const uint64_t q_desc = make_smem_desc(smem_u32(smem + L::kFix0), 16, 1024);
       const uint64_t do_desc = make_smem_desc(smem_u32(smem + L::kFix1), 16, 1024);
       bool ok = true;
-      auto load_walk = [&](int it) {                     // K and V tiles of iteration `it` into buffer it & 1
+      auto load_walk = [&](int it) {                     // K and V tiles of key tile `it` into buffer it & 1
         uint8_t *dst = smem + L::kWalk + (it & 1) * 2 * L::kTileBytes;
         mbar_arrive_expect_tx(&ctrl->walk_full[it & 1], 2 * L::kTileBytes);
         for (int c = 0; c < L::kChunks; ++c) {
           tma_load_3d(dst + c * L::kRegion, &tmap_k, &ctrl->walk_full[it & 1], c * 64, g, kv0 + it * kTile);
           tma_load_3d(dst + L::kTileBytes + c * L::kRegion, &tmap_v, &ctrl->walk_full[it & 1], c * 64, g, kv0 + it * kTile);
         }
+      };
+      auto issue_scores = [&](int i) -> bool {           // S = Q K^T, dP = dO V^T for the 64 keys of step i
+        const int it = i >> 1, h = i & 1;
+        if (h == 0) {
+          if (!mbar_wait(&ctrl->walk_full[it & 1], (it >> 1) & 1, abort_flag)) return false;
+          tc_fence_after();
+        }
+        const uint32_t walk = smem_u32(smem + L::kWalk + (it & 1) * 2 * L::kTileBytes) + h * 64 * 128;   // keys 64 h ..
+        const uint64_t k_desc = make_smem_desc(walk, 16, 1024);
+        const uint64_t v_desc = make_smem_desc(walk + L::kTileBytes, 16, 1024);
+#pragma unroll
+        for (int k = 0; k < D / 16; ++k) {
+          const uint64_t off = (uint64_t)(((k >> 2) * L::kRegion + (k & 3) * 32) >> 4);
+          mma_ss(tS + (i & 1) * 64, q_desc + off, k_desc + off, idesc_nt, k > 0);
+        }
+#pragma unroll
+        for (int k = 0; k < D / 16; ++k) {
+          const uint64_t off = (uint64_t)(((k >> 2) * L::kRegion + (k & 3) * 32) >> 4);
+          mma_ss(tDP + (i & 1) * 64, do_desc + off, v_desc + off, idesc_nt, k > 0);
+        }
+        mma_commit(&ctrl->sd_full[i & 1]);
+        return true;
+      };
+      auto issue_grads = [&](int i) -> bool {            // dQ += dS K over the 64 keys of step i (16 at a time)
+        const int it = i >> 1, h = i & 1;
+        if (!mbar_wait(&ctrl->rows_done[i & 1], (i >> 1) & 1, abort_flag)) return false;
+        tc_fence_after();
+        const uint64_t k_mn = make_smem_desc(smem_u32(smem + L::kWalk + (it & 1) * 2 * L::kTileBytes), L::kRegion, 1024);
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+          mma_ts(tDQ, tDP + (i & 1) * 64 + k * 8, k_mn + (uint64_t)(((h * 64 + k * 16) * 128) >> 4), idesc_nn,
+                 (i > 0 || k > 0) ? 1u : 0u);
+        if (h == 1 || i + 1 == n_steps) mma_commit(&ctrl->walk_free[it & 1]);   // last use of the tile's K and V
+        return true;
       };
       mbar_arrive_expect_tx(&ctrl->fix_full, 2 * L::kTileBytes);
       for (int c = 0; c < L::kChunks; ++c) {
@@ -409,39 +483,22 @@ ba_bwd_dq_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
       if (n_iter > 0) load_walk(0);
       if (n_iter > 1) load_walk(1);
       ok = mbar_wait(&ctrl->fix_full, 0, abort_flag);
-      for (int it = 0; it < n_iter && ok; ++it) {
-        const int bf = it & 1;
-        const uint32_t walk = smem_u32(smem + L::kWalk + bf * 2 * L::kTileBytes);
-        const uint64_t k_desc = make_smem_desc(walk, 16, 1024);
-        const uint64_t v_desc = make_smem_desc(walk + L::kTileBytes, 16, 1024);
-        const uint64_t k_mn = make_smem_desc(walk, L::kRegion, 1024);
-        ok = mbar_wait(&ctrl->walk_full[bf], (it >> 1) & 1, abort_flag);
-        if (!ok) break;
-        tc_fence_after();
-#pragma unroll
-        for (int k = 0; k < D / 16; ++k) {
-          const uint64_t off = (uint64_t)(((k >> 2) * L::kRegion + (k & 3) * 32) >> 4);
-          mma_ss(tS, q_desc + off, k_desc + off, idesc_nt, k > 0);
+      int reload = -1;                                   // key tile whose buffer is refilled once its products have completed
+      for (int i = 0; i <= n_steps && ok; ++i) {
+        if (i < n_steps) ok = issue_scores(i);
+        if (ok && reload >= 0) {
+          if (reload + 2 < n_iter) {
+            ok = mbar_wait(&ctrl->walk_free[reload & 1], (reload >> 1) & 1, abort_flag);
+            if (ok) load_walk(reload + 2);
+          }
+          reload = -1;
         }
-#pragma unroll
-        for (int k = 0; k < D / 16; ++k) {
-          const uint64_t off = (uint64_t)(((k >> 2) * L::kRegion + (k & 3) * 32) >> 4);
-          mma_ss(tDP, do_desc + off, v_desc + off, idesc_nt, k > 0);
+        if (ok && i > 0) {
+          ok = issue_grads(i - 1);
+          if ((i - 1) & 1) reload = (i - 1) >> 1;
         }
-        mma_commit(&ctrl->sd_full);
-        if (it > 0) {                                    // the previous iteration's K tile has been read: refill its buffer
-          ok = mbar_wait(&ctrl->acc_done, (it - 1) & 1, abort_flag);
-          if (!ok) break;
-          if (it + 1 < n_iter) load_walk(it + 1);
-        }
-        ok = mbar_wait(&ctrl->rows_done, it & 1, abort_flag);
-        if (!ok) break;
-        tc_fence_after();
-#pragma unroll
-        for (int k = 0; k < kTile / 16; ++k)             // contraction over the 128 keys of the tile
-          mma_ts(tDQ, tDP + k * 8, k_mn + (uint64_t)((k * 2048) >> 4), idesc_nn, (it > 0 || k > 0) ? 1u : 0u);
-        mma_commit(&ctrl->acc_done);
       }
+      if (ok) mma_commit(&ctrl->fin);
     }
   } else {
     const int r = tid;
@@ -455,18 +512,18 @@ ba_bwd_dq_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
       dl = __ldg(p.delta + (size_t)tok_i * p.Hq + head);
     }
     bool ok = true;
-    for (int it = 0; it < n_iter; ++it) {
-      const int kr = kv0 + it * kTile;
-      const int n_ok = row_ok ? max(0, min(kTile, tok_i - kr + 1)) : 0;
-      ok = mbar_wait(&ctrl->sd_full, it & 1, abort_flag);
+    for (int i = 0; i < n_steps; ++i) {
+      const int kr = kv0 + i * 64;
+      const int n_ok = row_ok ? max(0, min(64, tok_i - kr + 1)) : 0;
+      ok = mbar_wait(&ctrl->sd_full[i & 1], (i >> 1) & 1, abort_flag);
       if (!ok) break;
       tc_fence_after();
-      bwd_row_ds(tS + lane_off, tDP + lane_off, n_ok, p.scale_log2, lse2, dl, p.scale);
+      bwd_row_ds(tS + (i & 1) * 64 + lane_off, tDP + (i & 1) * 64 + lane_off, n_ok, p.scale_log2, lse2, dl, p.scale);
       tc_fence_before();
-      mbar_arrive(&ctrl->rows_done);
+      mbar_arrive(&ctrl->rows_done[i & 1]);
     }
-    if (ok && n_iter > 0) ok = mbar_wait(&ctrl->acc_done, (n_iter - 1) & 1, abort_flag);
-    if (ok && n_iter > 0) {
+    if (ok && n_steps > 0) ok = mbar_wait(&ctrl->fin, 0, abort_flag);
+    if (ok && n_steps > 0) {
       tc_fence_after();
       store_acc_row<D>(tDQ + lane_off, p.dq, ((size_t)tok_i * p.Hq + head) * D, p.out_f32, row_ok);
     }
