@@ -31,7 +31,12 @@ int ba_heads_per_tile(const ba_config &c);
 
 namespace {
 
-constexpr int kBwdThreads = 160;      // warps 0-3: one thread per tile row (tensor-memory lane); warp 4: loads and MMA issue
+// warps 0-7: two threads per tile row (tensor-memory lane = tid & 127), warps w and w + 4 share a lane quarter and
+// take one half of every step's 64 columns each, so that every SM sub-partition has two warps to hide the
+// latency of tensor-memory loads, shared-memory reads and exponentials; warp 8: loads and MMA issue
+constexpr int kBwdThreads = 288;
+constexpr int kRowThreads = 256;
+constexpr int kCtlWarp = 8;
 constexpr int kTile = 128;
 
 struct BwdParams {
@@ -77,7 +82,7 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16
         "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
       : "memory");
 }
-__device__ __forceinline__ void named_barrier_128() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+__device__ __forceinline__ void named_barrier_rows() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
 
 __device__ __forceinline__ int upper_bound_dev(const int32_t *a, int n, int x) {
   int lo = 0, hi = n;
@@ -93,13 +98,12 @@ __device__ __forceinline__ int upper_bound_dev(const int32_t *a, int n, int x) {
 // scores and multiplies the previous step's P / dS.
 //
 // dQ kernel, one query row (= lane) against 64 keys: reads the row of S and dP from tensor memory in two chunks
-// of 32 columns, p = exp2(s * scale_log2 - lse_log2) where the mask allows, ds = p (dp - delta) scale, and writes
+// of 32 columns (one per thread of the row), p = exp2(s * scale_log2 - lse_log2) where the mask allows, ds = p (dp - delta) scale, and writes
 // dS back over the dP columns as bf16 (two per column), the A operand of dQ += dS K.
-// `n_ok`: columns 0 .. n_ok - 1 are visible to this row (0: none).
-__device__ __forceinline__ void bwd_row_ds(uint32_t tS, uint32_t tDP, int n_ok, float scale_log2, float lse_log2,
+// `n_ok`: columns 0 .. n_ok - 1 of the step are visible to this row (0: none); the thread takes chunk `c` (0 or 1).
+__device__ __forceinline__ void bwd_row_ds(uint32_t tS, uint32_t tDP, int c, int n_ok, float scale_log2, float lse_log2,
                                            float delta, float scale) {
-#pragma unroll
-  for (int c = 0; c < 2; ++c) {
+  {
     uint32_t s[32], dp[32];
     tmem_ld_32x32b_x32(tS + c * 32, s);
     tmem_ld_32x32b_x32(tDP + c * 32, dp);
@@ -117,19 +121,19 @@ __device__ __forceinline__ void bwd_row_ds(uint32_t tS, uint32_t tDP, int n_ok, 
       __nv_bfloat162 dv = __floats2bfloat162_rn(d0, d1);
       dw[i] = *reinterpret_cast<uint32_t *>(&dv);
     }
-    tmem_st16(tDP + c * 16, dw);         // columns 16 c .. 16 c + 15: inside the part of dP already read
+    tmem_st16(tDP + c * 32, dw);         // over the first 16 of the 32 columns this thread has just read
   }
   tmem_wait_st();
 }
 
 // dK/dV kernel, one key (= lane `j`) against 64 query rows of a tile (= columns): S^T and dP^T come from tensor
-// memory in two chunks of 32 columns; the per-row values (lse * log2 e, dO . O, number of keys of this tile the
+// memory in two chunks of 32 columns (one per thread of the key); the per-row values (lse * log2 e, dO . O, number of keys of this tile the
 // row sees) are read from shared memory, the same address by every thread.  P^T goes back over the S^T
-// columns and dS^T over the dP^T columns as bf16.
-__device__ __forceinline__ void bwd_key_p_ds(uint32_t tST, uint32_t tDPT, int j, const float4 *stats,
+// columns and dS^T over the dP^T columns as bf16 -- each thread over columns it has read itself, because the other
+// thread of the lane works on its own 32 columns at its own pace.
+__device__ __forceinline__ void bwd_key_p_ds(uint32_t tST, uint32_t tDPT, int c, int j, const float4 *stats,
                                              float scale_log2, float scale) {
-#pragma unroll
-  for (int c = 0; c < 2; ++c) {
+  {
     uint32_t s[32], dp[32];
     tmem_ld_32x32b_x32(tST + c * 32, s);
     tmem_ld_32x32b_x32(tDPT + c * 32, dp);
@@ -148,17 +152,20 @@ __device__ __forceinline__ void bwd_key_p_ds(uint32_t tST, uint32_t tDPT, int j,
       pw[i] = *reinterpret_cast<uint32_t *>(&pv);
       dw[i] = *reinterpret_cast<uint32_t *>(&dv);
     }
-    tmem_st16(tST + c * 16, pw);
-    tmem_st16(tDPT + c * 16, dw);
+    tmem_st16(tST + c * 32, pw);         // over the first 16 of the 32 columns this thread has just read
+    tmem_st16(tDPT + c * 32, dw);
   }
   tmem_wait_st();
 }
 
 // Writes one accumulator row (D fp32 columns of tensor memory, lane = row) to global memory.
+// The two threads of a row take alternate chunks of 32 columns (`half` = 0 or 1).
 template <int D>
-__device__ __forceinline__ void store_acc_row(uint32_t tAcc, void *dst_base, size_t elem_off, int out_f32, bool valid) {
+__device__ __forceinline__ void store_acc_row(uint32_t tAcc, void *dst_base, size_t elem_off, int out_f32, bool valid,
+                                              int half) {
 #pragma unroll
-  for (int c = 0; c < D / 32; ++c) {
+  for (int cc = 0; cc < D / 64; ++cc) {
+    const int c = 2 * cc + half;
     uint32_t a[32];
     tmem_ld_32x32b_x32(tAcc + c * 32, a);
     tmem_wait_ld();
@@ -233,12 +240,12 @@ ba_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
     mbar_init(&ctrl->fix_full, 1); mbar_init(&ctrl->fin, 1);
     for (int i = 0; i < 2; ++i) {
       mbar_init(&ctrl->walk_full[i], 1); mbar_init(&ctrl->walk_free[i], 1);
-      mbar_init(&ctrl->sd_full[i], 1); mbar_init(&ctrl->rows_done[i], 128);
+      mbar_init(&ctrl->sd_full[i], 1); mbar_init(&ctrl->rows_done[i], kRowThreads);
     }
     ctrl->abort_flag = 0;
     fence_barrier_init();
   }
-  if (warp == 4) { tmem_alloc(&ctrl->tmem_base, 512); tmem_relinquish(); }
+  if (warp == kCtlWarp) { tmem_alloc(&ctrl->tmem_base, 512); tmem_relinquish(); }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -248,7 +255,7 @@ ba_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
   const uint32_t tST = tmem, tDPT = tmem + 128, tDV = tmem + 256, tDK = tmem + 384;
   const int n_steps = 2 * n_iter;                        // step i: query rows 64 (i & 1) .. + 63 of tile i >> 1
 
-  if (warp == 4) {
+  if (warp == kCtlWarp) {
     if (elect_one()) {
       constexpr uint32_t idesc_nt = make_idesc_bf16(128, 64, 0);                // both operands K-major, 64 query rows
       constexpr uint32_t idesc_tn = make_idesc_bf16(128, D, 1);                 // A from tensor memory, B MN-major
@@ -299,11 +306,11 @@ ba_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
         const uint64_t do_mn = make_smem_desc(walk + L::kTileBytes, L::kRegion, 1024);
 #pragma unroll
         for (int k = 0; k < 4; ++k)
-          mma_ts(tDV, tST + (i & 1) * 64 + k * 8, do_mn + (uint64_t)(((h * 64 + k * 16) * 128) >> 4), idesc_tn,
+          mma_ts(tDV, tST + (i & 1) * 64 + (k >> 1) * 32 + (k & 1) * 8, do_mn + (uint64_t)(((h * 64 + k * 16) * 128) >> 4), idesc_tn,
                  (i > 0 || k > 0) ? 1u : 0u);
 #pragma unroll
         for (int k = 0; k < 4; ++k)
-          mma_ts(tDK, tDPT + (i & 1) * 64 + k * 8, q_mn + (uint64_t)(((h * 64 + k * 16) * 128) >> 4), idesc_tn,
+          mma_ts(tDK, tDPT + (i & 1) * 64 + (k >> 1) * 32 + (k & 1) * 8, q_mn + (uint64_t)(((h * 64 + k * 16) * 128) >> 4), idesc_tn,
                  (i > 0 || k > 0) ? 1u : 0u);
         if (h == 1) mma_commit(&ctrl->walk_free[it & 1]);   // the tile's Q and dO have been read for the last time
         return true;
@@ -334,31 +341,34 @@ ba_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
       if (ok) mma_commit(&ctrl->fin);
     }
   } else {
-    const int j = tid;                                   // key of the tile = tensor-memory lane
-    const uint32_t lane_off = (uint32_t)(warp * 32) << 16;
+    const int j = tid & 127;                             // key of the tile = tensor-memory lane
+    const int ch = tid >> 7;                             // which 32 of a step's 64 columns this thread takes
+    const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
     float4 *stats = reinterpret_cast<float4 *>(smem + L::kStats);
     bool ok = true;
     for (int i = 0; i < n_steps; ++i) {
       const int it = i >> 1, h = i & 1;
       if (h == 0) {
         // this thread also prepares what every key thread needs to know about query row `tid` of the tile
-        int row0, row_end, head0; bool causal;
-        iter_rows(it, row0, row_end, causal, head0);
-        const int tok_i = row0 + (tid >> p.hpt_log2);
-        const int head = head0 + (tid & (p.hpt - 1));
-        float4 st = make_float4(0.f, 0.f, __int_as_float(0), 0.f);
-        if (tok_i < row_end) {
-          st.x = __ldg(p.lse + (size_t)tok_i * p.Hq + head) * 1.4426950408889634f;
-          st.y = __ldg(p.delta + (size_t)tok_i * p.Hq + head);
-          st.z = __int_as_float(causal ? max(0, min(n_keys, tok_i - k0 + 1)) : n_keys);   // keys 0 .. z - 1 of the tile are visible
+        if (tid < 128) {
+          int row0, row_end, head0; bool causal;
+          iter_rows(it, row0, row_end, causal, head0);
+          const int tok_i = row0 + (tid >> p.hpt_log2);
+          const int head = head0 + (tid & (p.hpt - 1));
+          float4 st = make_float4(0.f, 0.f, __int_as_float(0), 0.f);
+          if (tok_i < row_end) {
+            st.x = __ldg(p.lse + (size_t)tok_i * p.Hq + head) * 1.4426950408889634f;
+            st.y = __ldg(p.delta + (size_t)tok_i * p.Hq + head);
+            st.z = __int_as_float(causal ? max(0, min(n_keys, tok_i - k0 + 1)) : n_keys);   // keys 0 .. z - 1 of the tile are visible
+          }
+          stats[(it & 1) * 128 + tid] = st;
         }
-        stats[(it & 1) * 128 + tid] = st;
-        named_barrier_128();
+        named_barrier_rows();
       }
       ok = mbar_wait(&ctrl->sd_full[i & 1], (i >> 1) & 1, abort_flag);
       if (!ok) break;
       tc_fence_after();
-      bwd_key_p_ds(tST + (i & 1) * 64 + lane_off, tDPT + (i & 1) * 64 + lane_off, j, stats + (it & 1) * 128 + h * 64,
+      bwd_key_p_ds(tST + (i & 1) * 64 + lane_off, tDPT + (i & 1) * 64 + lane_off, ch, j, stats + (it & 1) * 128 + h * 64,
                    p.scale_log2, p.scale);
       tc_fence_before();
       mbar_arrive(&ctrl->rows_done[i & 1]);
@@ -369,14 +379,14 @@ ba_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
       tc_fence_after();
       const bool valid = j < n_keys;
       const size_t off = ((size_t)(k0 + j) * p.Hkv + g) * D;
-      store_acc_row<D>(tDV + lane_off, p.dv, off, p.out_f32, valid);
-      store_acc_row<D>(tDK + lane_off, p.dk, off, p.out_f32, valid);
+      store_acc_row<D>(tDV + lane_off, p.dv, off, p.out_f32, valid, ch);
+      store_acc_row<D>(tDK + lane_off, p.dk, off, p.out_f32, valid, ch);
     }
   }
   tc_fence_before();
   __syncthreads();
   if (tid == 0 && ctrl->abort_flag) ba_record_status(p.status, BA_ERR_TIMEOUT);
-  if (warp == 4) tmem_dealloc(tmem, 512);
+  if (warp == kCtlWarp) tmem_dealloc(tmem, 512);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -412,12 +422,12 @@ ba_bwd_dq_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
     mbar_init(&ctrl->fix_full, 1); mbar_init(&ctrl->fin, 1);
     for (int i = 0; i < 2; ++i) {
       mbar_init(&ctrl->walk_full[i], 1); mbar_init(&ctrl->walk_free[i], 1);
-      mbar_init(&ctrl->sd_full[i], 1); mbar_init(&ctrl->rows_done[i], 128);
+      mbar_init(&ctrl->sd_full[i], 1); mbar_init(&ctrl->rows_done[i], kRowThreads);
     }
     ctrl->abort_flag = 0;
     fence_barrier_init();
   }
-  if (warp == 4) { tmem_alloc(&ctrl->tmem_base, 512); tmem_relinquish(); }
+  if (warp == kCtlWarp) { tmem_alloc(&ctrl->tmem_base, 512); tmem_relinquish(); }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -426,7 +436,7 @@ ba_bwd_dq_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
   // tensor memory: S buffers at columns 0 and 64, dP buffers at 128 and 192 (64 keys each), dQ
   const uint32_t tS = tmem, tDP = tmem + 128, tDQ = tmem + 256;
 
-  if (warp == 4) {
+  if (warp == kCtlWarp) {
     if (elect_one()) {
       constexpr uint32_t idesc_nt = make_idesc_bf16(128, 64, 0);
       constexpr uint32_t idesc_nn = make_idesc_bf16(128, D, 1);                 // A from tensor memory (dS), B MN-major (K)
@@ -470,7 +480,7 @@ ba_bwd_dq_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
         const uint64_t k_mn = make_smem_desc(smem_u32(smem + L::kWalk + (it & 1) * 2 * L::kTileBytes), L::kRegion, 1024);
 #pragma unroll
         for (int k = 0; k < 4; ++k)
-          mma_ts(tDQ, tDP + (i & 1) * 64 + k * 8, k_mn + (uint64_t)(((h * 64 + k * 16) * 128) >> 4), idesc_nn,
+          mma_ts(tDQ, tDP + (i & 1) * 64 + (k >> 1) * 32 + (k & 1) * 8, k_mn + (uint64_t)(((h * 64 + k * 16) * 128) >> 4), idesc_nn,
                  (i > 0 || k > 0) ? 1u : 0u);
         if (h == 1 || i + 1 == n_steps) mma_commit(&ctrl->walk_free[it & 1]);   // last use of the tile's K and V
         return true;
@@ -501,8 +511,9 @@ ba_bwd_dq_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
       if (ok) mma_commit(&ctrl->fin);
     }
   } else {
-    const int r = tid;
-    const uint32_t lane_off = (uint32_t)(warp * 32) << 16;
+    const int r = tid & 127;                             // row of the query tile = tensor-memory lane
+    const int ch = tid >> 7;                             // which 32 of a step's 64 columns this thread takes
+    const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
     const int tok_i = q0 + (r >> p.hpt_log2);
     const int head = head0 + (r & (p.hpt - 1));
     const bool row_ok = tok_i < q_end;
@@ -518,20 +529,20 @@ ba_bwd_dq_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
       ok = mbar_wait(&ctrl->sd_full[i & 1], (i >> 1) & 1, abort_flag);
       if (!ok) break;
       tc_fence_after();
-      bwd_row_ds(tS + (i & 1) * 64 + lane_off, tDP + (i & 1) * 64 + lane_off, n_ok, p.scale_log2, lse2, dl, p.scale);
+      bwd_row_ds(tS + (i & 1) * 64 + lane_off, tDP + (i & 1) * 64 + lane_off, ch, n_ok, p.scale_log2, lse2, dl, p.scale);
       tc_fence_before();
       mbar_arrive(&ctrl->rows_done[i & 1]);
     }
     if (ok && n_steps > 0) ok = mbar_wait(&ctrl->fin, 0, abort_flag);
     if (ok && n_steps > 0) {
       tc_fence_after();
-      store_acc_row<D>(tDQ + lane_off, p.dq, ((size_t)tok_i * p.Hq + head) * D, p.out_f32, row_ok);
+      store_acc_row<D>(tDQ + lane_off, p.dq, ((size_t)tok_i * p.Hq + head) * D, p.out_f32, row_ok, ch);
     }
   }
   tc_fence_before();
   __syncthreads();
   if (tid == 0 && ctrl->abort_flag) ba_record_status(p.status, BA_ERR_TIMEOUT);
-  if (warp == 4) tmem_dealloc(tmem, 512);
+  if (warp == kCtlWarp) tmem_dealloc(tmem, 512);
 }
 
 // delta[row, head] = dO . O
