@@ -61,7 +61,7 @@ struct BwdLayout {
   // buffers of two tiles each for the ones it walks over
   static constexpr int kFix0 = 0, kFix1 = kTileBytes;
   static constexpr int kWalk = 2 * kTileBytes;            // buffer b: tiles at kWalk + b * 2 * kTileBytes, + kTileBytes
-  static constexpr int kStats = 6 * kTileBytes;           // dK/dV kernel: per query row {lse * log2 e, dO . O, visible keys, -}, two buffers
+  static constexpr int kStats = 6 * kTileBytes;           // dK/dV kernel: per query row lse * log2 e, dO . O * scale, visible keys; two buffers of each
   static constexpr int kCtrl = kStats + 2 * 128 * 16;
   static constexpr int kBytes = kCtrl + 256;
 };
@@ -97,64 +97,93 @@ __device__ __forceinline__ int upper_bound_dev(const int32_t *a, int n, int x) {
 // accumulators, so the threads turn one step's scores into P / dS while the tensor core forms the next step's
 // scores and multiplies the previous step's P / dS.
 //
-// dQ kernel, one query row (= lane) against 64 keys: reads the row of S and dP from tensor memory in two chunks
-// of 32 columns (one per thread of the row), p = exp2(s * scale_log2 - lse_log2) where the mask allows, ds = p (dp - delta) scale, and writes
-// dS back over the dP columns as bf16 (two per column), the A operand of dQ += dS K.
-// `n_ok`: columns 0 .. n_ok - 1 of the step are visible to this row (0: none); the thread takes chunk `c` (0 or 1).
+__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+
+// The arithmetic of both helpers is packed fp32x2: for a pair of columns, x = s * scale_log2 - lse_log2 (one FMA),
+// p = exp2(x) (two), t = dp * scale - delta * scale (one FMA), ds = p * t (one multiply).  kMasked = false is for
+// steps in which every (row, key) pair is visible: no comparison at all.
+//
+// dQ kernel, one query row (= lane) against 64 keys: the thread takes chunk `c` (32 columns) of the step's S and
+// dP and writes dS back over the first 16 dP columns it has read, as bf16 (two per column): the A operand of
+// dQ += dS K.  `n_ok`: columns 0 .. n_ok - 1 of the step are visible to this row (0: none).
+template <bool kMasked>
 __device__ __forceinline__ void bwd_row_ds(uint32_t tS, uint32_t tDP, int c, int n_ok, float scale_log2, float lse_log2,
-                                           float delta, float scale) {
-  {
-    uint32_t s[32], dp[32];
-    tmem_ld_32x32b_x32(tS + c * 32, s);
-    tmem_ld_32x32b_x32(tDP + c * 32, dp);
-    tmem_wait_ld();
-    uint32_t dw[16];
+                                           float delta_scaled, float scale) {
+  uint32_t s[32], dp[32];
+  tmem_ld_32x32b_x32(tS + c * 32, s);
+  tmem_ld_32x32b_x32(tDP + c * 32, dp);
+  tmem_wait_ld();
+  const uint64_t sl2 = pack2(scale_log2, scale_log2), nl2 = pack2(-lse_log2, -lse_log2);
+  const uint64_t sc2 = pack2(scale, scale), nd2 = pack2(-delta_scaled, -delta_scaled);
+  uint32_t dw[16];
 #pragma unroll
-    for (int i = 0; i < 16; ++i) {
+  for (int i = 0; i < 16; ++i) {
+    const uint64_t x2 = fma2(pack2(__uint_as_float(s[2 * i]), __uint_as_float(s[2 * i + 1])), sl2, nl2);
+    float x0, x1;
+    unpack2(x2, x0, x1);
+    float p0 = ex2(x0), p1 = ex2(x1);
+    if (kMasked) {
       const int e0 = c * 32 + 2 * i;
-      float p0 = ex2(fmaf(__uint_as_float(s[2 * i]), scale_log2, -lse_log2));
-      float p1 = ex2(fmaf(__uint_as_float(s[2 * i + 1]), scale_log2, -lse_log2));
       if (e0 >= n_ok) p0 = 0.f;
       if (e0 + 1 >= n_ok) p1 = 0.f;
-      const float d0 = p0 * (__uint_as_float(dp[2 * i]) - delta) * scale;
-      const float d1 = p1 * (__uint_as_float(dp[2 * i + 1]) - delta) * scale;
-      __nv_bfloat162 dv = __floats2bfloat162_rn(d0, d1);
-      dw[i] = *reinterpret_cast<uint32_t *>(&dv);
     }
-    tmem_st16(tDP + c * 32, dw);         // over the first 16 of the 32 columns this thread has just read
+    const uint64_t t2 = fma2(pack2(__uint_as_float(dp[2 * i]), __uint_as_float(dp[2 * i + 1])), sc2, nd2);
+    float d0, d1;
+    unpack2(mul2(pack2(p0, p1), t2), d0, d1);
+    __nv_bfloat162 dv = __floats2bfloat162_rn(d0, d1);
+    dw[i] = *reinterpret_cast<uint32_t *>(&dv);
   }
+  tmem_st16(tDP + c * 32, dw);
   tmem_wait_st();
 }
 
-// dK/dV kernel, one key (= lane `j`) against 64 query rows of a tile (= columns): S^T and dP^T come from tensor
-// memory in two chunks of 32 columns (one per thread of the key); the per-row values (lse * log2 e, dO . O, number of keys of this tile the
-// row sees) are read from shared memory, the same address by every thread.  P^T goes back over the S^T
-// columns and dS^T over the dP^T columns as bf16 -- each thread over columns it has read itself, because the other
-// thread of the lane works on its own 32 columns at its own pace.
-__device__ __forceinline__ void bwd_key_p_ds(uint32_t tST, uint32_t tDPT, int c, int j, const float4 *stats,
-                                             float scale_log2, float scale) {
-  {
-    uint32_t s[32], dp[32];
-    tmem_ld_32x32b_x32(tST + c * 32, s);
-    tmem_ld_32x32b_x32(tDPT + c * 32, dp);
-    tmem_wait_ld();
-    uint32_t pw[16], dw[16];
+// dK/dV kernel, one key (= lane `j`) against 64 query rows of a tile (= columns): the thread takes chunk `c`
+// (32 columns) of the step's S^T and dP^T; the per-row values -- lse * log2 e, dO . O * scale, and the number of
+// keys of this tile the row sees -- are read from shared memory, the same address by every thread.  P^T goes back
+// over the S^T columns and dS^T over the dP^T columns as bf16 -- each thread over columns it has read itself,
+// because the other thread of the lane works on its own 32 columns at its own pace.
+template <bool kMasked>
+__device__ __forceinline__ void bwd_key_p_ds(uint32_t tST, uint32_t tDPT, int c, int j, const float *lse2, const float *dls,
+                                             const int *lim, float scale_log2, float scale) {
+  uint32_t s[32], dp[32];
+  tmem_ld_32x32b_x32(tST + c * 32, s);
+  tmem_ld_32x32b_x32(tDPT + c * 32, dp);
+  tmem_wait_ld();
+  const uint64_t sl2 = pack2(scale_log2, scale_log2), sc2 = pack2(scale, scale);
+  uint32_t pw[16], dw[16];
 #pragma unroll
-    for (int i = 0; i < 16; ++i) {
-      const float4 a = stats[c * 32 + 2 * i], b = stats[c * 32 + 2 * i + 1];
-      float p0 = ex2(fmaf(__uint_as_float(s[2 * i]), scale_log2, -a.x));
-      float p1 = ex2(fmaf(__uint_as_float(s[2 * i + 1]), scale_log2, -b.x));
-      if (j >= __float_as_int(a.z)) p0 = 0.f;
-      if (j >= __float_as_int(b.z)) p1 = 0.f;
-      const float d0 = p0 * (__uint_as_float(dp[2 * i]) - a.y) * scale;
-      const float d1 = p1 * (__uint_as_float(dp[2 * i + 1]) - b.y) * scale;
+  for (int q = 0; q < 8; ++q) {                          // four columns at a time: one 16-byte read of each per-row array
+    const float4 l4 = *reinterpret_cast<const float4 *>(lse2 + c * 32 + 4 * q);
+    const float4 d4 = *reinterpret_cast<const float4 *>(dls + c * 32 + 4 * q);
+    int4 m4 = make_int4(0, 0, 0, 0);
+    if (kMasked) m4 = *reinterpret_cast<const int4 *>(lim + c * 32 + 4 * q);
+#pragma unroll
+    for (int e = 0; e < 2; ++e) {
+      const int i = 2 * q + e;
+      const uint64_t nl2 = e ? pack2(-l4.z, -l4.w) : pack2(-l4.x, -l4.y);
+      const uint64_t nd2 = e ? pack2(-d4.z, -d4.w) : pack2(-d4.x, -d4.y);
+      const uint64_t x2 = fma2(pack2(__uint_as_float(s[2 * i]), __uint_as_float(s[2 * i + 1])), sl2, nl2);
+      float x0, x1;
+      unpack2(x2, x0, x1);
+      float p0 = ex2(x0), p1 = ex2(x1);
+      if (kMasked) {
+        if (j >= (e ? m4.z : m4.x)) p0 = 0.f;
+        if (j >= (e ? m4.w : m4.y)) p1 = 0.f;
+      }
+      const uint64_t t2 = fma2(pack2(__uint_as_float(dp[2 * i]), __uint_as_float(dp[2 * i + 1])), sc2, nd2);
+      float d0, d1;
+      unpack2(mul2(pack2(p0, p1), t2), d0, d1);
       __nv_bfloat162 pv = __floats2bfloat162_rn(p0, p1), dv = __floats2bfloat162_rn(d0, d1);
       pw[i] = *reinterpret_cast<uint32_t *>(&pv);
       dw[i] = *reinterpret_cast<uint32_t *>(&dv);
     }
-    tmem_st16(tST + c * 32, pw);         // over the first 16 of the 32 columns this thread has just read
-    tmem_st16(tDPT + c * 32, dw);
   }
+  tmem_st16(tST + c * 32, pw);
+  tmem_st16(tDPT + c * 32, dw);
   tmem_wait_st();
 }
 
@@ -344,32 +373,44 @@ ba_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
     const int j = tid & 127;                             // key of the tile = tensor-memory lane
     const int ch = tid >> 7;                             // which 32 of a step's 64 columns this thread takes
     const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
-    float4 *stats = reinterpret_cast<float4 *>(smem + L::kStats);
+    // per query row of the tile, two buffers: lse * log2 e [128], dO . O * scale [128], visible keys [128]
+    float *st_lse = reinterpret_cast<float *>(smem + L::kStats);
+    float *st_dls = st_lse + 2 * 128;
+    int *st_lim = reinterpret_cast<int *>(st_dls + 2 * 128);
     bool ok = true;
     for (int i = 0; i < n_steps; ++i) {
       const int it = i >> 1, h = i & 1;
+      int row0, row_end, head0; bool causal;
+      iter_rows(it, row0, row_end, causal, head0);
       if (h == 0) {
-        // this thread also prepares what every key thread needs to know about query row `tid` of the tile
         if (tid < 128) {
-          int row0, row_end, head0; bool causal;
-          iter_rows(it, row0, row_end, causal, head0);
+          // this thread also prepares what every key thread needs to know about query row `tid` of the tile
           const int tok_i = row0 + (tid >> p.hpt_log2);
           const int head = head0 + (tid & (p.hpt - 1));
-          float4 st = make_float4(0.f, 0.f, __int_as_float(0), 0.f);
+          float l2 = 0.f, dl = 0.f; int lm = 0;
           if (tok_i < row_end) {
-            st.x = __ldg(p.lse + (size_t)tok_i * p.Hq + head) * 1.4426950408889634f;
-            st.y = __ldg(p.delta + (size_t)tok_i * p.Hq + head);
-            st.z = __int_as_float(causal ? max(0, min(n_keys, tok_i - k0 + 1)) : n_keys);   // keys 0 .. z - 1 of the tile are visible
+            l2 = __ldg(p.lse + (size_t)tok_i * p.Hq + head) * 1.4426950408889634f;
+            dl = __ldg(p.delta + (size_t)tok_i * p.Hq + head) * p.scale;
+            lm = causal ? max(0, min(n_keys, tok_i - k0 + 1)) : n_keys;      // keys 0 .. lm - 1 of the tile are visible
           }
-          stats[(it & 1) * 128 + tid] = st;
+          st_lse[(it & 1) * 128 + tid] = l2; st_dls[(it & 1) * 128 + tid] = dl; st_lim[(it & 1) * 128 + tid] = lm;
         }
         named_barrier_rows();
       }
+      // every pair of this step visible?  (all 128 keys exist, the step's rows exist and, in the causal range,
+      // already its first row sees the tile's last key)
+      const int tok_first = row0 + ((h * 64) >> p.hpt_log2), tok_last = row0 + ((h * 64 + 63) >> p.hpt_log2);
+      const bool all_visible = n_keys == kTile && tok_last < row_end && (!causal || tok_first - k0 + 1 >= kTile);
       ok = mbar_wait(&ctrl->sd_full[i & 1], (i >> 1) & 1, abort_flag);
       if (!ok) break;
       tc_fence_after();
-      bwd_key_p_ds(tST + (i & 1) * 64 + lane_off, tDPT + (i & 1) * 64 + lane_off, ch, j, stats + (it & 1) * 128 + h * 64,
-                   p.scale_log2, p.scale);
+      const int so = (it & 1) * 128 + h * 64;
+      if (all_visible)
+        bwd_key_p_ds<false>(tST + (i & 1) * 64 + lane_off, tDPT + (i & 1) * 64 + lane_off, ch, j, st_lse + so, st_dls + so,
+                            st_lim + so, p.scale_log2, p.scale);
+      else
+        bwd_key_p_ds<true>(tST + (i & 1) * 64 + lane_off, tDPT + (i & 1) * 64 + lane_off, ch, j, st_lse + so, st_dls + so,
+                           st_lim + so, p.scale_log2, p.scale);
       tc_fence_before();
       mbar_arrive(&ctrl->rows_done[i & 1]);
     }
@@ -520,16 +561,21 @@ ba_bwd_dq_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
     float lse2 = 0.f, dl = 0.f;
     if (row_ok) {
       lse2 = __ldg(p.lse + (size_t)tok_i * p.Hq + head) * 1.4426950408889634f;
-      dl = __ldg(p.delta + (size_t)tok_i * p.Hq + head);
+      dl = __ldg(p.delta + (size_t)tok_i * p.Hq + head) * p.scale;
     }
     bool ok = true;
     for (int i = 0; i < n_steps; ++i) {
       const int kr = kv0 + i * 64;
       const int n_ok = row_ok ? max(0, min(64, tok_i - kr + 1)) : 0;
+      // every pair of this step visible?  (every row of the tile exists and already the first one sees the step's last key)
+      const bool all_visible = q0 + p.tok <= q_end && q0 - kr + 1 >= 64;
       ok = mbar_wait(&ctrl->sd_full[i & 1], (i >> 1) & 1, abort_flag);
       if (!ok) break;
       tc_fence_after();
-      bwd_row_ds(tS + (i & 1) * 64 + lane_off, tDP + (i & 1) * 64 + lane_off, ch, n_ok, p.scale_log2, lse2, dl, p.scale);
+      if (all_visible)
+        bwd_row_ds<false>(tS + (i & 1) * 64 + lane_off, tDP + (i & 1) * 64 + lane_off, ch, n_ok, p.scale_log2, lse2, dl, p.scale);
+      else
+        bwd_row_ds<true>(tS + (i & 1) * 64 + lane_off, tDP + (i & 1) * 64 + lane_off, ch, n_ok, p.scale_log2, lse2, dl, p.scale);
       tc_fence_before();
       mbar_arrive(&ctrl->rows_done[i & 1]);
     }
@@ -545,24 +591,29 @@ ba_bwd_dq_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
   if (warp == kCtlWarp) tmem_dealloc(tmem, 512);
 }
 
-// delta[row, head] = dO . O
+// delta[row, head] = dO . O: D / 8 threads per (row, head), each with one 16-byte vector of both operands
 template <int D>
 __global__ void __launch_bounds__(256)
 ba_bwd_delta_kernel(const __nv_bfloat16 *__restrict__ o, const __nv_bfloat16 *__restrict__ d_o, float *__restrict__ delta,
                     int n_rows_heads) {
-  const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
-  if (warp >= n_rows_heads) return;
-  const __nv_bfloat162 *a = reinterpret_cast<const __nv_bfloat162 *>(o + (size_t)warp * D);
-  const __nv_bfloat162 *b = reinterpret_cast<const __nv_bfloat162 *>(d_o + (size_t)warp * D);
+  constexpr int kLanes = D / 8;                          // 8 or 16 threads per row
+  const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  const long long rh = t / kLanes;
+  const int v = (int)(t - rh * kLanes);
   float acc = 0.f;
-  for (int i = lane; i < D / 2; i += 32) {
-    const float2 x = __bfloat1622float2(a[i]), y = __bfloat1622float2(b[i]);
-    acc = fmaf(x.x, y.x, acc);
-    acc = fmaf(x.y, y.y, acc);
+  if (rh < n_rows_heads) {
+    const uint4 a = __ldg(reinterpret_cast<const uint4 *>(o + rh * D) + v);
+    const uint4 b = __ldg(reinterpret_cast<const uint4 *>(d_o + rh * D) + v);
+    const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      acc = fmaf(__uint_as_float(aw[i] << 16), __uint_as_float(bw[i] << 16), acc);
+      acc = fmaf(__uint_as_float(aw[i] & 0xffff0000u), __uint_as_float(bw[i] & 0xffff0000u), acc);
+    }
   }
 #pragma unroll
-  for (int s = 16; s > 0; s >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, s);
-  if (lane == 0) delta[warp] = acc;
+  for (int sft = kLanes / 2; sft > 0; sft >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, sft);
+  if (rh < n_rows_heads && v == 0) delta[rh] = acc;
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
@@ -633,7 +684,7 @@ ba_status ba_bwd_sm100_launch(ba_ctx *ctx, const void *q, const void *k, const v
   float *delta = reinterpret_cast<float *>(reinterpret_cast<char *>(ctx->workspace) + ba_scratch_offset(ctx));
   p.delta = delta;
   const int n_rh = T * Hq;
-  const long long threads = (long long)n_rh * 32;
+  const long long threads = (long long)n_rh * (D / 8);
   if (D == 128)
     ba_bwd_delta_kernel<128><<<(unsigned)((threads + 255) / 256), 256, 0, stream>>>(
         (const __nv_bfloat16 *)o, (const __nv_bfloat16 *)d_o, delta, n_rh);
