@@ -840,3 +840,52 @@ def test_rotation_table_of_overwritten_tables_is_not_reused():
     assert not out.any()
     other.close()
     c.close()
+
+
+def test_reencode_on_a_second_stream_beside_the_attention_gives_the_same_bits():
+    """The serving loop the benchmark times: layer l+1 is re-encoded on a second stream (same context, the
+    tables' own deltas: no workspace involved) while layer l attends on the first, with events in between.
+    Outputs and re-encoded keys of every layer must be bit-identical to running everything on one stream."""
+    w = W.config2()
+    L = 6
+    c = ctx_for(w)
+    seg, buf = c.segment(w.block_lens, w.seq_nblocks, B.BA_MODE_BLOCK)
+    t = ob.segment_tables(w.block_lens, w.seq_nblocks)
+    Tc, Tf = t["n_cached_tokens"], t["n_final_tokens"]
+    xs = [{k: dev(v) for k, v in W.warm_inputs(w, l).items()} for l in range(L)]
+    def run(overlap):
+        k_re = [torch.zeros(Tc, w.n_kv_heads, w.head_dim, dtype=torch.bfloat16, device="cuda") for _ in range(L)]
+        o = [torch.zeros(Tf, w.n_q_heads, w.head_dim, dtype=torch.bfloat16, device="cuda") for _ in range(L)]
+        main = torch.cuda.Stream(priority=-1)
+        side = torch.cuda.Stream(priority=0) if overlap else main
+        start = torch.cuda.Event(); start.record(torch.cuda.current_stream())
+        main.wait_event(start); side.wait_event(start)
+        ev_re, ev_att = [], []
+        def attend(l):
+            main.wait_event(ev_re[l])
+            B.ba_final_attend(c.ctx, xs[l]["q_f"], xs[l]["k_f"], xs[l]["v_f"], Tf, k_re[l], xs[l]["v_cache"], Tc, None, 0,
+                              o[l], None, seg, B.BA_MODE_BLOCK, B.BA_OUT_BF16, stream=main)
+            e = torch.cuda.Event(); e.record(main); ev_att.append(e)
+        for l in range(L):
+            if l >= 2:
+                side.wait_event(ev_att[l - 2])
+            B.ba_reencode_k(c.ctx, xs[l]["k_cache"], None, Tc, k_re[l], seg.cache_cu, seg.cache_delta,
+                            seg.n_cached_blocks, Tc, stream=side)
+            e = torch.cuda.Event(); e.record(side); ev_re.append(e)
+            if l >= 1:
+                attend(l - 1)
+        attend(L - 1)
+        torch.cuda.synchronize()
+        return k_re, o
+    k1, o1 = run(False)
+    for _ in range(3):
+        k2, o2 = run(True)
+        for l in range(L):
+            assert torch.equal(k1[l], k2[l]) and torch.equal(o1[l], o2[l]), l
+    assert c.device_status() == B.BA_OK
+    o_ref, _ = ob.final_attend(*(W.bf16_bits_to_f64(W.warm_inputs(w, 3)[k]) for k in ("q_f", "k_f", "v_f")),
+                               ob.reencode_blocks(W.bf16_bits_to_f64(W.warm_inputs(w, 3)["k_cache"]), None, t["cache_cu"],
+                                                  t["cache_delta"], w.rope_theta),
+                               W.bf16_bits_to_f64(W.warm_inputs(w, 3)["v_cache"]), w.block_lens, w.seq_nblocks)
+    check_attention(o1[3].float().cpu().numpy(), o_ref, bf16_store=True)
+    c.close()
