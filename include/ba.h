@@ -90,6 +90,10 @@ typedef struct {
   int32_t q_tile_tokens;   /* tokens per query tile of the attention kernels */
   int32_t n_prompt_items;  /* work items of ba_block_prefill / ba_final_attend for these tables when the */
   int32_t n_final_items;   /* lengths were host arrays (exact launch size); 0 when they were on the device */
+  /* 128-key tiles the work items of ba_final_attend see, when the lengths were host arrays (else 0):
+   * sum, minimum and maximum over the items, [0..2] with the cached keys of a sequence packed in one run,
+   * [3..5] with every cached block starting a tile of its own (pools, fused path).  Used to balance the launch. */
+  int32_t final_key_tiles[6];
   /* per sequence, [batch + 1] */
   int32_t *cu_seq;         /* first row of the sequence, prompt packing */
   int32_t *cu_cache_seq;   /* first row of the sequence, cache packing */
@@ -150,6 +154,11 @@ ba_status ba_selftest_wait_expiry(ba_ctx *ctx, void *stream);
 
 /* Number of this library's kernels launched through `ctx` so far. */
 int64_t ba_launch_count(const ba_ctx *ctx);
+
+/* Diagnostic: how the last attention launch through `ctx` was laid out.  out[0] = CTAs, out[1] = partial
+ * results per row that a second kernel merges (1: none), out[2] = CTAs that each took the tail of one work
+ * item in a balanced launch (0: not balanced), out[3] = key tiles of such a tail. */
+ba_status ba_last_attend_shape(const ba_ctx *ctx, int32_t out[4]);
 
 /* Bytes of the table buffer ba_segment() needs for these sizes. */
 ba_status ba_segments_bytes(int32_t batch, int32_t n_blocks, int32_t n_tokens, size_t *bytes);

@@ -25,7 +25,7 @@ EXPORTS = [
     "ba_launch_count", "ba_segments_bytes", "ba_segment", "ba_reencode_k", "ba_block_prefill",
     "ba_final_attend", "ba_reencode_k_noalloc", "ba_selftest_wait_expiry", "ba_reencode_k_deferred", "ba_flush",
     "ba_final_attend_fused", "ba_reencode_k_paged", "ba_final_attend_paged", "ba_final_attend_fused_paged",
-    "ba_block_prefill_bwd",
+    "ba_block_prefill_bwd", "ba_last_attend_shape",
 ]
 BA_NOALLOC_MAX_BLOCKS = 4096
 
@@ -39,7 +39,8 @@ class ba_config(C.Structure):
 class ba_segments(C.Structure):
     _fields_ = [("batch", C.c_int32), ("n_blocks", C.c_int32), ("n_tokens", C.c_int32),
                 ("n_cached_blocks", C.c_int32), ("mode", C.c_int32), ("q_tile_tokens", C.c_int32),
-                ("n_prompt_items", C.c_int32), ("n_final_items", C.c_int32)] + [
+                ("n_prompt_items", C.c_int32), ("n_final_items", C.c_int32),
+                ("final_key_tiles", C.c_int32 * 6)] + [
         (n, C.c_void_p) for n in (
             "cu_seq", "cu_cache_seq", "cu_final_seq", "cu_seq_block", "cu_block", "block_delta",
             "block_seq", "block_kv_begin", "block_part_off", "block_is_final", "cache_block",
@@ -84,6 +85,7 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.ba_last_device_status.argtypes = [vp]
     lib.ba_launch_count.argtypes = [vp]
     lib.ba_launch_count.restype = C.c_int64
+    lib.ba_last_attend_shape.argtypes = [vp, C.POINTER(i32 * 4)]
     lib.ba_segments_bytes.argtypes = [i32, i32, i32, C.POINTER(sz)]
     lib.ba_segment.argtypes = [vp, vp, vp, i32, i32, i32, C.c_int, vp, sz, C.POINTER(ba_segments), vp]
     lib.ba_reencode_k.argtypes = [vp, vp, vp, i32, vp, vp, vp, i32, i32, vp]
@@ -166,6 +168,13 @@ def ba_last_device_status(ctx) -> int:
 
 def ba_launch_count(ctx) -> int:
     return int(load_library().ba_launch_count(ctx))
+
+
+def ba_last_attend_shape(ctx) -> dict:
+    """Layout of the last attention launch: CTAs, partial results per row, balanced tails and their key tiles."""
+    out = (C.c_int32 * 4)()
+    _check(load_library().ba_last_attend_shape(ctx, C.byref(out)), "ba_last_attend_shape")
+    return {"ctas": out[0], "partials": out[1], "balanced_tails": out[2], "tail_tiles": out[3]}
 
 
 def ba_segments_bytes(batch: int, n_blocks: int, n_tokens: int) -> int:

@@ -1,5 +1,6 @@
 // Host side of the C ABI: argument checks, table-buffer layout, workspace
 // bookkeeping and dispatch to the kernels.  No kernel code lives here.
+#include <algorithm>
 #include <new>
 #include <string.h>
 
@@ -190,6 +191,12 @@ ba_status ba_last_device_status(ba_ctx *ctx) {
 
 int64_t ba_launch_count(const ba_ctx *ctx) { return ctx ? ctx->launches : 0; }
 
+ba_status ba_last_attend_shape(const ba_ctx *ctx, int32_t out[4]) {
+  if (!ctx || !out) return BA_ERR_INVALID_ARG;
+  for (int i = 0; i < 4; ++i) out[i] = ctx->last_attend[i];
+  return BA_OK;
+}
+
 ba_status ba_segments_bytes(int32_t batch, int32_t n_blocks, int32_t n_tokens, size_t *bytes) {
   if (!bytes || batch < 1 || n_blocks < batch || n_tokens < n_blocks) return BA_ERR_INVALID_ARG;
   *bytes = table_layout(batch, n_blocks, n_tokens).bytes;
@@ -241,6 +248,28 @@ ba_status ba_segment(ba_ctx *ctx, const int32_t *block_lens, const int32_t *seq_
     for (int b = 0; b < n_blocks; ++b) items += (block_lens[b] + tt - 1) / tt;
     for (int q = 0, b = 0; q < batch; ++q) { b += seq_nblocks[q]; fitems += (block_lens[b - 1] + tt - 1) / tt; }
     out->n_prompt_items = (int32_t)items; out->n_final_items = (int32_t)fitems;
+    // key tiles per item of the final blocks (the counting of the attention kernel, done here on the host)
+    long long sum[2] = {0, 0}, mn[2] = {INT32_MAX, INT32_MAX}, mx[2] = {0, 0};
+    for (int q = 0, b = 0; q < batch; ++q) {
+      long long cached = 0, walked = 0;
+      for (int c = 0; c + 1 < seq_nblocks[q]; ++c) { cached += block_lens[b + c]; walked += (block_lens[b + c] + 127) / 128; }
+      b += seq_nblocks[q];
+      const long long ct[2] = {(cached + 127) / 128, walked};
+      const int fin = block_lens[b - 1];
+      for (int r0 = 0; r0 < fin; r0 += tt) {
+        const long long own = (std::min(fin, r0 + tt) + 127) / 128;
+        for (int k = 0; k < 2; ++k) {
+          const long long n = ct[k] + own;
+          sum[k] += n; mn[k] = std::min(mn[k], n); mx[k] = std::max(mx[k], n);
+        }
+      }
+    }
+    for (int k = 0; k < 2; ++k) {
+      const bool fits = sum[k] <= INT32_MAX;
+      out->final_key_tiles[3 * k] = fits ? (int32_t)sum[k] : 0;
+      out->final_key_tiles[3 * k + 1] = fits ? (int32_t)mn[k] : 0;
+      out->final_key_tiles[3 * k + 2] = fits ? (int32_t)mx[k] : 0;
+    }
   }
   auto next = [&]() { return (int32_t *)(base + L.off[i++]); };
   out->cu_seq = next(); out->cu_cache_seq = next(); out->cu_final_seq = next(); out->cu_seq_block = next();

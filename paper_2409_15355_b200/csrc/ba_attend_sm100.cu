@@ -63,6 +63,8 @@ constexpr int kStages = 3;           // ring of K/V tiles (K_j, V_j, K_j+1, ...)
 constexpr float kRescaleThreshold = 8.0f;
 constexpr int kBgStageBytes = 16384; // two spare warps x two stages of source rows
 constexpr int kWorkSlots = 4;      // ring of published work entries (power of two)
+constexpr int kBalTableOff = 512;  // balanced launch: prefix table of front tiles, in the control area behind Ctrl
+constexpr int kBalMaxPairs = 120;  // its capacity (items per head chunk); the spare warps' barriers follow at 1024
 // Register split after launch (168 per thread): the service warps give registers to the softmax warps.
 // 128 * kServiceRegs + 256 * kSoftmaxRegs <= 384 * 168.  The MMA thread keeps a work entry, descriptors
 // and ring positions live and spills below about 88; the softmax warps start to spill below 208.  On the
@@ -86,6 +88,10 @@ struct AttnParams {
   float *lse_part;                // [n_splits, n_q_rows, Hq] natural-log denominators (-inf: split saw no key)
   const int32_t *v_src_off;       // non-null: values of cached block c start at pool row v_src_off[c]
   int persistent;                 // 1: CTAs draw work from counters[0]; 0: CTA b handles entry b only
+  // balanced > 0 (final block over a long cache, fewer items than CTAs): the first `balanced` CTAs each take the
+  // last bal_len key tiles of one item (slot 0 of its partial results); the other CTAs share the key tiles in
+  // front of those, cut into equal runs whatever item they fall in (slots 1 ..).  n_splits is the slot count.
+  int balanced, bal_len;
   // three device words, zero at launch and zero again when the launch ends (its last CTA clears them):
   // [0] next entry of the work list, [1] next chunk of the background job, [2] CTAs that have finished
   int32_t *counters;
@@ -118,6 +124,15 @@ struct Layout {
   static constexpr int kBytes = kBg + 4 * kBgStageBytes;
 };
 
+// What the scheduling thread publishes to the other roles of its CTA.
+struct WorkEntry {
+  int pair;            // item (index into the list of query tile pairs); < 0: no more work
+  int chunk;           // head chunk
+  int tile0, n_tiles;  // key tiles [tile0, tile0 + n_tiles) of the item
+  int split;           // slot of the partial results this entry writes
+  int fill;            // slots fill .. n_splits - 1 of the item stay unused: this entry marks them empty
+};
+
 struct Ctrl {
   uint64_t q_full[2];
   uint64_t q_empty;               // every QK^T of the current item has completed: Q may be reloaded
@@ -129,7 +144,7 @@ struct Ctrl {
   uint64_t o_free[2];             // the softmax warps have read O_t out of tensor memory
   uint64_t work_full[kWorkSlots];  // work entry published by the scheduler (producer thread)
   uint64_t work_empty[kWorkSlots]; // entry read by the MMA thread and the 8 softmax warps
-  int work_ring[kWorkSlots];
+  WorkEntry work_ring[kWorkSlots];
   int tile_valid[8];              // pool mode: valid key columns of the cached tiles in flight
   uint32_t tmem_base;
   int abort_flag;
@@ -137,6 +152,7 @@ struct Ctrl {
   uint64_t cs_full[2];            // fused: the block's (cos, sin) row has been staged for softmax group t
   uint64_t qraw_full[2];          // fused: the plain query tile t has landed in the buffer of the version being prepared
 };
+static_assert(sizeof(Ctrl) <= kBalTableOff && kBalTableOff + (kBalMaxPairs + 1) * 4 <= 1024, "control area layout");
 
 // One work item: two query tiles of one block (or final block) and the key ranges they see.
 struct Item {
@@ -203,34 +219,48 @@ struct Work {
   Item it;
   int head0, kv_head;
   int tile0, n_tiles;   // key tiles [tile0, tile0 + n_tiles) of the item (split-KV share)
-  int split;
+  int split, fill;
 };
 
-// Decodes work index w.  Returns false past the end of the list.
+// Entry w of the global work list (equal shares of every item's key tiles).  pair < 0 past the end.
 //  Prefill: items heaviest-first (descending pair index: within a sequence an item's cost grows
 //  with its index, the final block comes last), then head chunk, then split.
 //  Final attend: all items cost about the same, so the pair index varies fastest instead: the
 //  CTAs running at the same time then work on the same (KV head, key range) for different query
 //  tiles and each K/V tile comes from HBM once and from L2 for the others.
-__device__ __forceinline__ bool next_work(const AttnParams &p, int w, Work &wk) {
+__device__ __forceinline__ WorkEntry list_entry(const AttnParams &p, int w) {
+  WorkEntry e = {-1, 0, 0, 0, 0, 0};
   const int per_pair = p.n_chunks * p.n_splits;
   const int total_pairs = __ldg(p.seg.totals + (p.final_only ? 3 : 2));
   int rank, rem;
   if (p.final_only) {
-    if (total_pairs <= 0) return false;
+    if (total_pairs <= 0) return e;
     rem = w / total_pairs; rank = w - rem * total_pairs;
-    if (rem >= per_pair) return false;
+    if (rem >= per_pair) return e;
   } else {
     rank = w / per_pair; rem = w - rank * per_pair;
-    if (rank >= total_pairs) return false;
+    if (rank >= total_pairs) return e;
   }
-  if (!resolve_item(p, total_pairs - 1 - rank, wk.it)) return false;
-  const int chunk = rem / p.n_splits;
-  wk.split = rem - chunk * p.n_splits;
-  wk.head0 = chunk * p.hpt;
+  Item it;
+  if (!resolve_item(p, total_pairs - 1 - rank, it)) return e;
+  e.pair = total_pairs - 1 - rank;
+  e.chunk = rem / p.n_splits;
+  e.split = rem - e.chunk * p.n_splits;
+  e.fill = p.n_splits;
+  e.tile0 = (int)(((long long)it.n_tiles * e.split) / p.n_splits);
+  e.n_tiles = (int)(((long long)it.n_tiles * (e.split + 1)) / p.n_splits) - e.tile0;
+  return e;
+}
+
+// A published entry, decoded by the role that reads it.  Returns false at the end of the work.
+__device__ __forceinline__ bool load_work(const AttnParams &p, const WorkEntry &e, Work &wk) {
+  if (e.pair < 0 || !resolve_item(p, e.pair, wk.it)) return false;
+  wk.head0 = e.chunk * p.hpt;
   wk.kv_head = wk.head0 / p.G;
-  wk.tile0 = (int)(((long long)wk.it.n_tiles * wk.split) / p.n_splits);
-  wk.n_tiles = (int)(((long long)wk.it.n_tiles * (wk.split + 1)) / p.n_splits) - wk.tile0;
+  wk.tile0 = e.tile0;
+  wk.n_tiles = e.n_tiles;
+  wk.split = e.split;
+  wk.fill = e.fill;
   return true;
 }
 
@@ -363,9 +393,83 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
   if (warp == 8) {
     // ------------------------------------------------------------ TMA producer
     asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kProdRegs));
+    // balanced launch, a CTA that shares the front key tiles: prefix sum of the front tiles of every item (the
+    // same for every head chunk), one item per lane, kept in shared memory for the scheduling thread
+    int *bal_cu = reinterpret_cast<int *>(smem + L::kCtrl + kBalTableOff);
+    int bal_np = 0;
+    if (p.balanced && tables_ok) {
+      bal_np = __ldg(p.seg.totals + 3);
+      if (bal_np < 1 || bal_np > kBalMaxPairs || bal_np * p.n_chunks != p.balanced) {
+        ba_record_status(p.status, BA_ERR_SHAPE);          // the tables describe another launch than the host sized
+        bal_np = 0;
+      } else if ((int)blockIdx.x >= p.balanced) {
+        const int lane = tid & 31;
+        int carry = 0;
+        for (int base = 0; base < bal_np; base += 32) {
+          const int i = base + lane;
+          int x = 0;
+          Item it;
+          if (i < bal_np && resolve_item(p, bal_np - 1 - i, it)) x = max(0, it.n_tiles - p.bal_len);
+#pragma unroll
+          for (int o = 1; o < 32; o <<= 1) {
+            const int y = __shfl_up_sync(0xffffffffu, x, o);
+            if (lane >= o) x += y;
+          }
+          if (i < bal_np) bal_cu[i + 1] = carry + x;
+          carry += __shfl_sync(0xffffffffu, x, 31);
+        }
+        if (lane == 0) bal_cu[0] = 0;
+        __syncwarp();
+      }
+    }
     if (elect_one()) {
       prefetch_tmap(&tmap_q); prefetch_tmap(&tmap_k); prefetch_tmap(&tmap_v);
       prefetch_tmap(&tmap_kc); prefetch_tmap(&tmap_vc);
+      // balanced launch: run [bal_pos, bal_end) of the front tiles of all (chunk, item), bal_hm of them per chunk
+      int bal_pos = 0, bal_end = 0, bal_hm = 0, bal_nh = 0;
+      long long bal_all = 0;
+      if (bal_np > 0 && (int)blockIdx.x >= p.balanced) {
+        bal_hm = bal_cu[bal_np];
+        bal_all = (long long)bal_hm * p.n_chunks;
+        bal_nh = (int)gridDim.x - p.balanced;
+        const int j = (int)blockIdx.x - p.balanced;
+        bal_pos = (int)(bal_all * j / bal_nh);
+        bal_end = (int)(bal_all * (j + 1) / bal_nh);
+      }
+      auto balanced_entry = [&](int n_done) -> WorkEntry {
+        WorkEntry e = {-1, 0, 0, 0, 0, 0};
+        if (bal_np == 0) return e;
+        const int b = (int)blockIdx.x;
+        if (b < p.balanced) {                              // the last bal_len key tiles of item b
+          if (n_done > 0) return e;
+          Item it;
+          const int pair = bal_np - 1 - b % bal_np;
+          if (!resolve_item(p, pair, it)) return e;
+          e.pair = pair; e.chunk = b / bal_np;
+          e.tile0 = max(0, it.n_tiles - p.bal_len);
+          e.n_tiles = it.n_tiles - e.tile0;
+          e.split = 0;
+          e.fill = e.tile0 == 0 ? 1 : p.n_splits;           // nothing in front: the other slots stay empty
+          return e;
+        }
+        if (bal_pos >= bal_end) return e;
+        const int chunk = bal_pos / bal_hm, r = bal_pos - chunk * bal_hm;
+        int lo = 0, hi = bal_np + 1;                        // item i with bal_cu[i] <= r < bal_cu[i + 1]
+        while (lo < hi) { const int mid = (lo + hi) >> 1; if (bal_cu[mid] <= r) lo = mid + 1; else hi = mid; }
+        const int i = lo - 1;
+        const int front_end = chunk * bal_hm + bal_cu[i + 1];
+        const int n = min(bal_end, front_end) - bal_pos;
+        // the slot counts the CTAs from the one that holds the first front tile of the item
+        const long long g0 = (long long)chunk * bal_hm + bal_cu[i];
+        const int j_first = (int)(((g0 + 1) * bal_nh - 1) / bal_all);
+        e.split = 1 + ((int)blockIdx.x - p.balanced) - j_first;
+        if (e.split >= p.n_splits) { ba_record_status(p.status, BA_ERR_SHAPE); return e; }
+        e.pair = bal_np - 1 - i; e.chunk = chunk;
+        e.tile0 = r - bal_cu[i]; e.n_tiles = n;
+        e.fill = bal_pos + n == front_end ? e.split + 1 : p.n_splits;
+        bal_pos += n;
+        return e;
+      };
       int gidx = 0;                       // K/V tiles requested so far (ring position)
       int n_items = 0;                    // items with at least one tile so far
       bool ok = true;
@@ -376,10 +480,17 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
         const int slot = n_work & (kWorkSlots - 1);
         ok = mbar_wait(&ctrl->work_empty[slot], ((n_work / kWorkSlots) & 1) ^ 1, abort_flag);
         if (!ok) break;
-        // persistent launch: next entry of the global list; one-item launch: this CTA's own entry, then stop
-        const int w = p.persistent ? atomicAdd(p.counters, 1) : (n_work == 0 ? (int)blockIdx.x : 0x7fffffff);
-        const bool more = tables_ok && next_work(p, w, wk);
-        ctrl->work_ring[slot] = more ? w : -1;
+        // balanced launch: the next piece of this CTA's share; persistent launch: next entry of the global list;
+        // one-item launch: this CTA's own entry, then stop
+        WorkEntry e = {-1, 0, 0, 0, 0, 0};
+        if (tables_ok) {
+          if (p.balanced) e = balanced_entry(n_work);
+          else if (p.persistent) e = list_entry(p, atomicAdd(p.counters, 1));
+          else if (n_work == 0) e = list_entry(p, (int)blockIdx.x);
+        }
+        const bool more = load_work(p, e, wk);
+        if (!more) e.pair = -1;
+        ctrl->work_ring[slot] = e;
         mbar_arrive(&ctrl->work_full[slot]);
         ++n_work;
         if (!more) break;
@@ -562,9 +673,9 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
         const int slot = n_work & (kWorkSlots - 1);
         ok = mbar_wait(&ctrl->work_full[slot], (n_work / kWorkSlots) & 1, abort_flag);
         if (!ok) break;
-        const int w = ctrl->work_ring[slot];
+        const WorkEntry e = ctrl->work_ring[slot];
         ++n_work;
-        if (w < 0 || !next_work(p, w, wk)) break;
+        if (!load_work(p, e, wk)) break;
         mbar_arrive(&ctrl->work_empty[slot]);          // the entry has been decoded into registers
         const int n_tiles = wk.n_tiles, n_qt = wk.it.n_qt;
         if (n_tiles == 0) continue;
@@ -665,9 +776,9 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
       const int slot = n_work & (kWorkSlots - 1);
       ok = mbar_wait(&ctrl->work_full[slot], (n_work / kWorkSlots) & 1, abort_flag);
       if (!ok) break;
-      const int w = ctrl->work_ring[slot];
+      const WorkEntry e = ctrl->work_ring[slot];
       ++n_work;
-      if (w < 0 || !next_work(p, w, wk)) break;
+      if (!load_work(p, e, wk)) break;
       __syncwarp();
       if ((tid & 31) == 0) mbar_arrive(&ctrl->work_empty[slot]);   // one arrival per softmax warp
       const Item &it = wk.it;
@@ -883,8 +994,18 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
             for (int i = 0; i < 32; ++i) o[i] = 0u;
           }
           if (row_valid) {
-            if (partial || p.out_f32) {
-              float4 *dst = reinterpret_cast<float4 *>((partial ? part : reinterpret_cast<float *>(p.o) + orow) + c * 32);
+            if (partial) {
+              // 32-byte stores (the workspace is aligned for them): a thread owns a row, so each fills a whole sector
+              float *dst = part + c * 32;
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {
+                float v[8];
+#pragma unroll
+                for (int e = 0; e < 8; ++e) v[e] = __uint_as_float(o[8 * i + e]) * inv;
+                st_global_v8(dst + 8 * i, v);
+              }
+            } else if (p.out_f32) {
+              float4 *dst = reinterpret_cast<float4 *>(reinterpret_cast<float *>(p.o) + orow + c * 32);
 #pragma unroll
               for (int i = 0; i < 8; ++i)
                 dst[i] = make_float4(__uint_as_float(o[4 * i]) * inv, __uint_as_float(o[4 * i + 1]) * inv,
@@ -911,8 +1032,11 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
           mbar_arrive(&ctrl->o_free[t]);
         }
         if (row_valid) {
-          if (partial) p.lse_part[((size_t)wk.split * p.n_q_rows + row_tok) * p.Hq + head] = lse_val;
-          else if (p.lse) p.lse[(size_t)row_tok * p.Hq + head] = lse_val;
+          if (partial) {
+            p.lse_part[((size_t)wk.split * p.n_q_rows + row_tok) * p.Hq + head] = lse_val;
+            for (int s = wk.fill; s < p.n_splits; ++s)      // slots no entry of this item writes: empty
+              p.lse_part[((size_t)s * p.n_q_rows + row_tok) * p.Hq + head] = -INFINITY;
+          } else if (p.lse) p.lse[(size_t)row_tok * p.Hq + head] = lse_val;
         }
       }
       }
@@ -963,6 +1087,7 @@ ba_combine_splits_kernel(const float *__restrict__ o_part, const float *__restri
 #pragma unroll
     for (int s = 0; s < kNS; ++s) {
       const float w = (ls[s] == -INFINITY) ? 0.f : __expf(ls[s] - mx);
+      if (w == 0.f) x[s] = make_float4(0.f, 0.f, 0.f, 0.f);   // an empty slot holds no values at all
       den += w;
       acc.x = fmaf(w, x[s].x, acc.x); acc.y = fmaf(w, x[s].y, acc.y); acc.z = fmaf(w, x[s].z, acc.z); acc.w = fmaf(w, x[s].w, acc.w);
     }
@@ -971,7 +1096,8 @@ ba_combine_splits_kernel(const float *__restrict__ o_part, const float *__restri
     for (int s = 0; s < n_splits; ++s) {
       const float ls = __ldg(lse_part + (size_t)s * n_rows_heads + rh);
       const float w = (ls == -INFINITY) ? 0.f : __expf(ls - mx);
-      const float4 x = __ldg(reinterpret_cast<const float4 *>(o_part + ((size_t)s * n_rows_heads + rh) * D) + v);
+      float4 x = __ldg(reinterpret_cast<const float4 *>(o_part + ((size_t)s * n_rows_heads + rh) * D) + v);
+      if (w == 0.f) x = make_float4(0.f, 0.f, 0.f, 0.f);
       den += w;
       acc.x = fmaf(w, x.x, acc.x); acc.y = fmaf(w, x.y, acc.y); acc.z = fmaf(w, x.z, acc.z); acc.w = fmaf(w, x.w, acc.w);
     }
@@ -1120,6 +1246,7 @@ ba_status ba_attend_sm100_launch(ba_ctx *ctx, const ba_attend_args &a, const ba_
   p.scale = ctx->scale;
   p.scale_log2 = ctx->scale * 1.4426950408889634f;
   p.final_only = a.final_only;
+  p.balanced = 0; p.bal_len = 0;
   p.v_src_off = a.final_only ? a.v_src_off : nullptr;
   p.fused = a.final_only && a.fused && a.n_cache_rows > 0;
   p.k_src_off = p.fused ? a.k_src_off : nullptr;
@@ -1150,7 +1277,11 @@ ba_status ba_attend_sm100_launch(ba_ctx *ctx, const ba_attend_args &a, const ba_
   const long long items = (long long)((a.n_q_rows + pair_tok - 1) / pair_tok) * (Hq / p.hpt);
   int n_splits = 1;
   if (a.final_only && items < 2LL * ctx->sm_count) {
-    const long long avg_tiles = ((long long)a.n_cache_rows / seg->batch + pair_tok) / kBlockN + 1;
+    // key tiles of an average item: counted by ba_segment() when it saw the lengths, else estimated
+    const int32_t *ft = seg->final_key_tiles + (p.walk ? 3 : 0);
+    const long long avg_tiles = (ft[0] > 0 && seg->n_final_items > 0)
+                                    ? (ft[0] + seg->n_final_items - 1) / seg->n_final_items
+                                    : ((long long)a.n_cache_rows / seg->batch + pair_tok) / kBlockN + 1;
     const size_t per_split = (size_t)a.n_q_rows * Hq * (D + 1) * sizeof(float);
     // the angle table of a queued re-encoding job sits at the end of the workspace and is read by
     // this very launch: the partial results must stay below it
@@ -1163,6 +1294,28 @@ ba_status ba_attend_sm100_launch(ba_ctx *ctx, const ba_attend_args &a, const ba_
       const long long cost = waves * ((avg_tiles + ns - 1) / ns + 3);
       if (best < 0 || cost < best) { best = cost; n_splits = ns; }
     }
+    // Balanced launch (item sizes known on the host, fewer items than SMs, every item longer than an SM's
+    // share of the tiles): one CTA per item takes the item's last `len` key tiles, the remaining CTAs share the
+    // tiles in front of those in equal runs.  `len` starts at the even share and grows until the CTAs that
+    // work on several pieces (each with its own start-up and write-out, counted as 3 tiles, plus 1 for their
+    // table) are no longer the slower ones.  Taken when the same cost model puts it ahead of equal splits.
+    const long long n_main = (long long)seg->n_final_items * (Hq / p.hpt);
+    const long long n_front = ctx->sm_count - n_main;
+    if (ft[0] > 0 && n_main > 0 && n_front > 0 && seg->n_final_items <= kBalMaxPairs) {
+      const long long total = (long long)ft[0] * (Hq / p.hpt), n_min = ft[1], n_max = ft[2];
+      for (long long len = (total + ctx->sm_count - 1) / ctx->sm_count; len <= n_min; ++len) {
+        const long long front = total - n_main * len;
+        if (front <= 0) break;
+        const long long run = (front + n_front - 1) / n_front, run_min = front / n_front;
+        if (run_min < 1) break;
+        const long long piece = (front + n_main - 1) / n_main;          // average front tiles of an item
+        const long long cost_front = run + 3 * ((run + piece - 1) / piece + 1) + 1;
+        if (cost_front > len + 3) continue;
+        const long long slots = 1 + (n_max - len + run_min - 1) / run_min + 1;
+        if (len + 3 < best && slots <= cap) { p.balanced = (int)n_main; p.bal_len = (int)len; n_splits = (int)slots; }
+        break;
+      }
+    }
   }
   p.n_splits = n_splits;
   p.n_chunks = Hq / p.hpt;
@@ -1171,7 +1324,7 @@ ba_status ba_attend_sm100_launch(ba_ctx *ctx, const ba_attend_args &a, const ba_
   // over a long cache: about two, the write-out of a CTA's first entry overlaps the start of its second).
   // Shorter lists are launched one CTA per entry.
   const long long work_upper = (long long)pairs_upper * (Hq / p.hpt) * n_splits;
-  p.persistent = items * n_splits > (a.final_only ? 1LL : 2LL) * ctx->sm_count;
+  p.persistent = !p.balanced && items * n_splits > (a.final_only ? 1LL : 2LL) * ctx->sm_count;
   // the counters live in the last 256 bytes below the scratch area: zeroed by ba_create, left at zero by every launch
   int32_t *counters = nullptr;
   if (ctx->workspace && ctx->workspace_bytes >= ba_scratch_offset(ctx))
@@ -1201,7 +1354,7 @@ ba_status ba_attend_sm100_launch(ba_ctx *ctx, const ba_attend_args &a, const ba_
     if (!mvc) return BA_ERR_CUDA;
     tvc = *mvc;
   }
-  dim3 grid((unsigned)(p.persistent ? ctx->sm_count : work_upper));
+  dim3 grid((unsigned)((p.persistent || p.balanced) ? ctx->sm_count : work_upper));
   // a queued re-encoding job rides along in the spare warps; a job whose rows do not fit the
   // staging buffers is run on its own first
   p.bg.n_rows = 0; p.bg_rows_per_chunk = 0;
@@ -1244,6 +1397,8 @@ ba_status ba_attend_sm100_launch(ba_ctx *ctx, const ba_attend_args &a, const ba_
   }
   BA_CUDA_TRY(cudaGetLastError());
   ctx->launches += 1;
+  ctx->last_attend[0] = (int32_t)grid.x; ctx->last_attend[1] = n_splits;
+  ctx->last_attend[2] = p.balanced; ctx->last_attend[3] = p.bal_len;
   if (side_job) BA_CUDA_TRY(cudaStreamWaitEvent(stream, ctx->ev_join, 0));
   if (n_splits > 1) {
     const int n_rh = a.n_q_rows * Hq;

@@ -61,6 +61,7 @@ struct ba_ctx {
   size_t workspace_bytes;
   int32_t *dev_status;      // device word: first non-zero ba_status recorded by a kernel
   int64_t launches;
+  int32_t last_attend[4];          // layout of the last attention launch: CTAs, partial slots, balanced tails, tail tiles
   // a re-encoding job queued by ba_reencode_k_deferred: carried along by the next attention
   // launch (or run by ba_flush); its angle table sits at the very end of the workspace
   ba_reencode_job pending;

@@ -229,4 +229,11 @@ __device__ __forceinline__ float ex2(float x) {
   return y;
 }
 
+// One 32-byte store (the address must be 32-byte aligned).
+__device__ __forceinline__ void st_global_v8(float *dst, const float (&v)[8]) {
+  asm volatile("st.global.v8.f32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(dst), "f"(v[0]), "f"(v[1]), "f"(v[2]),
+               "f"(v[3]), "f"(v[4]), "f"(v[5]), "f"(v[6]), "f"(v[7])
+               : "memory");
+}
+
 }  // namespace sm100

@@ -70,6 +70,9 @@ class Context:
     def launches(self) -> int:
         return B.ba_launch_count(self.ctx)
 
+    def last_attend_shape(self) -> dict:
+        return B.ba_last_attend_shape(self.ctx)
+
 
 _TABLE_SIZES = {
     "cu_seq": ("batch", 1), "cu_cache_seq": ("batch", 1), "cu_final_seq": ("batch", 1),

@@ -335,7 +335,7 @@ def test_prefill_full_causal_32k_sampled_rows():
 
 # --------------------------------------------------------------------------- warm path
 def run_warm(w, mode, out_dtype=B.BA_OUT_F32, layer=0, v_from_pool=True, fused=False,
-             layout=B.BA_ROPE_ADJACENT):
+             layout=B.BA_ROPE_ADJACENT, shape_out=None):
     """ba_segment -> ba_reencode_k -> ba_final_attend (or ba_final_attend_fused on the keys as
     cached), against oracle re-encode + final attend.  The oracle attends its own unrounded fp64
     re-encoded keys."""
@@ -374,6 +374,8 @@ def run_warm(w, mode, out_dtype=B.BA_OUT_F32, layer=0, v_from_pool=True, fused=F
                         seg.n_cached_blocks, Tc)
         B.ba_final_attend(c.ctx, q_f, k_f, v_f, Tf, k_re, v_cache, Tc, v_off, n_v, o, lse, seg, mode, out_dtype)
     assert c.device_status() == B.BA_OK
+    if shape_out is not None:
+        shape_out.append(c.last_attend_shape())
     k_ref = ob.reencode_blocks(W.bf16_bits_to_f64(k_src_np), off_np, t["cache_cu"], t["cache_delta"], w.rope_theta,
                                layout)
     o_ref, lse_ref = ob.final_attend(W.bf16_bits_to_f64(x["q_f"]), W.bf16_bits_to_f64(x["k_f"]),
@@ -551,6 +553,29 @@ def test_paged_cache_bad_page_numbers_are_reported_and_bad_sizes_refused():
                                   seg.cache_delta, seg.n_cached_blocks, 256)
         assert e.value.status == B.BA_ERR_UNSUPPORTED
     c.close()
+
+
+def _balanced_cases():
+    """Final blocks over long caches with fewer work items than SMs: the launch gives one CTA the tail of each
+    item and lets the others share the key tiles in front (ragged cached blocks, ragged final blocks, two
+    sequences of unequal length, two head chunks per KV group, head_dim 64)."""
+    rng = np.random.default_rng(77)
+    one = [int(v) for v in rng.integers(300, 900, 20)] + [700]
+    two_a = [int(v) for v in rng.integers(200, 700, 20)] + [300]
+    two_b = [int(v) for v in rng.integers(200, 700, 23)] + [330]
+    d64 = [int(v) for v in rng.integers(500, 1500, 8)] + [1390]
+    return [W.Workload("balanced_one_sequence", 32, 8, 128, 5e5, one, [21], seed=81),
+            W.Workload("balanced_two_sequences", 32, 8, 128, 5e5, two_a + two_b, [21, 24], seed=82),
+            W.Workload("balanced_head_dim_64_two_chunks", 16, 2, 64, 1e4, d64, [9], seed=83)]
+
+
+@pytest.mark.parametrize("w", _balanced_cases(), ids=lambda w: w.name)
+@pytest.mark.parametrize("fused", [False, True], ids=["reencode_then_attend", "fused"])
+def test_balanced_launch_parity(w, fused):
+    shapes = []
+    o, lse, o_ref, lse_ref = run_warm(w, B.BA_MODE_BLOCK, fused=fused, shape_out=shapes)
+    assert shapes[-1]["balanced_tails"] > 0 and shapes[-1]["partials"] >= 2, shapes
+    check_attention(o, o_ref, lse, lse_ref)
 
 
 def test_warm_path_32k_full_size():
