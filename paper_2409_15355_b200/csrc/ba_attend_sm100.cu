@@ -92,6 +92,7 @@ struct AttnParams {
   // last bal_len key tiles of one item (slot 0 of its partial results); the other CTAs share the key tiles in
   // front of those, cut into equal runs whatever item they fall in (slots 1 ..).  n_splits is the slot count.
   int balanced, bal_len;
+  int q_double;                   // plain path, no background job: two pairs of query buffers (see Ctrl)
   // three device words, zero at launch and zero again when the launch ends (its last CTA clears them):
   // [0] next entry of the work list, [1] next chunk of the background job, [2] CTAs that have finished
   int32_t *counters;
@@ -134,8 +135,10 @@ struct WorkEntry {
 };
 
 struct Ctrl {
-  uint64_t q_full[2];
-  uint64_t q_empty;               // every QK^T of the current item has completed: Q may be reloaded
+  // [buffer pair][query tile].  Plain path without a background job: the query tiles of successive entries
+  // alternate between two pairs of buffers, so the next entry's queries are fetched while the current one runs.
+  uint64_t q_full[2][2];
+  uint64_t q_empty[2];            // every QK^T of the entry that used this buffer pair has completed: it may be reloaded
   uint64_t kv_full[kStages];
   uint64_t kv_empty[kStages];
   uint64_t s_full[2];
@@ -366,7 +369,7 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
   const int tid = threadIdx.x, warp = tid >> 5;
 
   if (tid == 0) {
-    mbar_init(&ctrl->q_full[0], 1); mbar_init(&ctrl->q_full[1], 1); mbar_init(&ctrl->q_empty, 1);
+    for (int b = 0; b < 2; ++b) { mbar_init(&ctrl->q_full[b][0], 1); mbar_init(&ctrl->q_full[b][1], 1); mbar_init(&ctrl->q_empty[b], 1); }
     for (int s = 0; s < kStages; ++s) { mbar_init(&ctrl->kv_full[s], 1); mbar_init(&ctrl->kv_empty[s], 1); }
     for (int t = 0; t < 2; ++t) {
       mbar_init(&ctrl->s_full[t], 1); mbar_init(&ctrl->p_full[t][0], 128); mbar_init(&ctrl->p_full[t][1], 128);
@@ -498,14 +501,18 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
         const Item &it = wk.it;
         if (!kFused) {      // (on the fused path the softmax warps fetch the query tiles themselves)
           // the Q buffers are free once every QK^T of the previous item has completed
-          ok = mbar_wait(&ctrl->q_empty, (n_items & 1) ^ 1, abort_flag);
+          const int qb = p.q_double ? (n_items & 1) : 0;           // buffer pair of this entry
+          const int q_use = p.q_double ? (n_items >> 1) : n_items;  // earlier entries that used it
+          ok = mbar_wait(&ctrl->q_empty[qb], (q_use & 1) ^ 1, abort_flag);
           if (!ok) break;
           ++n_items;
-          for (int t = 0; t < it.n_qt; ++t) {
-            mbar_arrive_expect_tx(&ctrl->q_full[t], L::kTileBytes);
+          for (int t = 0; t < 2; ++t) {
+            if (t >= it.n_qt) { mbar_arrive(&ctrl->q_full[qb][t]); continue; }   // (every entry moves both barriers on)
+            mbar_arrive_expect_tx(&ctrl->q_full[qb][t], L::kTileBytes);
+            uint8_t *dst = smem + (qb ? L::kBg + t * L::kTileBytes : (t ? L::kQ1 : L::kQ0));
             for (int c = 0; c < L::kChunks; ++c)
-              tma_load_3d(smem + (t ? L::kQ1 : L::kQ0) + c * L::kRegionBytes, &tmap_q, &ctrl->q_full[t], c * 64,
-                          wk.head0, it.q_row0 + t * p.tok);
+              tma_load_3d(dst + c * L::kRegionBytes, &tmap_q, &ctrl->q_full[qb][t], c * 64, wk.head0,
+                          it.q_row0 + t * p.tok);
           }
         }
         // walk mode: cached keys are taken block by block (block pc, row offset poff inside it).  The
@@ -642,9 +649,10 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
       int ver_end[2] = {-1, -1};           // the current version of tile t serves cached key tiles below this index
       int walk_pc = 0, walk_end = -1;      // block of the current cached tile and the tile index where it ends
       int cached_end = 0;                  // tiles [tile0, cached_end) of the entry are cached keys
+      int q_buf = 0;                       // plain path: buffer pair that holds the entry's query tiles
       // S_t = Q_t K^T for tile `jrel` of the entry, whose keys sit at ring position idx
       auto issue_qk = [&](int t, int jrel, int idx) -> bool {
-        if (!kFused) { issue_qk_with(t, jrel, idx, q_desc[t]); return true; }
+        if (!kFused) { issue_qk_with(t, jrel, idx, q_buf ? qb_desc[t] : q_desc[t]); return true; }
         const int jt = wk.tile0 + jrel;
         bool change = false;
         if (jt < cached_end) {
@@ -684,9 +692,12 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
         walk_end = -1; ver_end[0] = ver_end[1] = -1;
         cached_end = min(wk.tile0 + n_tiles, wk.it.n_cache_tiles);
         if (!kFused) {
+          // (query tile 0 is part of every entry: q_uses[0] counts the entries)
+          q_buf = p.q_double ? (q_uses[0] & 1) : 0;
+          const int q_use = p.q_double ? (q_uses[0] >> 1) : q_uses[0];
 #pragma unroll
           for (int t = 0; t < 2; ++t)
-            if (t < n_qt && ok) ok = mbar_wait(&ctrl->q_full[t], q_uses[t] & 1, abort_flag);
+            if (t < n_qt && ok) ok = mbar_wait(&ctrl->q_full[q_buf][t], q_use & 1, abort_flag);
         }
         if (ok) ok = wait_kv(gidx);
         if (!ok) break;
@@ -696,7 +707,7 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
           if (t < n_qt && ok) ok = issue_qk(t, 0, gidx);
         if (!ok) break;
         mma_commit(&ctrl->kv_empty[gidx % kStages]);
-        if (n_tiles == 1) mma_commit(&ctrl->q_empty);
+        if (n_tiles == 1) mma_commit(&ctrl->q_empty[q_buf]);
         for (int j = 0; j < n_tiles && ok; ++j) {
           const bool last = j + 1 == n_tiles;
           const int iv = gidx + 2 * j + 1, ik = gidx + 2 * j + 2;   // ring positions of V_j and K_(j+1)
@@ -731,7 +742,7 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
               BA_TR(2, j, t * 4 + 3);
               if (t + 1 == n_qt) {
                 mma_commit(&ctrl->kv_empty[ik % kStages]);
-                if (j + 2 == n_tiles) mma_commit(&ctrl->q_empty);   // that was the item's last QK^T
+                if (j + 2 == n_tiles) mma_commit(&ctrl->q_empty[q_buf]);   // that was the item's last QK^T
               }
             }
           }
@@ -1246,7 +1257,7 @@ ba_status ba_attend_sm100_launch(ba_ctx *ctx, const ba_attend_args &a, const ba_
   p.scale = ctx->scale;
   p.scale_log2 = ctx->scale * 1.4426950408889634f;
   p.final_only = a.final_only;
-  p.balanced = 0; p.bal_len = 0;
+  p.balanced = 0; p.bal_len = 0; p.q_double = 0;
   p.v_src_off = a.final_only ? a.v_src_off : nullptr;
   p.fused = a.final_only && a.fused && a.n_cache_rows > 0;
   p.k_src_off = p.fused ? a.k_src_off : nullptr;
@@ -1371,6 +1382,7 @@ ba_status ba_attend_sm100_launch(ba_ctx *ctx, const ba_attend_args &a, const ba_
       if (fs != BA_OK) return fs;
     }
   }
+  p.q_double = (!p.fused && p.bg.n_rows == 0) ? 1 : 0;     // the staging area is free: second pair of query buffers
   // Side output of the fused call: the re-encoded keys, written by the stand-alone re-encoding kernel on the
   // context's side stream beside the attention launch (which cannot share an SM with anything and leaves
   // some SMs idle in its last wave); the caller's stream continues only when both are done.  (Measured
