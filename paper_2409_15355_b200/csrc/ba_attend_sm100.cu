@@ -128,6 +128,7 @@ struct Layout {
 // What the scheduling thread publishes to the other roles of its CTA.
 struct WorkEntry {
   int pair;            // item (index into the list of query tile pairs); < 0: no more work
+  int unit;            // the sequence (final attend) or block (prefill) of the item
   int chunk;           // head chunk
   int tile0, n_tiles;  // key tiles [tile0, tile0 + n_tiles) of the item
   int split;           // slot of the partial results this entry writes
@@ -184,12 +185,26 @@ __device__ __forceinline__ int upper_bound_tbl(const int32_t *a, int n, int x) {
   return lo;
 }
 
-__device__ __forceinline__ bool resolve_item(const AttnParams &p, int pair, Item &it) {
+// The sequence (final attend) or block (prefill) that item `pair` belongs to; -1 past the end of the list.
+__device__ __forceinline__ int find_unit(const AttnParams &p, int pair) {
+  const ba_segments &sg = p.seg;
+  if (p.final_only) {
+    if (pair >= __ldg(sg.totals + 3)) return -1;
+    if (sg.batch == 1) return 0;
+    return upper_bound_tbl(sg.cu_ftile, sg.batch + 1, pair) - 1;
+  }
+  if (pair >= __ldg(sg.totals + 2)) return -1;
+  return upper_bound_tbl(sg.cu_qtile, sg.n_blocks + 1, pair) - 1;
+}
+
+// Item `pair` of sequence / block `unit`.  The table look-ups are independent of one another (the search for the
+// unit, a chain of dependent loads, is done once by the scheduling thread and published with the entry).
+__device__ __forceinline__ bool resolve_item(const AttnParams &p, int pair, int unit, Item &it) {
   const ba_segments &sg = p.seg;
   const int pair_tok = 2 * p.tok;
+  if (unit < 0) return false;
   if (p.final_only) {
-    if (pair >= __ldg(sg.totals + 3)) return false;
-    int s = upper_bound_tbl(sg.cu_ftile, sg.batch + 1, pair) - 1;
+    const int s = unit;
     int f0 = __ldg(sg.cu_final_seq + s), f1 = __ldg(sg.cu_final_seq + s + 1);
     it.q_row0 = f0 + (pair - __ldg(sg.cu_ftile + s)) * pair_tok;
     it.q_rows = min(pair_tok, f1 - it.q_row0);
@@ -197,12 +212,11 @@ __device__ __forceinline__ bool resolve_item(const AttnParams &p, int pair, Item
     it.cache_len = __ldg(sg.cu_cache_seq + s + 1) - it.cache_row0;
     it.own_row0 = f0;
     it.cb0 = __ldg(sg.cu_seq_block + s) - s;           // every earlier sequence has one final block
-    it.ctile0 = __ldg(sg.cache_tile_cu + it.cb0);
+    it.ctile0 = p.walk ? __ldg(sg.cache_tile_cu + it.cb0) : 0;
     it.n_cache_tiles = p.walk ? __ldg(sg.cache_tile_cu + (__ldg(sg.cu_seq_block + s + 1) - s - 1)) - it.ctile0
                                    : (it.cache_len + kBlockN - 1) / kBlockN;
   } else {
-    if (pair >= __ldg(sg.totals + 2)) return false;
-    int b = upper_bound_tbl(sg.cu_qtile, sg.n_blocks + 1, pair) - 1;
+    const int b = unit;
     int b0 = __ldg(sg.cu_block + b), b1 = __ldg(sg.cu_block + b + 1);
     it.q_row0 = b0 + (pair - __ldg(sg.cu_qtile + b)) * pair_tok;
     it.q_rows = min(pair_tok, b1 - it.q_row0);
@@ -232,7 +246,7 @@ struct Work {
 //  CTAs running at the same time then work on the same (KV head, key range) for different query
 //  tiles and each K/V tile comes from HBM once and from L2 for the others.
 __device__ __forceinline__ WorkEntry list_entry(const AttnParams &p, int w) {
-  WorkEntry e = {-1, 0, 0, 0, 0, 0};
+  WorkEntry e = {-1, -1, 0, 0, 0, 0, 0};
   const int per_pair = p.n_chunks * p.n_splits;
   const int total_pairs = __ldg(p.seg.totals + (p.final_only ? 3 : 2));
   int rank, rem;
@@ -245,7 +259,8 @@ __device__ __forceinline__ WorkEntry list_entry(const AttnParams &p, int w) {
     if (rank >= total_pairs) return e;
   }
   Item it;
-  if (!resolve_item(p, total_pairs - 1 - rank, it)) return e;
+  e.unit = find_unit(p, total_pairs - 1 - rank);
+  if (!resolve_item(p, total_pairs - 1 - rank, e.unit, it)) return e;
   e.pair = total_pairs - 1 - rank;
   e.chunk = rem / p.n_splits;
   e.split = rem - e.chunk * p.n_splits;
@@ -257,7 +272,7 @@ __device__ __forceinline__ WorkEntry list_entry(const AttnParams &p, int w) {
 
 // A published entry, decoded by the role that reads it.  Returns false at the end of the work.
 __device__ __forceinline__ bool load_work(const AttnParams &p, const WorkEntry &e, Work &wk) {
-  if (e.pair < 0 || !resolve_item(p, e.pair, wk.it)) return false;
+  if (e.pair < 0 || !resolve_item(p, e.pair, e.unit, wk.it)) return false;
   wk.head0 = e.chunk * p.hpt;
   wk.kv_head = wk.head0 / p.G;
   wk.tile0 = e.tile0;
@@ -412,7 +427,7 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
           const int i = base + lane;
           int x = 0;
           Item it;
-          if (i < bal_np && resolve_item(p, bal_np - 1 - i, it)) x = max(0, it.n_tiles - p.bal_len);
+          if (i < bal_np && resolve_item(p, bal_np - 1 - i, find_unit(p, bal_np - 1 - i), it)) x = max(0, it.n_tiles - p.bal_len);
 #pragma unroll
           for (int o = 1; o < 32; o <<= 1) {
             const int y = __shfl_up_sync(0xffffffffu, x, o);
@@ -440,14 +455,15 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
         bal_end = (int)(bal_all * (j + 1) / bal_nh);
       }
       auto balanced_entry = [&](int n_done) -> WorkEntry {
-        WorkEntry e = {-1, 0, 0, 0, 0, 0};
+        WorkEntry e = {-1, -1, 0, 0, 0, 0, 0};
         if (bal_np == 0) return e;
         const int b = (int)blockIdx.x;
         if (b < p.balanced) {                              // the last bal_len key tiles of item b
           if (n_done > 0) return e;
           Item it;
           const int pair = bal_np - 1 - b % bal_np;
-          if (!resolve_item(p, pair, it)) return e;
+          e.unit = find_unit(p, pair);
+          if (!resolve_item(p, pair, e.unit, it)) return e;
           e.pair = pair; e.chunk = b / bal_np;
           e.tile0 = max(0, it.n_tiles - p.bal_len);
           e.n_tiles = it.n_tiles - e.tile0;
@@ -468,6 +484,7 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
         e.split = 1 + ((int)blockIdx.x - p.balanced) - j_first;
         if (e.split >= p.n_splits) { ba_record_status(p.status, BA_ERR_SHAPE); return e; }
         e.pair = bal_np - 1 - i; e.chunk = chunk;
+        e.unit = find_unit(p, e.pair);
         e.tile0 = r - bal_cu[i]; e.n_tiles = n;
         e.fill = bal_pos + n == front_end ? e.split + 1 : p.n_splits;
         bal_pos += n;
@@ -485,7 +502,7 @@ ba_attend_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
         if (!ok) break;
         // balanced launch: the next piece of this CTA's share; persistent launch: next entry of the global list;
         // one-item launch: this CTA's own entry, then stop
-        WorkEntry e = {-1, 0, 0, 0, 0, 0};
+        WorkEntry e = {-1, -1, 0, 0, 0, 0, 0};
         if (tables_ok) {
           if (p.balanced) e = balanced_entry(n_work);
           else if (p.persistent) e = list_entry(p, atomicAdd(p.counters, 1));
