@@ -185,7 +185,12 @@ ba_status ba_last_device_status(ba_ctx *ctx) {
   BA_CUDA_TRY(cudaDeviceSynchronize());
   int32_t h = 0;
   BA_CUDA_TRY(cudaMemcpy(&h, ctx->dev_status, 4, cudaMemcpyDeviceToHost));
-  if (h != 0) BA_CUDA_TRY(cudaMemset(ctx->dev_status, 0, 4));
+  if (h != 0) {
+    BA_CUDA_TRY(cudaMemset(ctx->dev_status, 0, 4));
+    // a launch that gave up may have left its work counters half-way: back to zero for the next one
+    if (ctx->workspace && ctx->workspace_bytes >= ba_scratch_offset(ctx))
+      BA_CUDA_TRY(cudaMemset((char *)ctx->workspace + ba_scratch_offset(ctx) - 256, 0, 256));
+  }
   return (ba_status)h;
 }
 

@@ -576,6 +576,11 @@ def test_balanced_launch_parity(w, fused):
     o, lse, o_ref, lse_ref = run_warm(w, B.BA_MODE_BLOCK, fused=fused, shape_out=shapes)
     assert shapes[-1]["balanced_tails"] > 0 and shapes[-1]["partials"] >= 2, shapes
     check_attention(o, o_ref, lse, lse_ref)
+    if w.name == "balanced_two_sequences":
+        # whichever CTA merges an item's partial results, the sum runs in the same order: the same bits every time
+        for _ in range(3):
+            o2, lse2, _, _ = run_warm(w, B.BA_MODE_BLOCK, fused=fused)
+            assert np.array_equal(o, o2) and np.array_equal(lse, lse2)
 
 
 def test_warm_path_32k_full_size():
