@@ -96,6 +96,18 @@ def test_tables_bit_exact(w, mode):
     for k in TABLE_KEYS:
         assert got[k].tolist() == ref[k].tolist(), k
     assert got["totals"][0] == ref["n_cached_tokens"] and got["totals"][1] == ref["n_final_tokens"]
+    # host-side counts that size and balance the attention launches: work items, and the 128-key tiles the
+    # items of the final blocks see (cached keys in one run per sequence / a fresh tile per cached block)
+    tt = seg.q_tile_tokens
+    assert seg.n_prompt_items == sum(-(-n // tt) for n in w.block_lens)
+    packed, walked = [], []
+    for cached, fin in zip(w.cached_lens_per_seq(), w.final_lens()):
+        for r0 in range(0, fin, tt):
+            own = -(-min(fin, r0 + tt) // 128)
+            packed.append(-(-sum(cached) // 128) + own)
+            walked.append(sum(-(-n // 128) for n in cached) + own)
+    assert seg.n_final_items == len(packed)
+    assert list(seg.final_key_tiles) == [sum(packed), min(packed), max(packed), sum(walked), min(walked), max(walked)]
     c.close()
 
 
