@@ -504,11 +504,30 @@ def paged_case(w, page_rows, layer=0, layout=B.BA_ROPE_ADJACENT):
     return t, x, dev(k_pool), dev(v_pool), pages, (d_cu, d_idx), k_ref, o_ref, lse_ref
 
 
+def _balanced_cases():
+    """Final blocks over long caches with fewer work items than SMs: the launch gives one CTA the tail of each
+    item and lets the others share the key tiles in front (ragged cached blocks, ragged final blocks, two
+    sequences of unequal length, two head chunks per KV group, head_dim 64)."""
+    rng = np.random.default_rng(77)
+    one = [int(v) for v in rng.integers(300, 900, 20)] + [700]
+    two_a = [int(v) for v in rng.integers(200, 700, 20)] + [300]
+    two_b = [int(v) for v in rng.integers(200, 700, 23)] + [330]
+    d64 = [int(v) for v in rng.integers(500, 1500, 8)] + [1390]
+    return [W.Workload("balanced_one_sequence", 32, 8, 128, 5e5, one, [21], seed=81),
+            W.Workload("balanced_two_sequences", 32, 8, 128, 5e5, two_a + two_b, [21, 24], seed=82),
+            W.Workload("balanced_head_dim_64_two_chunks", 16, 2, 64, 1e4, d64, [9], seed=83)]
+
+
 PAGED_CASES = [(W.config1(), 16), (W.config2(), 16), (W.config2(), 64), (W.config2(), 128), (W.config2(), 256),
                (W.random_ragged(41, 3, 6, 300, 8, 2, 128), 32), (W.random_ragged(42, 5, 4, 200, 4, 2, 64), 16)]
 
 
-@pytest.mark.parametrize("w,page_rows", PAGED_CASES, ids=lambda v: v.name if hasattr(v, "name") else f"p{v}")
+def _paged_cases():
+    # a long cache under few work items: paged values and keys in the balanced launch
+    return PAGED_CASES + [(_balanced_cases()[0], 64)]
+
+
+@pytest.mark.parametrize("w,page_rows", _paged_cases(), ids=lambda v: v.name if hasattr(v, "name") else f"p{v}")
 def test_paged_cache_reencode_and_attend(w, page_rows):
     """Section 2.5 step 1 with a paged cache: cached keys gathered through the page table and re-encoded
     (ba_reencode_k_paged), values read from their pages in place by ba_final_attend_paged (one copy per
@@ -536,6 +555,8 @@ def test_paged_cache_reencode_and_attend(w, page_rows):
         k_re = None
     B.ba_final_attend_paged(c.ctx, q_f, k_f, v_f, Tf, k_re, Tc, v_pool, pages, o, lse, seg, B.BA_MODE_BLOCK, B.BA_OUT_F32)
     assert c.device_status() == B.BA_OK
+    if w.name.startswith("balanced"):
+        assert c.last_attend_shape()["balanced_tails"] > 0
     check_attention(o.cpu().numpy(), o_ref, lse.cpu().numpy(), lse_ref)
     o2 = torch.empty_like(o)
     k_out = torch.zeros_like(k_re) if Tc > 0 else None
@@ -565,20 +586,6 @@ def test_paged_cache_bad_page_numbers_are_reported_and_bad_sizes_refused():
                                   seg.cache_delta, seg.n_cached_blocks, 256)
         assert e.value.status == B.BA_ERR_UNSUPPORTED
     c.close()
-
-
-def _balanced_cases():
-    """Final blocks over long caches with fewer work items than SMs: the launch gives one CTA the tail of each
-    item and lets the others share the key tiles in front (ragged cached blocks, ragged final blocks, two
-    sequences of unequal length, two head chunks per KV group, head_dim 64)."""
-    rng = np.random.default_rng(77)
-    one = [int(v) for v in rng.integers(300, 900, 20)] + [700]
-    two_a = [int(v) for v in rng.integers(200, 700, 20)] + [300]
-    two_b = [int(v) for v in rng.integers(200, 700, 23)] + [330]
-    d64 = [int(v) for v in rng.integers(500, 1500, 8)] + [1390]
-    return [W.Workload("balanced_one_sequence", 32, 8, 128, 5e5, one, [21], seed=81),
-            W.Workload("balanced_two_sequences", 32, 8, 128, 5e5, two_a + two_b, [21, 24], seed=82),
-            W.Workload("balanced_head_dim_64_two_chunks", 16, 2, 64, 1e4, d64, [9], seed=83)]
 
 
 @pytest.mark.parametrize("w", _balanced_cases(), ids=lambda w: w.name)
