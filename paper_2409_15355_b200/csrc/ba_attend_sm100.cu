@@ -1315,7 +1315,7 @@ ba_status ba_attend_sm100_launch(ba_ctx *ctx, const ba_attend_args &a, const ba_
     // this very launch: the partial results must stay below it
     const size_t taken = ba_scratch_offset(ctx) + ctx->pending_table_bytes;
     const size_t avail = ctx->workspace_bytes > taken ? ctx->workspace_bytes - taken : 0;
-    const int cap = (int)min((size_t)16, per_split ? avail / per_split : 0);
+    const int cap = (int)min((size_t)32, per_split ? avail / per_split : 0);
     long long best = -1;
     for (int ns = 1; ns <= cap && ns <= avg_tiles; ++ns) {
       const long long waves = (items * ns + ctx->sm_count - 1) / ctx->sm_count;
