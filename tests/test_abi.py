@@ -58,3 +58,36 @@ def test_create_fails_loudly_without_a_device():
     with pytest.raises(B.BaError) as e:
         B.ba_create(cfg, 0, 1 << 20)
     assert e.value.status == B.BA_ERR_CUDA
+
+
+def test_struct_mirrors_match_the_header(tmp_path):
+    """The ctypes mirrors of the header's structs have the header's field names, order, offsets and sizes
+    (a C program compiled against include/ba.h prints them)."""
+    import shutil
+    import subprocess
+    gcc = shutil.which("gcc")
+    if gcc is None:
+        pytest.skip("no C compiler")
+    mirrors = {"ba_config": B.ba_config, "ba_segments": B.ba_segments, "ba_page_table": B.ba_page_table}
+    lines = ["#include <stdio.h>", "#include <stddef.h>", '#include "ba.h"', "int main(void) {"]
+    for name, cls in mirrors.items():
+        lines.append(f'  printf("{name} size %zu\\n", sizeof({name}));')
+        for field, _ in cls._fields_:
+            lines.append(f'  printf("{name} {field} %zu\\n", offsetof({name}, {field}));')
+    lines += ["  return 0;", "}"]
+    src = tmp_path / "layout.c"
+    src.write_text("\n".join(lines))
+    exe = tmp_path / "layout"
+    subprocess.run([gcc, "-I", os.path.join(ROOT, "include"), str(src), "-o", str(exe)], check=True)
+    out = subprocess.run([str(exe)], check=True, capture_output=True, text=True).stdout.split("\n")
+    got = {tuple(line.split()[:2]): int(line.split()[2]) for line in out if line}
+    for name, cls in mirrors.items():
+        assert got[(name, "size")] == C.sizeof(cls), name
+        for field, _ in cls._fields_:
+            assert got[(name, field)] == getattr(cls, field).offset, (name, field)
+    # no field of the header is missing from a mirror
+    text = re.sub(r"/\*.*?\*/", "", open(os.path.join(ROOT, "include", "ba.h")).read(), flags=re.S)
+    for name, cls in mirrors.items():
+        body = re.search(r"typedef struct \{([^}]*)\} " + name + ";", text).group(1)
+        fields = re.findall(r"\*?\b([a-z_0-9]+)(?:\[\d+\])?\s*[,;]", body)
+        assert [f for f, _ in cls._fields_] == fields, name
