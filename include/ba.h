@@ -160,6 +160,15 @@ int64_t ba_launch_count(const ba_ctx *ctx);
  * item in a balanced launch (0: not balanced), out[3] = key tiles of such a tail. */
 ba_status ba_last_attend_shape(const ba_ctx *ctx, int32_t out[4]);
 
+/* Diagnostic, no device needed: the planning step of ba_final_attend as a function of its inputs.  n_sms SMs,
+ * n_pairs work items per head chunk (ba_segments.n_final_items), n_head_chunks head chunks, avg_key_tiles 128-key
+ * tiles of an average item, key_tiles = {sum, minimum, maximum} of the key tiles over the n_pairs items (zeros:
+ * unknown), max_partials = the most partial results per row the workspace has room for.  out[0] = partial results
+ * per row (1: no split), out[1] = CTAs that take the tail of one item each (0: equal splits), out[2] = key tiles
+ * of such a tail. */
+ba_status ba_plan_final_attend(int32_t n_sms, int32_t n_pairs, int32_t n_head_chunks, int32_t avg_key_tiles,
+                               const int32_t key_tiles[3], int32_t max_partials, int32_t out[3]);
+
 /* Bytes of the table buffer ba_segment() needs for these sizes. */
 ba_status ba_segments_bytes(int32_t batch, int32_t n_blocks, int32_t n_tokens, size_t *bytes);
 

@@ -25,7 +25,7 @@ EXPORTS = [
     "ba_launch_count", "ba_segments_bytes", "ba_segment", "ba_reencode_k", "ba_block_prefill",
     "ba_final_attend", "ba_reencode_k_noalloc", "ba_selftest_wait_expiry", "ba_reencode_k_deferred", "ba_flush",
     "ba_final_attend_fused", "ba_reencode_k_paged", "ba_final_attend_paged", "ba_final_attend_fused_paged",
-    "ba_block_prefill_bwd", "ba_last_attend_shape",
+    "ba_block_prefill_bwd", "ba_last_attend_shape", "ba_plan_final_attend",
 ]
 BA_NOALLOC_MAX_BLOCKS = 4096
 
@@ -86,6 +86,7 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.ba_launch_count.argtypes = [vp]
     lib.ba_launch_count.restype = C.c_int64
     lib.ba_last_attend_shape.argtypes = [vp, C.POINTER(i32 * 4)]
+    lib.ba_plan_final_attend.argtypes = [i32, i32, i32, i32, C.POINTER(i32 * 3), i32, C.POINTER(i32 * 3)]
     lib.ba_segments_bytes.argtypes = [i32, i32, i32, C.POINTER(sz)]
     lib.ba_segment.argtypes = [vp, vp, vp, i32, i32, i32, C.c_int, vp, sz, C.POINTER(ba_segments), vp]
     lib.ba_reencode_k.argtypes = [vp, vp, vp, i32, vp, vp, vp, i32, i32, vp]
@@ -175,6 +176,16 @@ def ba_last_attend_shape(ctx) -> dict:
     out = (C.c_int32 * 4)()
     _check(load_library().ba_last_attend_shape(ctx, C.byref(out)), "ba_last_attend_shape")
     return {"ctas": out[0], "partials": out[1], "balanced_tails": out[2], "tail_tiles": out[3]}
+
+
+def ba_plan_final_attend(n_sms: int, n_pairs: int, n_head_chunks: int, avg_key_tiles: int, key_tiles,
+                         max_partials: int) -> dict:
+    """The planning step of ba_final_attend (host arithmetic only)."""
+    kt = (C.c_int32 * 3)(*[int(v) for v in key_tiles])
+    out = (C.c_int32 * 3)()
+    _check(load_library().ba_plan_final_attend(n_sms, n_pairs, n_head_chunks, avg_key_tiles, C.byref(kt), max_partials,
+                                               C.byref(out)), "ba_plan_final_attend")
+    return {"partials": out[0], "balanced_tails": out[1], "tail_tiles": out[2]}
 
 
 def ba_segments_bytes(batch: int, n_blocks: int, n_tokens: int) -> int:

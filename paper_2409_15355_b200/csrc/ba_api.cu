@@ -202,6 +202,15 @@ ba_status ba_last_attend_shape(const ba_ctx *ctx, int32_t out[4]) {
   return BA_OK;
 }
 
+ba_status ba_plan_final_attend(int32_t n_sms, int32_t n_pairs, int32_t n_head_chunks, int32_t avg_key_tiles,
+                               const int32_t key_tiles[3], int32_t max_partials, int32_t out[3]) {
+  if (!key_tiles || !out || n_sms < 1 || n_pairs < 1 || n_head_chunks < 1 || avg_key_tiles < 1) return BA_ERR_INVALID_ARG;
+  const ba_split_plan plan = ba_plan_splits(n_sms, (long long)n_pairs * n_head_chunks, n_pairs, n_head_chunks,
+                                            avg_key_tiles, key_tiles, max_partials);
+  out[0] = plan.n_splits; out[1] = plan.balanced; out[2] = plan.bal_len;
+  return BA_OK;
+}
+
 ba_status ba_segments_bytes(int32_t batch, int32_t n_blocks, int32_t n_tokens, size_t *bytes) {
   if (!bytes || batch < 1 || n_blocks < batch || n_tokens < n_blocks) return BA_ERR_INVALID_ARG;
   *bytes = table_layout(batch, n_blocks, n_tokens).bytes;

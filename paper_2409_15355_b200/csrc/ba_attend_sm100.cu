@@ -64,7 +64,7 @@ constexpr float kRescaleThreshold = 8.0f;
 constexpr int kBgStageBytes = 16384; // two spare warps x two stages of source rows
 constexpr int kWorkSlots = 4;      // ring of published work entries (power of two)
 constexpr int kBalTableOff = 512;  // balanced launch: prefix table of front tiles, in the control area behind Ctrl
-constexpr int kBalMaxPairs = 120;  // its capacity (items per head chunk); the spare warps' barriers follow at 1024
+// (its capacity, kBalMaxPairs items per head chunk, is declared with the planning arithmetic; the spare warps' barriers follow at 1024)
 // Register split after launch (168 per thread): the service warps give registers to the softmax warps.
 // 128 * kServiceRegs + 256 * kSoftmaxRegs <= 384 * 168.  The MMA thread keeps a work entry, descriptors
 // and ring positions live and spills below about 88; the softmax warps start to spill below 208.  On the
@@ -1316,34 +1316,9 @@ ba_status ba_attend_sm100_launch(ba_ctx *ctx, const ba_attend_args &a, const ba_
     const size_t taken = ba_scratch_offset(ctx) + ctx->pending_table_bytes;
     const size_t avail = ctx->workspace_bytes > taken ? ctx->workspace_bytes - taken : 0;
     const int cap = (int)min((size_t)32, per_split ? avail / per_split : 0);
-    long long best = -1;
-    for (int ns = 1; ns <= cap && ns <= avg_tiles; ++ns) {
-      const long long waves = (items * ns + ctx->sm_count - 1) / ctx->sm_count;
-      const long long cost = waves * ((avg_tiles + ns - 1) / ns + 3);
-      if (best < 0 || cost < best) { best = cost; n_splits = ns; }
-    }
-    // Balanced launch (item sizes known on the host, fewer items than SMs, every item longer than an SM's
-    // share of the tiles): one CTA per item takes the item's last `len` key tiles, the remaining CTAs share the
-    // tiles in front of those in equal runs.  `len` starts at the even share and grows until the CTAs that
-    // work on several pieces (each with its own start-up and write-out, counted as 3 tiles, plus 1 for their
-    // table) are no longer the slower ones.  Taken when the same cost model puts it ahead of equal splits.
-    const long long n_main = (long long)seg->n_final_items * (Hq / p.hpt);
-    const long long n_front = ctx->sm_count - n_main;
-    if (ft[0] > 0 && n_main > 0 && n_front > 0 && seg->n_final_items <= kBalMaxPairs) {
-      const long long total = (long long)ft[0] * (Hq / p.hpt), n_min = ft[1], n_max = ft[2];
-      for (long long len = (total + ctx->sm_count - 1) / ctx->sm_count; len <= n_min; ++len) {
-        const long long front = total - n_main * len;
-        if (front <= 0) break;
-        const long long run = (front + n_front - 1) / n_front, run_min = front / n_front;
-        if (run_min < 1) break;
-        const long long piece = (front + n_main - 1) / n_main;          // average front tiles of an item
-        const long long cost_front = run + 3 * ((run + piece - 1) / piece + 1) + 1;
-        if (cost_front > len + 3) continue;
-        const long long slots = 1 + (n_max - len + run_min - 1) / run_min + 1;
-        if (len + 3 < best && slots <= cap) { p.balanced = (int)n_main; p.bal_len = (int)len; n_splits = (int)slots; }
-        break;
-      }
-    }
+    // equal splits or the balanced launch (ba_plan_splits, above the kernels' common declarations)
+    const ba_split_plan plan = ba_plan_splits(ctx->sm_count, items, seg->n_final_items, Hq / p.hpt, avg_tiles, ft, cap);
+    n_splits = plan.n_splits; p.balanced = plan.balanced; p.bal_len = plan.bal_len;
   }
   p.n_splits = n_splits;
   p.n_chunks = Hq / p.hpt;

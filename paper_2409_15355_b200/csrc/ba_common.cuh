@@ -91,6 +91,49 @@ static inline size_t ba_align_up(size_t x, size_t a) { return (x + a - 1) / a * 
 // so the regions may be reused from call to call.
 static inline size_t ba_scratch_offset(const ba_ctx *) { return 64 * 1024; }
 
+// How ba_final_attend divides the key tiles of its work items among CTAs (pure host arithmetic, also reachable
+// through ba_plan_final_attend).  Inputs: SMs; work items (query tile pairs x head chunks); pairs and head chunks;
+// key tiles of an average item; sum / minimum / maximum of the key tiles over the pairs when known (else zeros);
+// the most partial results per row the workspace has room for.
+//  * Equal splits: n_splits entries per item, the count that minimises waves x (tiles per entry + 3), the 3
+//    standing for an entry's start-up and write-out.
+//  * Balanced launch (item sizes known, fewer items than SMs, every item longer than an SM's share of the tiles):
+//    one CTA per item takes the item's last `len` key tiles, the remaining CTAs share the tiles in front of those
+//    in equal runs.  `len` starts at the even share and grows until the CTAs that work on several pieces (each
+//    with its own start-up and write-out, plus 1 for their table) are no longer the slower ones.  Taken when the
+//    same cost model puts it ahead of equal splits; n_splits is then the number of partial results per row.
+constexpr int kBalMaxPairs = 120;        // the balanced launch keeps a prefix table of this many pairs in shared memory
+struct ba_split_plan { int n_splits, balanced, bal_len; };
+static inline ba_split_plan ba_plan_splits(int sm_count, long long items, int n_pairs, int n_chunks, long long avg_tiles,
+                                           const int32_t *key_tiles, int cap) {
+  ba_split_plan plan = {1, 0, 0};
+  if (items >= 2LL * sm_count || cap < 1) return plan;
+  long long best = -1;
+  for (int ns = 1; ns <= cap && ns <= avg_tiles; ++ns) {
+    const long long waves = (items * ns + sm_count - 1) / sm_count;
+    const long long cost = waves * ((avg_tiles + ns - 1) / ns + 3);
+    if (best < 0 || cost < best) { best = cost; plan.n_splits = ns; }
+  }
+  const long long n_main = (long long)n_pairs * n_chunks;
+  const long long n_front = sm_count - n_main;
+  if (key_tiles[0] > 0 && n_main > 0 && n_front > 0 && n_pairs <= kBalMaxPairs) {
+    const long long total = (long long)key_tiles[0] * n_chunks, n_min = key_tiles[1], n_max = key_tiles[2];
+    for (long long len = (total + sm_count - 1) / sm_count; len <= n_min; ++len) {
+      const long long front = total - n_main * len;
+      if (front <= 0) break;
+      const long long run = (front + n_front - 1) / n_front, run_min = front / n_front;
+      if (run_min < 1) break;
+      const long long piece = (front + n_main - 1) / n_main;          // average front tiles of an item
+      const long long cost_front = run + 3 * ((run + piece - 1) / piece + 1) + 1;
+      if (cost_front > len + 3) continue;
+      const long long slots = 1 + (n_max - len + run_min - 1) / run_min + 1;
+      if (len + 3 < best && slots <= cap) { plan.balanced = (int)n_main; plan.bal_len = (int)len; plan.n_splits = (int)slots; }
+      break;
+    }
+  }
+  return plan;
+}
+
 // Records the first device-side problem; later ones are dropped.
 __device__ __forceinline__ void ba_record_status(int32_t *status, int32_t code) {
   atomicCAS(status, 0, code);
