@@ -370,6 +370,7 @@ def run_ours(args):
     ms_local = ev0.elapsed_time(ev1) / args.steps
     clocks = sampler.stop()
     launches = ctx.launches() - launches0
+    attend_launch = ctx.last_attend_shape()      # how the library laid out the attention launches just timed
     assert ctx.device_status() == B.BA_OK
     ms, us_per_layer = aggregate(ms_local, float(L), dev)
 
@@ -568,7 +569,7 @@ def run_ours(args):
                     "peak_source": f"{peaks['source']} bf16 burst (cuBLAS 8192^3, best of 10)",
                     "frac_of_sustained": achieved / sustained if sustained else None,
                     "peak_sustained": sustained,
-                    "attend_us_per_launch": att_ms * 1e3,
+                    "attend_us_per_launch": att_ms * 1e3, "attend_launch": attend_launch,
                     "algorithmic_flops_per_launch": flops}
         # the metric itself: re-encode + attend of one layer against max(FLOPs / tensor peak, bytes / HBM peak)
         att_bytes = (2.0 * Tc * w.n_kv_heads + 2.0 * Tf * w.n_kv_heads + 2.0 * Tf * w.n_q_heads) * w.head_dim * 2
